@@ -1,0 +1,239 @@
+/*
+ * mole.h -- C ABI of the B200 (sm_100a) inference-time Mixture-of-Lookup-Experts layer
+ * (arXiv 2503.15798, "Mixture of Lookup Experts").
+ *
+ * What the layer computes (Eq. 4 and Eq. 8 of the paper, shared expert left to the caller):
+ * for every token t with hidden state h_t (d values) and input id i_t,
+ *
+ *     z_j   = sum_c h_t[c] * W_r[c][j]                     j = 0..N-1      (router logits)
+ *     g     = softmax(z)   over ALL N experts, no top-k                     (Eq. 4)
+ *     out_t = res_t + sum_j g_j * LUT[i_t][j][:]                            (Eq. 8)
+ *
+ * LUT is the per-layer table of pre-computed expert outputs of Eq. 6-7,
+ * LUT[i][j] = FFN_j(Embedding(i)), row-major [V][N][d]; res_t = h_t unless a separate
+ * residual is given.  Arithmetic: logits, softmax and the weighted sum are fp32; gates are
+ * never rounded below fp32; the only rounding to the storage type is at the store of out.
+ *
+ * Conventions shared by every entry point
+ *  - All functions return an int: MOLE_OK (0) or a positive MOLE_ERR_* code.  Nothing is
+ *    thrown, printed or aborted.  mole_status_string() names a code; mole_last_cuda_error()
+ *    gives the CUDA runtime's text for the calling thread's last MOLE_ERR_CUDA.
+ *  - "device" pointers are device memory of the CURRENT CUDA device; "host" pointers are
+ *    host memory.  The caller owns every buffer; the library allocates nothing except inside
+ *    mole_offload_create()/mole_host_alloc() (freed by their destroy/free calls).
+ *  - Calls are asynchronous: work is enqueued on `stream` (a cudaStream_t passed as void*,
+ *    NULL = the legacy default stream) and MOLE_OK means "enqueued".  No call synchronises
+ *    the device or the stream.
+ *  - Shapes: M = B*T tokens, flattened; position (b, t) uses ids[b*T + t], its own input id.
+ *    B*T == 0 is a successful no-op.  1 <= N <= 64, V >= 1, d a multiple of 8 (bf16) or
+ *    4 (fp32) so that every row piece is a whole number of 16-byte vectors.
+ *  - Alignment: hidden, residual, lut, w_router, out must be 16-byte aligned; ids 4-byte
+ *    (8-byte for 64-bit ids).
+ *  - Aliasing: out may be exactly hidden (in place).  Any other overlap of out with an input
+ *    is the caller's error and is not detected.
+ *  - An id outside [0, V) never reads out of bounds: that token gets out_t = res_t and, if a
+ *    status word was supplied, MOLE_STATUS_BAD_ID is OR-ed into it.
+ *  - Results are deterministic: no atomics in the arithmetic, fixed summation order, and a
+ *    token's result does not depend on the batch it is in.
+ */
+#ifndef MOLE_H
+#define MOLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOLE_VERSION 100
+
+/* every entry point is exported from the shared library with default visibility */
+#if defined(__GNUC__)
+#define MOLE_API __attribute__((visibility("default")))
+#else
+#define MOLE_API
+#endif
+
+/* return codes */
+#define MOLE_OK 0
+#define MOLE_ERR_INVALID_ARG 1       /* null / misaligned pointer, negative size, bad enum */
+#define MOLE_ERR_UNSUPPORTED_SHAPE 2 /* N outside 1..64, d not a multiple of the vector width, ... */
+#define MOLE_ERR_CUDA 3              /* a CUDA runtime call failed; see mole_last_cuda_error() */
+#define MOLE_ERR_NOMEM 4             /* an allocation inside create()/host_alloc() failed */
+#define MOLE_ERR_TOO_LARGE 5         /* size beyond a stated maximum */
+
+/* bits OR-ed by kernels into an optional device status word (uint32_t, caller zeroes it) */
+#define MOLE_STATUS_BAD_ID 1u  /* some id was outside [0, V) */
+#define MOLE_STATUS_TIMEOUT 2u /* a bounded wait inside a kernel gave up; output of that token not written */
+
+/* element type of hidden / residual / lut / w_router / out */
+#define MOLE_DTYPE_BF16 0
+#define MOLE_DTYPE_F32 1
+
+/* mole_args.flags */
+#define MOLE_FLAG_IDS_INT64 1u /* ids are int64_t instead of int32_t */
+#define MOLE_FLAG_CHAIN 2u     /* launch with programmatic dependent launch: the kernel may start, \
+                                  and may read ids / lut / w_router, before the previous kernel    \
+                                  on the stream has finished; it reads hidden / residual only      \
+                                  after it has.  Only valid if ids, lut and w_router are not       \
+                                  written by that previous kernel. */
+
+/* mole_args.variant: how a token's d columns are spread over thread blocks */
+#define MOLE_VARIANT_AUTO 0    /* chosen from M, N, d */
+#define MOLE_VARIANT_REPLICATE 1 /* each of d_split blocks recomputes the full router */
+#define MOLE_VARIANT_CLUSTER 2 /* d_split blocks form a cluster and exchange partial logits */
+
+/*
+ * mole_layer_forward -- the fused layer, bf16, Eq. 4 + Eq. 8 (router, softmax over all N
+ * experts, gather of the N rows selected by the id, fp32 weighted sum, residual add).
+ *   hidden   device, bf16 [B*T][d]          router input and residual
+ *   ids      device, int32 [B*T]            0 <= id < V
+ *   lut      device, bf16 [V][N][d]         one layer's table (Eq. 7)
+ *   w_router device, bf16 [d][N]            logits = hidden @ w_router  (a torch
+ *                                           nn.Linear(d, N).weight must be transposed)
+ *   out      device, bf16 [B*T][d]          may be == hidden
+ * Errors: MOLE_ERR_INVALID_ARG, MOLE_ERR_UNSUPPORTED_SHAPE, MOLE_ERR_CUDA; nothing is
+ * launched when an error is returned.
+ */
+MOLE_API int mole_layer_forward(const void *hidden, const int32_t *ids, const void *lut, const void *w_router,
+                       void *out, int B, int T, int N, int d, int V, void *stream);
+
+/*
+ * mole_layer_forward_ex -- the same operation with every option.  The appendix listing of
+ * the paper routes on the normalised hidden state but adds the un-normalised residual plus
+ * the shared expert's output; `residual` lets a caller do exactly that.
+ */
+typedef struct mole_args {
+    uint32_t struct_size;  /* sizeof(mole_args), checked */
+    uint32_t flags;        /* MOLE_FLAG_* */
+    const void *hidden;    /* device [M][d], dtype */
+    const void *ids;       /* device [M], int32 (int64 with MOLE_FLAG_IDS_INT64) */
+    const void *lut;       /* device [V][N][d], dtype */
+    const void *w_router;  /* device [d][N], dtype */
+    void *out;             /* device [M][d], dtype */
+    const void *residual;  /* device [M][d], dtype, or NULL => hidden.  Must not alias out unless it is hidden */
+    float *gates_out;      /* device [M][N] fp32 softmax weights, or NULL */
+    uint32_t *status;      /* device status word (MOLE_STATUS_* bits OR-ed in), or NULL */
+    int32_t B, T, N, d, V;
+    int32_t dtype;         /* MOLE_DTYPE_* */
+    int32_t variant;       /* MOLE_VARIANT_* */
+    int32_t d_split;       /* blocks per token (1, 2, 4 or 8; d/d_split must stay a multiple of the vector width); 0 = auto */
+    void *stream;          /* cudaStream_t */
+} mole_args;
+
+MOLE_API int mole_layer_forward_ex(const mole_args *args);
+
+/*
+ * mole_decode_step -- L layers back to back (Eq. 8 applied layer after layer; the attention
+ * and shared-expert blocks that a full model runs in between are not part of this library).
+ * Layer l reads table lut_base + l*lut_layer_stride_bytes and router w_router_base +
+ * l*wr_layer_stride_bytes; its output is the next layer's hidden.  Launches are chained with
+ * programmatic dependent launch, so layer l+1's row gathers (which depend only on ids) are in
+ * flight while layer l finishes.
+ *   hidden_in device [M][d], read only      out device [M][d] final result (may be == hidden_in
+ *   tmp       device [M][d] scratch for the ping-pong (may be NULL when L == 1)   only if L == 1)
+ * dtype as MOLE_DTYPE_*.  status (device, may be NULL) as in mole_args.
+ */
+MOLE_API int mole_decode_step(const void *hidden_in, const int32_t *ids, const void *lut_base,
+                     int64_t lut_layer_stride_bytes, const void *w_router_base,
+                     int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status, int L, int B,
+                     int T, int N, int d, int V, int dtype, void *stream);
+
+/*
+ * mole_decode_step_host -- mole_decode_step for a caller whose activations live in HOST
+ * memory: copies hidden_host and ids_host to the device buffers, runs the L layers, copies
+ * the result to out_host, all on `stream` (asynchronous when the host buffers are pinned).
+ *   hidden_host, out_host  host [M][d]      ids_host host int32 [M]
+ *   dev_hidden, dev_out, dev_tmp device [M][d] scratch owned by the caller; dev_ids device int32 [M]
+ * The result is in out_host once the stream has been synchronised.
+ */
+MOLE_API int mole_decode_step_host(const void *hidden_host, const int32_t *ids_host, void *out_host, void *dev_hidden,
+                          int32_t *dev_ids, void *dev_out, void *dev_tmp, const void *lut_base,
+                          int64_t lut_layer_stride_bytes, const void *w_router_base,
+                          int64_t wr_layer_stride_bytes, uint32_t *status, int L, int B, int T, int N, int d,
+                          int V, int dtype, void *stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Offload mode: the table stays in pinned host memory (the paper keeps it "offloaded to the
+ * storage device" and moves only the looked-up rows, Sec. 3.3 and the inference listing).
+ * Per step the distinct ids are found on the device and only their rows cross the host link.
+ * ------------------------------------------------------------------------------------- */
+
+/*
+ * mole_dedup_ids -- distinct ids of one step.
+ *   ids     device int32 [M]
+ *   scratch device int32 [V]; must be all zero on entry (zero it once after allocation);
+ *           the kernel leaves it all zero again.  Calls sharing one scratch array must not
+ *           overlap on the GPU.
+ *   uniq    device int32 [>= min(M, V)]: the distinct in-range ids, in order of first occurrence
+ *   slot    device int32 [M]: uniq[slot[t]] == ids[t]; -1 for an id outside [0, V)
+ *   count   device int32 [1]: number of distinct in-range ids
+ * M <= MOLE_DEDUP_MAX_TOKENS.  M == 0 writes count = 0.
+ */
+#define MOLE_DEDUP_MAX_TOKENS (1 << 20)
+MOLE_API int mole_dedup_ids(const int32_t *ids, int M, int V, int32_t *scratch, int32_t *uniq, int32_t *slot,
+                   int32_t *count, uint32_t *status, void *stream);
+
+/*
+ * mole_fetch_rows -- copy rows uniq[0..count) of a table in pinned, device-mapped host
+ * memory into a dense device staging buffer: staging[u] = lut_host[uniq[u]] (row_bytes each,
+ * a multiple of 16).  The reads are issued by the GPU across the host link; `count` is read on
+ * the device, so there is no host round trip.  lut_host is the HOST pointer of memory from
+ * mole_host_alloc() / cudaHostAlloc / cudaHostRegister; max_rows bounds the launch
+ * (count <= max_rows, staging holds max_rows rows).
+ */
+MOLE_API int mole_fetch_rows(const void *lut_host, const int32_t *uniq, const int32_t *count, int max_rows,
+                    int64_t row_bytes, void *staging, void *stream);
+
+/* pinned, device-mapped host memory for a table (cudaHostAlloc); free with mole_host_free */
+MOLE_API int mole_host_alloc(void **ptr, size_t bytes);
+MOLE_API int mole_host_free(void *ptr);
+
+/*
+ * Offload context: owns n_buffers staging buffers [max_tokens][N][d], their uniq / slot /
+ * count arrays, one V-entry dedup scratch table and the events that order the side stream
+ * against the main stream.  Not thread-safe; use one context per decoding stream.
+ */
+typedef struct mole_offload_ctx mole_offload_ctx;
+
+MOLE_API int mole_offload_create(mole_offload_ctx **ctx, int max_tokens, int N, int d, int V, int dtype, int n_buffers);
+MOLE_API int mole_offload_destroy(mole_offload_ctx *ctx);
+
+/*
+ * mole_offload_prefetch -- on side_stream: wait until buffer `buf`'s previous consumer has
+ * finished, deduplicate ids (device), fetch the distinct rows of lut_host_layer (HOST pointer,
+ * pinned + mapped, [V][N][d]) into the buffer's staging area, record the buffer's ready event.
+ * ids must stay unchanged until the work has run.
+ */
+MOLE_API int mole_offload_prefetch(mole_offload_ctx *ctx, int buf, const int32_t *ids, int M, const void *lut_host_layer,
+                          void *side_stream);
+
+/*
+ * mole_layer_forward_offload -- on stream: wait for buffer `buf`'s ready event, run the fused
+ * layer with the gather reading staging[slot[t]], record the buffer's consumed event.
+ * B*T must equal the M given to the matching prefetch.  Output is bit-identical to
+ * mole_layer_forward on the same inputs.
+ */
+MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const void *hidden, const void *w_router, void *out,
+                               uint32_t *status, int B, int T, void *stream);
+
+/* device pointers of a buffer's arrays, for inspection: uniq [max_tokens], slot [max_tokens], count [1], staging */
+MOLE_API int mole_offload_buffers(mole_offload_ctx *ctx, int buf, const int32_t **uniq, const int32_t **slot,
+                         const int32_t **count, const void **staging);
+
+/* --------------------------------------------------------------------------------------- */
+
+MOLE_API const char *mole_status_string(int code);
+MOLE_API const char *mole_last_cuda_error(void);
+MOLE_API int mole_version(void);
+
+/* launch shape mole_layer_forward_ex would pick (for tests and benchmarks): blocks per token,
+ * threads per block, dynamic shared memory, variant.  Pure host arithmetic, no CUDA call. */
+MOLE_API int mole_plan(int M, int N, int d, int dtype, int variant, int d_split, int *out_d_split, int *out_threads,
+              int *out_smem_bytes, int *out_variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOLE_H */

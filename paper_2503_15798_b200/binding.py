@@ -1,0 +1,303 @@
+"""Python face of the C-ABI library declared in ``include/mole.h``.
+
+Argument marshalling only: every function takes torch tensors (used for device memory and
+streams, nothing else), checks shapes and dtypes, and passes raw pointers and sizes to the
+entry point of the same name.  No arithmetic of the layer happens here, and there is no
+fallback: if ``libmole_b200.so`` has not been built, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmole_b200.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, ERR_NOMEM, ERR_TOO_LARGE = range(6)
+STATUS_BAD_ID, STATUS_TIMEOUT = 1, 2
+DTYPE_BF16, DTYPE_F32 = 0, 1
+FLAG_IDS_INT64, FLAG_CHAIN = 1, 2
+VARIANT_AUTO, VARIANT_REPLICATE, VARIANT_CLUSTER = 0, 1, 2
+
+# every symbol include/mole.h declares
+EXPORTS = (
+    "mole_layer_forward", "mole_layer_forward_ex", "mole_decode_step", "mole_decode_step_host",
+    "mole_dedup_ids", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
+    "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_buffers",
+    "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan",
+)
+
+
+class MoleArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", c_uint32), ("flags", c_uint32),
+        ("hidden", c_void_p), ("ids", c_void_p), ("lut", c_void_p), ("w_router", c_void_p), ("out", c_void_p),
+        ("residual", c_void_p), ("gates_out", c_void_p), ("status", c_void_p),
+        ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
+        ("dtype", c_int32), ("variant", c_int32), ("d_split", c_int32),
+        ("stream", c_void_p),
+    ]
+
+
+class MoleError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().mole_status_string(code).decode()
+        if code == ERR_CUDA:
+            msg += ": " + lib().mole_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} (code {code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if it is missing -- there is no other implementation."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2503_15798_b200.build` "
+                "(nvcc, sm_100a); this package has no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ip = c_void_p, c_void_p
+        L.mole_layer_forward.argtypes = [vp, ip, vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp]
+        L.mole_layer_forward_ex.argtypes = [POINTER(MoleArgs)]
+        L.mole_decode_step.argtypes = [vp, ip, vp, c_int64, vp, c_int64, vp, vp, vp, c_int, c_int, c_int, c_int,
+                                       c_int, c_int, c_int, vp]
+        L.mole_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, c_int64, vp, c_int64, vp, c_int, c_int,
+                                            c_int, c_int, c_int, c_int, c_int, vp]
+        L.mole_dedup_ids.argtypes = [ip, c_int, c_int, ip, ip, ip, ip, vp, vp]
+        L.mole_fetch_rows.argtypes = [vp, ip, ip, c_int, c_int64, vp, vp]
+        L.mole_host_alloc.argtypes = [POINTER(c_void_p), c_size_t]
+        L.mole_host_free.argtypes = [vp]
+        L.mole_offload_create.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_int]
+        L.mole_offload_destroy.argtypes = [vp]
+        L.mole_offload_prefetch.argtypes = [vp, c_int, ip, c_int, vp, vp]
+        L.mole_layer_forward_offload.argtypes = [vp, c_int, vp, vp, vp, vp, c_int, c_int, vp]
+        L.mole_offload_buffers.argtypes = [vp, c_int, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
+                                           POINTER(c_void_p)]
+        L.mole_status_string.argtypes = [c_int]
+        L.mole_status_string.restype = c_char_p
+        L.mole_last_cuda_error.argtypes = []
+        L.mole_last_cuda_error.restype = c_char_p
+        L.mole_version.argtypes = []
+        L.mole_plan.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
+                                POINTER(c_int), POINTER(c_int)]
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if fn.restype is not c_char_p:
+                fn.restype = c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise MoleError(code, where)
+
+
+def _dtype_tag(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    raise TypeError(f"unsupported element type {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _dev(t: torch.Tensor, name: str):
+    if not (t.is_cuda and t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+
+
+def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_out=None, status=None,
+                  variant: int = VARIANT_AUTO, d_split: int = 0, chain: bool = False, stream=None, B=None, T=None):
+    """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d],
+    w_router [d][N]; returns out (allocated like hidden if not given)."""
+    for name, t in (("hidden", hidden), ("ids", ids), ("lut", lut), ("w_router", w_router)):
+        _dev(t, name)
+    V, N, d = lut.shape
+    M = hidden.numel() // d if d else 0
+    if hidden.shape[-1] != d or tuple(w_router.shape) != (d, N) or ids.numel() != M:
+        raise ValueError("shape mismatch between hidden, ids, lut and w_router")
+    tag = _dtype_tag(hidden)
+    if not (lut.dtype == w_router.dtype == hidden.dtype):
+        raise TypeError("hidden, lut and w_router must share one element type")
+    if out is None:
+        out = torch.empty_like(hidden)
+    _dev(out, "out")
+    flags = 0
+    if ids.dtype == torch.int64:
+        flags |= FLAG_IDS_INT64
+    elif ids.dtype != torch.int32:
+        raise TypeError("ids must be int32 or int64")
+    if chain:
+        flags |= FLAG_CHAIN
+    if B is None:
+        B, T = M, 1
+    a = MoleArgs()
+    a.struct_size = ctypes.sizeof(MoleArgs)
+    a.flags = flags
+    a.hidden, a.ids, a.lut, a.w_router, a.out = _ptr(hidden), _ptr(ids), _ptr(lut), _ptr(w_router), _ptr(out)
+    a.residual, a.gates_out, a.status = _ptr(residual), _ptr(gates_out), _ptr(status)
+    a.B, a.T, a.N, a.d, a.V = B, T, N, d, V
+    a.dtype, a.variant, a.d_split = tag, variant, d_split
+    a.stream = _stream(stream)
+    _check(lib().mole_layer_forward_ex(ctypes.byref(a)), "mole_layer_forward_ex")
+    return out
+
+
+def layer_forward_basic(hidden, ids, lut, w_router, out, stream=None):
+    """mole_layer_forward (bf16, int32 ids), the plain entry point."""
+    V, N, d = lut.shape
+    M = ids.numel()
+    _check(lib().mole_layer_forward(_ptr(hidden), _ptr(ids), _ptr(lut), _ptr(w_router), _ptr(out), M, 1, N, d, V,
+                                    _stream(stream)), "mole_layer_forward")
+    return out
+
+
+def decode_step(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None):
+    """mole_decode_step: luts [L][V][N][d], w_routers [L][d][N]; returns out."""
+    L, V, N, d = luts.shape
+    M = ids.numel()
+    tag = _dtype_tag(hidden_in)
+    _check(lib().mole_decode_step(_ptr(hidden_in), _ptr(ids), _ptr(luts), luts.stride(0) * luts.element_size(),
+                                  _ptr(w_routers), w_routers.stride(0) * w_routers.element_size(), _ptr(out),
+                                  _ptr(tmp), _ptr(status), L, M, 1, N, d, V, tag, _stream(stream)),
+           "mole_decode_step")
+    return out
+
+
+def decode_step_host(hidden_host, ids_host, out_host, dev_hidden, dev_ids, dev_out, dev_tmp, luts, w_routers,
+                     status=None, stream=None):
+    """mole_decode_step_host: activations in (pinned) host tensors, tables on the device."""
+    L, V, N, d = luts.shape
+    M = ids_host.numel()
+    tag = _dtype_tag(dev_hidden)
+    _check(lib().mole_decode_step_host(_ptr(hidden_host), _ptr(ids_host), _ptr(out_host), _ptr(dev_hidden),
+                                       _ptr(dev_ids), _ptr(dev_out), _ptr(dev_tmp), _ptr(luts),
+                                       luts.stride(0) * luts.element_size(), _ptr(w_routers),
+                                       w_routers.stride(0) * w_routers.element_size(), _ptr(status), L, M, 1, N, d,
+                                       V, tag, _stream(stream)), "mole_decode_step_host")
+    return out_host
+
+
+def dedup_ids(ids, V: int, scratch, uniq, slot, count, status=None, stream=None):
+    """mole_dedup_ids: all tensors int32 on the device; scratch [V] must be zero on entry."""
+    _check(lib().mole_dedup_ids(_ptr(ids), ids.numel(), V, _ptr(scratch), _ptr(uniq), _ptr(slot), _ptr(count),
+                                _ptr(status), _stream(stream)), "mole_dedup_ids")
+
+
+def fetch_rows(lut_host, uniq, count, max_rows: int, staging, stream=None):
+    """mole_fetch_rows: lut_host is a pinned host tensor [V][N][d]; staging a device tensor."""
+    row_bytes = lut_host[0].numel() * lut_host.element_size()
+    _check(lib().mole_fetch_rows(_ptr(lut_host), _ptr(uniq), _ptr(count), max_rows, row_bytes, _ptr(staging),
+                                 _stream(stream)), "mole_fetch_rows")
+
+
+class _DevicePointer:
+    """Lets torch view memory the library owns (CUDA array interface, no copy)."""
+
+    def __init__(self, ptr: int, shape, typestr: str):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False),
+                                         "version": 2}
+
+
+def _wrap_device(ptr: int, shape, typestr: str) -> torch.Tensor:
+    return torch.as_tensor(_DevicePointer(ptr, shape, typestr), device="cuda")
+
+
+class HostTable:
+    """A pinned, device-mapped host allocation from mole_host_alloc, viewed as a torch tensor."""
+
+    def __init__(self, shape, dtype=torch.bfloat16):
+        n = 1
+        for s in shape:
+            n *= s
+        self.nbytes = n * torch.empty((), dtype=dtype).element_size()
+        p = c_void_p()
+        _check(lib().mole_host_alloc(ctypes.byref(p), self.nbytes), "mole_host_alloc")
+        self.ptr = p.value
+        buf = (ctypes.c_uint8 * self.nbytes).from_address(self.ptr)
+        self.tensor = torch.frombuffer(buf, dtype=torch.uint8).view(dtype).view(*shape)
+
+    def free(self):
+        if self.ptr:
+            self.tensor = None
+            _check(lib().mole_host_free(self.ptr), "mole_host_free")
+            self.ptr = None
+
+
+class OffloadContext:
+    """mole_offload_create / prefetch / forward / destroy."""
+
+    def __init__(self, max_tokens: int, N: int, d: int, V: int, dtype=torch.bfloat16, n_buffers: int = 2):
+        self.max_tokens, self.N, self.d, self.V, self.dtype, self.n_buffers = max_tokens, N, d, V, dtype, n_buffers
+        tag = DTYPE_BF16 if dtype == torch.bfloat16 else DTYPE_F32
+        h = c_void_p()
+        _check(lib().mole_offload_create(ctypes.byref(h), max_tokens, N, d, V, tag, n_buffers), "mole_offload_create")
+        self.handle = h.value
+
+    def prefetch(self, buf: int, ids, lut_host_layer, side_stream=None):
+        _check(lib().mole_offload_prefetch(self.handle, buf, _ptr(ids), ids.numel(), _ptr(lut_host_layer),
+                                           _stream(side_stream)), "mole_offload_prefetch")
+
+    def forward(self, buf: int, hidden, w_router, out, status=None, stream=None):
+        M = hidden.numel() // self.d
+        _check(lib().mole_layer_forward_offload(self.handle, buf, _ptr(hidden), _ptr(w_router), _ptr(out),
+                                                _ptr(status), M, 1, _stream(stream)), "mole_layer_forward_offload")
+        return out
+
+    def buffers(self, buf: int):
+        """(uniq, slot, count, staging) device pointers of a buffer, as ints."""
+        u, s, c, g = c_void_p(), c_void_p(), c_void_p(), c_void_p()
+        _check(lib().mole_offload_buffers(self.handle, buf, ctypes.byref(u), ctypes.byref(s), ctypes.byref(c),
+                                          ctypes.byref(g)), "mole_offload_buffers")
+        return u.value, s.value, c.value, g.value
+
+    def read_buffer(self, buf: int):
+        """Host copies of a buffer's (uniq[:count], slot[:max_tokens], count); synchronises."""
+        u, s, c, _ = self.buffers(buf)
+        torch.cuda.synchronize()
+        n = int(_wrap_device(c, (1,), "<i4").cpu().item())
+        uniq = _wrap_device(u, (self.max_tokens,), "<i4").cpu()
+        slot = _wrap_device(s, (self.max_tokens,), "<i4").cpu()
+        return uniq[:n].clone(), slot, n
+
+    def destroy(self):
+        if self.handle:
+            _check(lib().mole_offload_destroy(self.handle), "mole_offload_destroy")
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def plan(M: int, N: int, d: int, dtype: int = DTYPE_BF16, variant: int = VARIANT_AUTO, d_split: int = 0):
+    """mole_plan: (d_split, threads, smem_bytes, variant) the launch would use."""
+    a, b, c, e = c_int(), c_int(), c_int(), c_int()
+    _check(lib().mole_plan(M, N, d, dtype, variant, d_split, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                           ctypes.byref(e)), "mole_plan")
+    return a.value, b.value, c.value, e.value
+
+
+def version() -> int:
+    return lib().mole_version()

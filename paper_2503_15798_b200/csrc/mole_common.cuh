@@ -1,0 +1,200 @@
+// Shared device helpers and host-side error plumbing of the MoLE sm_100a library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mole.h"
+
+namespace mole {
+
+// ---- host side -----------------------------------------------------------------------------
+void set_cuda_error(cudaError_t e);  // remembers the text for mole_last_cuda_error()
+
+#define MOLE_CUDA_TRY(expr)                       \
+    do {                                          \
+        cudaError_t e__ = (expr);                 \
+        if (e__ != cudaSuccess) {                 \
+            ::mole::set_cuda_error(e__);          \
+            return MOLE_ERR_CUDA;                 \
+        }                                         \
+    } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int elem_bytes(int dtype) { return dtype == MOLE_DTYPE_BF16 ? 2 : 4; }
+
+// Launch description of the fused layer kernel (filled by plan_layer, pure host arithmetic).
+struct LayerPlan {
+    int d_split;   // blocks per token
+    int dc;        // columns per block
+    int threads;   // threads per block
+    int smem;      // dynamic shared memory, bytes
+    int variant;   // MOLE_VARIANT_REPLICATE or MOLE_VARIANT_CLUSTER (d_split == 1 => REPLICATE)
+    int n_fast;    // N if the unrolled router path exists for it, else 0
+};
+int plan_layer(long long M, int N, int d, int dtype, int variant, int d_split, LayerPlan *plan);
+
+// One fused-layer launch; `row_index` is ids (resident mode) or slot (offload mode) and
+// `rows` the number of rows of `lut` that may be addressed.
+struct LayerLaunch {
+    const void *hidden, *residual, *row_index, *lut, *w_router;
+    void *out;
+    float *gates_out;
+    uint32_t *status;
+    long long M;
+    int N, d;
+    long long rows;
+    int dtype;
+    uint32_t flags;
+    int variant, d_split;
+    cudaStream_t stream;
+};
+int launch_layer(const LayerLaunch &L);
+
+#ifdef __CUDACC__
+// ---- device side ---------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// mbarrier + bulk-copy (TMA, untiled, no multicast) primitives
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Global -> this block's shared memory; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Bounded wait on a bulk-copy barrier.  Returns false if the data never arrived.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint32_t max_polls)
+{
+    for (uint32_t i = 0; i < max_polls; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) __nanosleep(64);
+    }
+    return false;
+}
+
+// programmatic dependent launch
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// thread-block cluster
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_f32(uint32_t local_smem_addr, uint32_t cta, float v)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(cta));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// 16-byte vectors of the two storage types
+template <typename T>
+struct Elem;
+template <>
+struct Elem<__nv_bfloat16> {
+    static constexpr int VEC = 8;
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&f)[8])
+    {
+        f[0] = __uint_as_float(v.x << 16);
+        f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16);
+        f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16);
+        f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16);
+        f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[8])
+    {
+        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]);
+        __nv_bfloat162 b = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(f[4], f[5]);
+        __nv_bfloat162 e = __floats2bfloat162_rn(f[6], f[7]);
+        uint4 v;
+        v.x = *reinterpret_cast<uint32_t *>(&a);
+        v.y = *reinterpret_cast<uint32_t *>(&b);
+        v.z = *reinterpret_cast<uint32_t *>(&c);
+        v.w = *reinterpret_cast<uint32_t *>(&e);
+        return v;
+    }
+    static __device__ __forceinline__ float scalar(const void *p, long long i)
+    {
+        return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p)[i]);
+    }
+    // L2-only load: for data another kernel wrote shortly before (never served from a stale L1 line)
+    static __device__ __forceinline__ float scalar_cg(const void *p, long long i)
+    {
+        const uint32_t bits = __ldcg(reinterpret_cast<const unsigned short *>(p) + i);
+        return __uint_as_float(bits << 16);
+    }
+};
+template <>
+struct Elem<float> {
+    static constexpr int VEC = 4;
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&f)[4])
+    {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[4])
+    {
+        uint4 v;
+        v.x = __float_as_uint(f[0]);
+        v.y = __float_as_uint(f[1]);
+        v.z = __float_as_uint(f[2]);
+        v.w = __float_as_uint(f[3]);
+        return v;
+    }
+    static __device__ __forceinline__ float scalar(const void *p, long long i)
+    {
+        return reinterpret_cast<const float *>(p)[i];
+    }
+    static __device__ __forceinline__ float scalar_cg(const void *p, long long i)
+    {
+        return __ldcg(reinterpret_cast<const float *>(p) + i);
+    }
+};
+#endif  // __CUDACC__
+
+}  // namespace mole

@@ -1,0 +1,336 @@
+// Offload mode of the MoLE layer: the table stays in pinned host memory (the paper keeps the
+// re-parameterised table on a storage device and moves only the looked-up rows, Sec. 3.3);
+// per step the distinct ids are found on the device, their rows are read across the host
+// link by the GPU itself into a dense staging buffer, and the fused layer gathers from there.
+#include <new>
+#include <string.h>
+
+#include "mole_common.cuh"
+
+namespace mole {
+
+constexpr int kDedupThreads = 1024;
+constexpr int kFetchThreads = 256;
+constexpr int kFetchVecPerThread = 4;  // 16-byte loads in flight per thread
+constexpr int kFetchChunk = kFetchThreads * kFetchVecPerThread * 16;
+
+// Distinct ids of a step, one thread block.  table[V] is all zero on entry and on exit.
+//  1. table[id] = max over the id's tokens of (M - t): the first occurrence wins.
+//  2. tokens that won are the representatives; an ordered block scan numbers them, so uniq
+//     comes out in order of first occurrence and the result does not depend on timing.
+//  3. every token copies its representative's number; representatives clear their table entry.
+__global__ void __launch_bounds__(kDedupThreads) mole_dedup_kernel(const int32_t *__restrict__ ids, int M, int V,
+                                                                   int32_t *table, int32_t *uniq, int32_t *slot,
+                                                                   int32_t *count, uint32_t *status)
+{
+    __shared__ int warp_tot[kDedupThreads / 32];
+    __shared__ int total;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int per = (M + nt - 1) / nt;  // contiguous run of tokens per thread
+    const int t0 = min(tid * per, M), t1 = min(t0 + per, M);
+    bool bad = false;
+
+    for (int t = t0; t < t1; ++t) {
+        const int id = ids[t];
+        if (id >= 0 && id < V) atomicMax(&table[id], M - t);
+        else bad = true;
+    }
+    __syncthreads();
+
+    int mine = 0;
+    for (int t = t0; t < t1; ++t) {
+        const int id = ids[t];
+        if (id >= 0 && id < V && table[id] == M - t) ++mine;
+    }
+    // exclusive scan of `mine` over the block
+    const int lane = tid & 31, warp = tid >> 5;
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < nt / 32) ? warp_tot[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += v;
+        }
+        if (lane < nt / 32) warp_tot[lane] = wi - w;
+        if (lane == 31) total = wi;
+    }
+    __syncthreads();
+    int pos = warp_tot[warp] + incl - mine;
+    for (int t = t0; t < t1; ++t) {
+        const int id = ids[t];
+        if (id >= 0 && id < V && table[id] == M - t) {
+            uniq[pos] = id;
+            slot[t] = pos;
+            ++pos;
+        }
+    }
+    __syncthreads();
+    for (int t = t0; t < t1; ++t) {
+        const int id = ids[t];
+        if (id >= 0 && id < V) {
+            const int rep = M - table[id];
+            if (rep != t) slot[t] = slot[rep];
+        } else {
+            slot[t] = -1;
+        }
+    }
+    __syncthreads();
+    for (int t = t0; t < t1; ++t) {
+        const int id = ids[t];
+        if (id >= 0 && id < V && table[id] == M - t) table[id] = 0;
+    }
+    if (tid == 0) *count = total;
+    if (bad && status) atomicOr(status, MOLE_STATUS_BAD_ID);
+}
+
+// staging[u] = table_host[uniq[u]] for u < *count.  blockIdx.y = u, blockIdx.x = 16 KB chunk of
+// the row.  All of a thread's loads are issued before its first store so that many reads are
+// in flight on the host link.
+__global__ void __launch_bounds__(kFetchThreads) mole_fetch_kernel(const unsigned char *__restrict__ table_host,
+                                                                   const int32_t *__restrict__ uniq,
+                                                                   const int32_t *__restrict__ count, long long row_bytes,
+                                                                   unsigned char *__restrict__ staging)
+{
+    const int u = blockIdx.y;
+    if (u >= *count) return;
+    const long long row = uniq[u];
+    const long long chunk0 = static_cast<long long>(blockIdx.x) * kFetchChunk;
+    const uint4 *src = reinterpret_cast<const uint4 *>(table_host + row * row_bytes + chunk0);
+    uint4 *dst = reinterpret_cast<uint4 *>(staging + static_cast<long long>(u) * row_bytes + chunk0);
+    const long long nvec = min(static_cast<long long>(kFetchChunk), row_bytes - chunk0) / 16;
+    uint4 v[kFetchVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kFetchVecPerThread; ++k) {
+        const long long i = static_cast<long long>(k) * kFetchThreads + threadIdx.x;
+        if (i < nvec) v[k] = __ldcs(src + i);
+    }
+#pragma unroll
+    for (int k = 0; k < kFetchVecPerThread; ++k) {
+        const long long i = static_cast<long long>(k) * kFetchThreads + threadIdx.x;
+        if (i < nvec) dst[i] = v[k];
+    }
+}
+
+static int launch_dedup(const int32_t *ids, int M, int V, int32_t *scratch, int32_t *uniq, int32_t *slot, int32_t *count,
+                        uint32_t *status, cudaStream_t st)
+{
+    mole_dedup_kernel<<<1, kDedupThreads, 0, st>>>(ids, M, V, scratch, uniq, slot, count, status);
+    MOLE_CUDA_TRY(cudaGetLastError());
+    return MOLE_OK;
+}
+
+static int launch_fetch(const void *lut_host, const int32_t *uniq, const int32_t *count, int max_rows, long long row_bytes,
+                        void *staging, cudaStream_t st)
+{
+    void *dev_alias = nullptr;
+    MOLE_CUDA_TRY(cudaHostGetDevicePointer(&dev_alias, const_cast<void *>(lut_host), 0));
+    dim3 grid(static_cast<unsigned>((row_bytes + kFetchChunk - 1) / kFetchChunk), static_cast<unsigned>(max_rows), 1);
+    mole_fetch_kernel<<<grid, kFetchThreads, 0, st>>>(static_cast<const unsigned char *>(dev_alias), uniq, count, row_bytes,
+                                                      static_cast<unsigned char *>(staging));
+    MOLE_CUDA_TRY(cudaGetLastError());
+    return MOLE_OK;
+}
+
+}  // namespace mole
+
+using namespace mole;
+
+struct mole_offload_ctx {
+    int max_tokens, N, d, V, dtype, n_buffers;
+    long long row_bytes;
+    int32_t *table;  // [V] dedup scratch, kept all zero between kernels
+    struct Buffer {
+        unsigned char *staging;  // [max_tokens][N][d]
+        int32_t *uniq, *slot, *count;
+        cudaEvent_t ready, consumed;
+        int M;  // tokens of the prefetch in flight
+    } *buf;
+};
+
+extern "C" {
+
+int mole_dedup_ids(const int32_t *ids, int M, int V, int32_t *scratch, int32_t *uniq, int32_t *slot, int32_t *count,
+                   uint32_t *status, void *stream)
+{
+    if (M < 0 || V < 1) return MOLE_ERR_INVALID_ARG;
+    if (M > MOLE_DEDUP_MAX_TOKENS) return MOLE_ERR_TOO_LARGE;
+    if (!count || !scratch || (M > 0 && (!ids || !uniq || !slot))) return MOLE_ERR_INVALID_ARG;
+    return launch_dedup(ids, M, V, scratch, uniq, slot, count, status, static_cast<cudaStream_t>(stream));
+}
+
+int mole_fetch_rows(const void *lut_host, const int32_t *uniq, const int32_t *count, int max_rows, int64_t row_bytes,
+                    void *staging, void *stream)
+{
+    if (max_rows < 0 || row_bytes < 16 || (row_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if (max_rows == 0) return MOLE_OK;
+    if (max_rows > 65535) return MOLE_ERR_TOO_LARGE;
+    if (!lut_host || !uniq || !count || !staging || !aligned16(lut_host) || !aligned16(staging)) return MOLE_ERR_INVALID_ARG;
+    return launch_fetch(lut_host, uniq, count, max_rows, row_bytes, staging, static_cast<cudaStream_t>(stream));
+}
+
+int mole_host_alloc(void **ptr, size_t bytes)
+{
+    if (!ptr || bytes == 0) return MOLE_ERR_INVALID_ARG;
+    *ptr = nullptr;
+    cudaError_t e = cudaHostAlloc(ptr, bytes, cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e == cudaErrorMemoryAllocation) {
+        set_cuda_error(e);
+        return MOLE_ERR_NOMEM;
+    }
+    MOLE_CUDA_TRY(e);
+    return MOLE_OK;
+}
+
+int mole_host_free(void *ptr)
+{
+    if (!ptr) return MOLE_OK;
+    MOLE_CUDA_TRY(cudaFreeHost(ptr));
+    return MOLE_OK;
+}
+
+int mole_offload_destroy(mole_offload_ctx *c)
+{
+    if (!c) return MOLE_OK;
+    if (c->buf) {
+        for (int b = 0; b < c->n_buffers; ++b) {
+            mole_offload_ctx::Buffer &B = c->buf[b];
+            if (B.staging) cudaFree(B.staging);
+            if (B.uniq) cudaFree(B.uniq);
+            if (B.slot) cudaFree(B.slot);
+            if (B.count) cudaFree(B.count);
+            if (B.ready) cudaEventDestroy(B.ready);
+            if (B.consumed) cudaEventDestroy(B.consumed);
+        }
+        delete[] c->buf;
+    }
+    if (c->table) cudaFree(c->table);
+    delete c;
+    (void)cudaGetLastError();
+    return MOLE_OK;
+}
+
+int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, int V, int dtype, int n_buffers)
+{
+    if (!out) return MOLE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
+    if (max_tokens < 1 || n_buffers < 1 || n_buffers > 16) return MOLE_ERR_INVALID_ARG;
+    if (max_tokens > 65535) return MOLE_ERR_TOO_LARGE;
+    LayerPlan plan;
+    int rc = plan_layer(max_tokens, N, d, dtype, MOLE_VARIANT_AUTO, 0, &plan);
+    if (rc != MOLE_OK) return rc;
+    if (V < 1) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    mole_offload_ctx *c = new (std::nothrow) mole_offload_ctx;
+    if (!c) return MOLE_ERR_NOMEM;
+    memset(c, 0, sizeof *c);
+    c->max_tokens = max_tokens;
+    c->N = N;
+    c->d = d;
+    c->V = V;
+    c->dtype = dtype;
+    c->n_buffers = n_buffers;
+    c->row_bytes = static_cast<long long>(N) * d * elem_bytes(dtype);
+    c->buf = new (std::nothrow) mole_offload_ctx::Buffer[n_buffers];
+    if (!c->buf) {
+        delete c;
+        return MOLE_ERR_NOMEM;
+    }
+    memset(c->buf, 0, sizeof(mole_offload_ctx::Buffer) * n_buffers);
+    cudaError_t e = cudaMalloc(&c->table, sizeof(int32_t) * static_cast<size_t>(V));
+    if (e == cudaSuccess) e = cudaMemset(c->table, 0, sizeof(int32_t) * static_cast<size_t>(V));
+    for (int b = 0; b < n_buffers && e == cudaSuccess; ++b) {
+        mole_offload_ctx::Buffer &B = c->buf[b];
+        e = cudaMalloc(&B.staging, static_cast<size_t>(c->row_bytes) * max_tokens);
+        if (e == cudaSuccess) e = cudaMalloc(&B.uniq, sizeof(int32_t) * max_tokens);
+        if (e == cudaSuccess) e = cudaMalloc(&B.slot, sizeof(int32_t) * max_tokens);
+        if (e == cudaSuccess) e = cudaMalloc(&B.count, sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaMemset(B.count, 0, sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&B.ready, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&B.consumed, cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        set_cuda_error(e);
+        mole_offload_destroy(c);
+        return e == cudaErrorMemoryAllocation ? MOLE_ERR_NOMEM : MOLE_ERR_CUDA;
+    }
+    *out = c;
+    return MOLE_OK;
+}
+
+int mole_offload_prefetch(mole_offload_ctx *c, int b, const int32_t *ids, int M, const void *lut_host_layer,
+                          void *side_stream)
+{
+    if (!c || b < 0 || b >= c->n_buffers || M < 0) return MOLE_ERR_INVALID_ARG;
+    if (M > c->max_tokens) return MOLE_ERR_TOO_LARGE;
+    mole_offload_ctx::Buffer &B = c->buf[b];
+    B.M = M;
+    if (M == 0) return MOLE_OK;
+    if (!ids || !lut_host_layer || !aligned16(lut_host_layer)) return MOLE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(side_stream);
+    // the staging area may still be read by the layer that consumed this buffer last
+    MOLE_CUDA_TRY(cudaStreamWaitEvent(st, B.consumed, 0));
+    int rc = launch_dedup(ids, M, c->V, c->table, B.uniq, B.slot, B.count, nullptr, st);
+    if (rc != MOLE_OK) return rc;
+    rc = launch_fetch(lut_host_layer, B.uniq, B.count, M, c->row_bytes, B.staging, st);
+    if (rc != MOLE_OK) return rc;
+    MOLE_CUDA_TRY(cudaEventRecord(B.ready, st));
+    return MOLE_OK;
+}
+
+int mole_layer_forward_offload(mole_offload_ctx *c, int b, const void *hidden, const void *w_router, void *out,
+                               uint32_t *status, int B_, int T, void *stream)
+{
+    if (!c || b < 0 || b >= c->n_buffers || B_ < 0 || T < 0) return MOLE_ERR_INVALID_ARG;
+    mole_offload_ctx::Buffer &B = c->buf[b];
+    const long long M = static_cast<long long>(B_) * T;
+    if (M != B.M) return MOLE_ERR_INVALID_ARG;
+    if (M == 0) return MOLE_OK;
+    if (!hidden || !w_router || !out || !aligned16(hidden) || !aligned16(w_router) || !aligned16(out))
+        return MOLE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MOLE_CUDA_TRY(cudaStreamWaitEvent(st, B.ready, 0));
+    LayerLaunch a;
+    a.hidden = hidden;
+    a.residual = nullptr;
+    a.row_index = B.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
+    a.lut = B.staging;
+    a.w_router = w_router;
+    a.out = out;
+    a.gates_out = nullptr;
+    a.status = status;
+    a.M = M;
+    a.N = c->N;
+    a.d = c->d;
+    a.rows = c->max_tokens;
+    a.dtype = c->dtype;
+    a.flags = 0;
+    a.variant = MOLE_VARIANT_AUTO;
+    a.d_split = 0;
+    a.stream = st;
+    int rc = launch_layer(a);
+    if (rc != MOLE_OK) return rc;
+    MOLE_CUDA_TRY(cudaEventRecord(B.consumed, st));
+    return MOLE_OK;
+}
+
+int mole_offload_buffers(mole_offload_ctx *c, int b, const int32_t **uniq, const int32_t **slot, const int32_t **count,
+                         const void **staging)
+{
+    if (!c || b < 0 || b >= c->n_buffers) return MOLE_ERR_INVALID_ARG;
+    if (uniq) *uniq = c->buf[b].uniq;
+    if (slot) *slot = c->buf[b].slot;
+    if (count) *count = c->buf[b].count;
+    if (staging) *staging = c->buf[b].staging;
+    return MOLE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,152 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol
+the header declares, names its status codes, plans launches, and rejects bad arguments
+before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2503_15798_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "mole.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(HEADER).read()
+    return sorted(set(re.findall(r"MOLE_API\s+(?:const\s+char\s*\*|int)\s*(mole_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert len(names) >= 17
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_version_and_status_strings(lib):
+    assert lib.mole_version() == 100
+    seen = {lib.mole_status_string(c).decode() for c in range(6)}
+    assert len(seen) == 6 and "ok" in seen
+    assert lib.mole_status_string(99).decode() == "unknown status"
+
+
+def test_args_struct_layout_matches_header(lib):
+    # 2 x u32, 8 pointers, 8 x i32, 1 pointer
+    assert ctypes.sizeof(binding.MoleArgs) == 8 + 8 * 8 + 8 * 4 + 8
+
+
+def test_plan_shapes():
+    P = binding.plan
+    # large batches: one block per token while a token's rows fit beside other blocks
+    assert P(16384, 16, 1024)[0] == 1 and P(16384, 16, 768)[0] == 1
+    # the 1B-shaped rows (128 KB per token) are always split
+    s, threads, smem, variant = P(16384, 32, 2048)
+    assert s >= 4 and smem <= 48 * 1024 and variant == binding.VARIANT_CLUSTER
+    # few tokens: split to occupy the SMs
+    assert P(64, 16, 768)[0] >= 2 and P(1, 16, 768)[0] >= 2
+    # explicit split and variant are honoured
+    assert P(64, 16, 768, binding.DTYPE_BF16, binding.VARIANT_REPLICATE, 4)[0::3] == (4, binding.VARIANT_REPLICATE)
+    # a split of one needs no cluster
+    assert P(64, 16, 768, binding.DTYPE_BF16, binding.VARIANT_CLUSTER, 1)[3] == binding.VARIANT_REPLICATE
+    # fp32 tiny shape
+    s, threads, smem, variant = P(64, 4, 64, binding.DTYPE_F32)
+    assert s == 1 and threads == 32 and smem >= 4 * 64 * 4
+
+
+def test_plan_rejects_bad_shapes():
+    for args in ((64, 0, 768), (64, 65, 768), (64, 16, 772), (64, 16, 4)):
+        with pytest.raises(binding.MoleError) as e:
+            binding.plan(*args)
+        assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(binding.MoleError) as e:
+        binding.plan(64, 16, 768, 7)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.MoleError) as e:
+        binding.plan(64, 16, 768, binding.DTYPE_BF16, 0, 3)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.MoleError) as e:  # 768 / 16 columns is not a whole number of vectors
+        binding.plan(64, 16, 40, binding.DTYPE_BF16, 0, 8)
+    assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
+
+
+def test_forward_rejects_bad_arguments_without_launching(lib):
+    good = 0x10000  # an aligned, non-null address that is never dereferenced: every call below fails validation
+    f = lib.mole_layer_forward
+    assert f(None, good, good, good, good, 4, 1, 16, 768, 100, None) == binding.ERR_INVALID_ARG
+    assert f(good, None, good, good, good, 4, 1, 16, 768, 100, None) == binding.ERR_INVALID_ARG
+    assert f(good, good, good + 8, good, good, 4, 1, 16, 768, 100, None) == binding.ERR_INVALID_ARG  # misaligned table
+    assert f(good, good, good, good, good, -1, 1, 16, 768, 100, None) == binding.ERR_INVALID_ARG
+    assert f(good, good, good, good, good, 4, 1, 65, 768, 100, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert f(good, good, good, good, good, 4, 1, 16, 772, 100, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert f(good, good, good, good, good, 4, 1, 16, 768, 0, None) == binding.ERR_UNSUPPORTED_SHAPE
+    # zero tokens: success, nothing launched, pointers not even looked at
+    assert f(None, None, None, None, None, 0, 7, 16, 768, 100, None) == binding.OK
+    assert f(None, None, None, None, None, 3, 0, 16, 768, 100, None) == binding.OK
+
+
+def test_ex_rejects_bad_struct(lib):
+    a = binding.MoleArgs()
+    assert lib.mole_layer_forward_ex(None) == binding.ERR_INVALID_ARG
+    a.struct_size = 12
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.struct_size = ctypes.sizeof(binding.MoleArgs)
+    a.flags = 0x80
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.flags = 0
+    a.B, a.T, a.N, a.d, a.V, a.dtype = 2, 2, 16, 768, 10, 5
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.dtype = binding.DTYPE_BF16
+    good = 0x10000
+    a.hidden = a.lut = a.w_router = a.out = good
+    a.ids = good + 2  # misaligned ids
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.ids = good
+    a.residual = good  # residual aliasing out while not being hidden ... here it IS hidden: allowed, so poison out
+    a.out = good + 0x100
+    a.residual = good + 0x100
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.residual = None
+    a.variant = 9
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+
+
+def test_decode_step_and_offload_argument_checks(lib):
+    good = 0x10000
+    ds = lib.mole_decode_step
+    assert ds(good, good, good, 16, good, 16, good + 0x100, None, None, 0, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
+    assert ds(good, good, good, 8, good, 16, good + 0x100, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
+    assert ds(good, good, good, 16, good, 16, good + 0x100, None, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
+    assert ds(good, good, good, 16, good, 16, good, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
+    assert ds(None, None, None, 16, None, 16, None, None, None, 2, 0, 1, 16, 768, 100, 0, None) == binding.OK
+    dd = lib.mole_dedup_ids
+    assert dd(good, -1, 10, good, good, good, good, None, None) == binding.ERR_INVALID_ARG
+    assert dd(good, (1 << 20) + 1, 10, good, good, good, good, None, None) == binding.ERR_TOO_LARGE
+    assert dd(good, 4, 10, None, good, good, good, None, None) == binding.ERR_INVALID_ARG
+    fr = lib.mole_fetch_rows
+    assert fr(good, good, good, 4, 24, good, None) == binding.ERR_INVALID_ARG  # row not a multiple of 16 bytes
+    assert fr(good, good, good, 70000, 32, good, None) == binding.ERR_TOO_LARGE
+    assert fr(None, None, None, 0, 32, None, None) == binding.OK
+    h = ctypes.c_void_p()
+    assert lib.mole_offload_create(None, 4, 16, 768, 100, 0, 2) == binding.ERR_INVALID_ARG
+    assert lib.mole_offload_create(ctypes.byref(h), 0, 16, 768, 100, 0, 2) == binding.ERR_INVALID_ARG
+    assert lib.mole_offload_create(ctypes.byref(h), 4, 65, 768, 100, 0, 2) == binding.ERR_UNSUPPORTED_SHAPE
+    assert lib.mole_offload_create(ctypes.byref(h), 70000, 16, 768, 100, 0, 2) == binding.ERR_TOO_LARGE
+    assert lib.mole_offload_destroy(None) == binding.OK
+    assert lib.mole_host_alloc(None, 16) == binding.ERR_INVALID_ARG
+    assert lib.mole_host_free(None) == binding.OK
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        binding.lib()
