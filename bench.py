@@ -1,0 +1,423 @@
+#!/usr/bin/env python3
+"""Benchmark of the fused MoLE layer (arXiv 2503.15798, Eq. 4 + Eq. 8) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 160m|410m|1b] [--batch M]
+                    [--impl mole|reference] [--no-sweep] [--no-cpu]
+
+A "step" is one decode step of the whole hot path: all L layers of the configuration applied
+to one batch of M tokens (router, softmax over all experts, row gather, weighted sum,
+residual), chained with programmatic dependent launch and replayed from a CUDA graph.  The
+metric is tokens/s for the L-layer step; the roofline block reports the layer kernel's
+algorithmic GB/s (gathered rows + hidden in/out + router weights) against the measured HBM
+copy bandwidth.  Every step uses a different pre-generated Zipf(1.1) id batch, and the table
+(GBs) is far larger than L2.
+
+With N > 1 (torchrun) every rank holds its own replica of the tables and its own batches
+(tokens are independent, so there is no collective on the data path): weak scaling.
+
+--impl reference times the CPU oracle (oracle/, plain C, fp64) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MoLE layer tokens/s (L-layer decode step) and achieved HBM GB/s"
+UNIT = "tokens/s"
+N_BATCHES = 32          # distinct id batches the steps rotate through
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=100)
+    ap.add_argument("--impl", default="mole", choices=["mole", "reference"])
+    ap.add_argument("--config", default="160m", choices=["160m", "410m", "1b"])
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-batch sweep and the isolated-launch rows")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--layers", type=int, default=0, help="override L (debugging; the line then says so)")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.period, self._stop, self._thread, self.h = period_s, threading.Event(), None, None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None and self.h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------------
+# the CPU oracle leg (only bench.py's baseline leg and --impl reference execute oracle/)
+# ------------------------------------------------------------------------------------------------------
+
+def time_oracle(table_bits, wr_bits, hidden_bits, id_batches, L, budget_s, threads):
+    """Oracle lookup-form layer (fp64) on host copies; returns tokens/s for the L-layer step
+    (= one-layer tokens/s divided by L), the number of timed layer calls and the seconds used."""
+    import oracle
+
+    oracle.layer_lookup(hidden_bits, id_batches[0], table_bits, wr_bits, threads=threads)  # warm the pages
+    calls, t0 = 0, time.perf_counter()
+    while True:
+        oracle.layer_lookup(hidden_bits, id_batches[calls % len(id_batches)], table_bits, wr_bits, threads=threads)
+        calls += 1
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or calls >= 4096:
+            break
+    M = hidden_bits.shape[0]
+    return M * calls / dt / L, calls, dt
+
+
+def host_bits(t):
+    import numpy as np
+    import torch
+
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores (rank 0 only)."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2503_15798_b200 import inputs
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sh = inputs.SHAPES[args.config]
+    L = args.layers or sh.L
+    M = args.batch
+    cores = oracle.effective_threads(len(os.sched_getaffinity(0)))
+    table = host_bits(inputs.make_table(sh.V, sh.N, sh.d, seed=1000, device="cpu"))
+    wr = host_bits(inputs.make_router(sh.d, sh.N, seed=2000, device="cpu"))
+    hidden = host_bits(inputs.make_hidden(M, sh.d, seed=3000, device="cpu"))
+    batches = [inputs.zipf_ids(M, sh.V, seed=4000 + b).astype(np.int64) for b in range(N_BATCHES)]
+    for w in range(max(args.warmup, 1)):
+        oracle.layer_lookup(hidden, batches[w % N_BATCHES], table, wr, threads=cores)
+    t0 = time.perf_counter()
+    for k in range(args.steps):  # each step: ONE layer of the L-layer step (a 1/L sample), scaled below
+        oracle.layer_lookup(hidden, batches[k % N_BATCHES], table, wr, threads=cores)
+    dt = time.perf_counter() - t0
+    value = M * args.steps / dt / L
+    sample = (f"each step = the oracle's lookup-form layer on 1 of the {L} layers ({M} tokens, one {sh.name}-shaped "
+              f"bf16 table on the host); tokens/s divided by L for the L-layer step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps * L, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(sh, L, M, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(sh, L, M, args):
+    return {
+        "workload": f"{sh.name}-shaped decode: V={sh.V}, d={sh.d}, N={sh.N}, L={L}, bf16 table "
+                    f"{sh.layer_table_bytes * L / 1e9:.2f} GB, batch {M}x1, ids Zipf(1.1), hidden N(0,1)",
+        "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": M, "seq_len": 1,
+        "l2": f"inputs larger than L2: {N_BATCHES} rotating id batches over a {sh.layer_table_bytes * L / 1e9:.1f} GB "
+              "table; no flush between steps (hot Zipf rows may hit L2, as in the workload)",
+        "parallelism": f"replicas x{args.gpus} (tokens independent, no collective)",
+    }
+
+
+# ------------------------------------------------------------------------------------------------------
+# the GPU arm
+# ------------------------------------------------------------------------------------------------------
+
+class StepGraphs:
+    """One CUDA graph per id batch; a graph holds the L chained layer launches of one step."""
+
+    def __init__(self, mole, luts, wrs, hidden, id_batches):
+        import torch
+
+        self.torch, self.graphs = torch, []
+        self.out = torch.empty_like(hidden)
+        self.tmp = torch.empty_like(hidden)
+        self.status = torch.zeros(1, dtype=torch.int32, device=hidden.device)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for ids in id_batches:  # warm-up launches outside capture (sets kernel attributes)
+                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        for ids in id_batches:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status)
+            self.graphs.append(g)
+
+    def run(self, k0, k1):
+        n = len(self.graphs)
+        for k in range(k0, k1):
+            self.graphs[k % n].replay()
+
+
+def timed_ms(torch, fn):
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    fn()
+    b.record()
+    b.synchronize()
+    return a.elapsed_time(b)
+
+
+def run_mole(args):
+    import numpy as np
+    import torch
+
+    from paper_2503_15798_b200 import binding as mole
+    from paper_2503_15798_b200 import build as lib_build
+    from paper_2503_15798_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        lib_build.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    else:
+        torch.cuda.set_device(local_rank)
+    mole.lib()  # fails loudly if the library is missing
+    dev = torch.device("cuda", local_rank)
+    sh = inputs.SHAPES[args.config]
+    L = args.layers or sh.L
+    M = args.batch
+    peak, peak_src = measured_peak()
+
+    # ---- resident inputs: L tables, routers, hidden, rotating id batches (per-rank seeds) ----------
+    luts = torch.empty((L, sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        inputs.make_table(sh.V, sh.N, sh.d, seed=1000 + l + 100 * rank, device=dev, out=luts[l])
+    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
+    max_m = max([M] + ([b for b in sh.batches] if not args.no_sweep else []))
+    hidden_all = inputs.make_hidden(max_m, sh.d, seed=3000 + rank, device=dev)
+
+    def batches_for(m):
+        return [inputs.make_ids(m, sh.V, seed=4000 + 1000 * rank + b + 7 * m, device=dev) for b in range(N_BATCHES)]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- headline: K steps of the L-layer chained step ---------------------------------------------------
+    hidden = hidden_all[:M].contiguous()
+    graphs = StepGraphs(mole, luts, wrs, hidden, batches_for(M))
+    graphs.run(0, max(args.warmup, 3))
+    barrier()
+    with ClockSampler(physical_gpu_index(local_rank)) as clocks:
+        ms = timed_ms(torch, lambda: graphs.run(0, args.steps))
+    barrier()
+    assert int(graphs.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * M * args.steps / (ms * 1e-3)
+    launches = args.steps * L
+    layer_bytes = sh.layer_bytes(M)
+    achieved = layer_bytes / (ms * 1e-3 / launches) / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": workload_config(sh, L, M, args),
+        "tokens_per_s_per_layer": value * L,
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "kernel": "mole_layer_kernel", "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": layer_bytes, "us_per_launch": ms * 1e3 / launches},
+        "clocks": clocks.summary(),
+    }
+
+    # ---- end to end: host buffers in, host buffer out, through the C ABI, every step ---------------------
+    h_host = hidden.cpu().pin_memory()
+    out_host = torch.empty_like(h_host).pin_memory()
+    ids_host = [b.cpu().pin_memory() for b in batches_for(M)]
+    dev_bufs = [torch.empty_like(hidden) for _ in range(3)]
+    dev_ids = torch.empty(M, dtype=torch.int32, device=dev)
+    e2e_steps = min(args.steps, 2000)
+
+    def e2e_run(n):
+        for k in range(n):
+            mole.decode_step_host(h_host, ids_host[k % N_BATCHES], out_host, dev_bufs[0], dev_ids, dev_bufs[1],
+                                  dev_bufs[2], luts, wrs)
+            torch.cuda.current_stream().synchronize()  # the caller reads out_host after every step
+
+    e2e_run(max(3, min(args.warmup, 50)))
+    barrier()
+    t0 = time.perf_counter()
+    ms_e2e = timed_ms(torch, lambda: e2e_run(e2e_steps))
+    wall_e2e = time.perf_counter() - t0
+    barrier()
+    if dist is not None:
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    line["e2e"] = {"value": world * M * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": M * sh.d * 2 + M * 4, "d2h_bytes_per_step": M * sh.d * 2,
+                   "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
+                   "how": "mole_decode_step_host: pinned host hidden+ids -> device, L chained layers, result -> "
+                          "pinned host, stream synchronised after every step"}
+
+    # ---- sweep over the configuration's batch sizes: chained step + isolated launches -----------------------
+    if not args.no_sweep and rank == 0:
+        sweep = []
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+        for m in sh.batches:
+            if m * sh.d * 2 > 2**31:
+                continue
+            hid = hidden_all[:m].contiguous()
+            bl = batches_for(m)
+            steps_m = max(50, min(args.steps, int(2e6 // max(m, 64))))
+            g = StepGraphs(mole, luts, wrs, hid, bl)
+            g.run(0, 20)
+            torch.cuda.synchronize()
+            ms_m = timed_ms(torch, lambda: g.run(0, steps_m))
+            us_layer = ms_m * 1e3 / (steps_m * L)
+            # isolated single launches of layer 0: steady (rotating ids) and cold (L2 flushed before each)
+            out = torch.empty_like(hid)
+            reps = 200 if m <= 1024 else 20
+            iso = []
+            for cold in (False, True):
+                ts = []
+                for r in range(reps):
+                    if cold:
+                        flush.fill_(r & 0xFF)
+                    ts.append(timed_ms(torch, lambda: mole.layer_forward(hid, bl[r % N_BATCHES], luts[0], wrs[0], out)))
+                iso.append(statistics.median(ts) * 1e3)
+            nbytes = sh.layer_bytes(m)
+            sweep.append({
+                "batch": m, "chained_us_per_layer": us_layer, "tokens_per_s_all_layers": m / (us_layer * L * 1e-6),
+                "tokens_per_s_per_layer": m / (us_layer * 1e-6), "chained_GBps": nbytes / us_layer / 1e3,
+                "chained_frac_of_peak": nbytes / us_layer / 1e3 / peak,
+                "isolated_steady_us": iso[0], "isolated_cold_us": iso[1],
+                "isolated_cold_GBps": nbytes / iso[1] / 1e3, "plan": mole.plan(m, sh.N, sh.d),
+            })
+            del g
+        line["sweep"] = sweep
+        del flush
+
+    # ---- the CPU oracle beside it (rank 0, N = 1 only) ------------------------------------------------------
+    if not args.no_cpu and rank == 0 and world == 1:
+        import oracle
+
+        cores = oracle.effective_threads(len(os.sched_getaffinity(0)))
+        table0 = host_bits(luts[0])
+        ids_np = [b.cpu().numpy().astype(np.int64) for b in batches_for(M)]
+        v_all, calls, dt = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 8.0, cores)
+        v_one, calls1, dt1 = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 4.0, 1)
+        line["cpu_baseline"] = {
+            "value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{calls} calls of the oracle's lookup-form layer (fp64) on a host copy of layer 0's table, "
+                      f"{M} tokens each, {dt:.1f} s; tokens/s divided by L={L} for the L-layer step",
+            "single_thread_value": v_one,
+        }
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_mole(args)
+
+
+if __name__ == "__main__":
+    main()
