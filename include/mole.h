@@ -176,6 +176,32 @@ MOLE_API int mole_dedup_ids(const int32_t *ids, int M, int V, int32_t *scratch, 
                    int32_t *count, uint32_t *status, void *stream);
 
 /*
+ * mole_dedup_ids_static -- mole_dedup_ids for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option -- a plug-in inside a server
+ * whose own allocator already holds all of the GPU's memory, or a decode loop that must never
+ * hit the device-wide synchronisation an allocation implies.  Such a caller still passes its
+ * inputs and outputs, but the V-entry scratch table is a fixed array inside the library's
+ * device image instead of a caller buffer: MOLE_STATIC_DEDUP_MAX_V int32 entries (256 KB) that
+ * every GPU which loads the library holds until the process exits.
+ *
+ *   ids, uniq, slot, count, status, stream: exactly as in mole_dedup_ids; results are identical.
+ *   V > MOLE_STATIC_DEDUP_MAX_V returns MOLE_ERR_TOO_LARGE and launches nothing.
+ *
+ * The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.  The
+ * first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and caches it; make that first call outside any stream capture.
+ * All calls on a device share the one array.  The kernel expects it all zero and leaves it all
+ * zero (it clears exactly the entries it set), so consecutive calls on one stream need no
+ * clearing in between -- but two calls that overlap on the GPU (different streams without an
+ * ordering between them) race on the array and give wrong results.
+ */
+#define MOLE_STATIC_DEDUP_MAX_V 65536
+MOLE_API int mole_dedup_ids_static(const int32_t *ids, int M, int V, int32_t *uniq, int32_t *slot, int32_t *count,
+                          uint32_t *status, void *stream);
+
+/*
  * mole_fetch_rows -- copy rows uniq[0..count) of a table in pinned, device-mapped host
  * memory into a dense device staging buffer: staging[u] = lut_host[uniq[u]] (row_bytes each,
  * a multiple of 16).  The reads are issued by the GPU across the host link; `count` is read on

@@ -25,7 +25,7 @@ VARIANT_AUTO, VARIANT_REPLICATE, VARIANT_CLUSTER = 0, 1, 2
 # every symbol include/mole.h declares
 EXPORTS = (
     "mole_layer_forward", "mole_layer_forward_ex", "mole_decode_step", "mole_decode_step_host",
-    "mole_dedup_ids", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
+    "mole_dedup_ids", "mole_dedup_ids_static", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
     "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_buffers",
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan",
 )
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.mole_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, c_int64, vp, c_int64, vp, c_int, c_int,
                                             c_int, c_int, c_int, c_int, c_int, vp]
         L.mole_dedup_ids.argtypes = [ip, c_int, c_int, ip, ip, ip, ip, vp, vp]
+        L.mole_dedup_ids_static.argtypes = [ip, c_int, c_int, ip, ip, ip, vp, vp]
         L.mole_fetch_rows.argtypes = [vp, ip, ip, c_int, c_int64, vp, vp]
         L.mole_host_alloc.argtypes = [POINTER(c_void_p), c_size_t]
         L.mole_host_free.argtypes = [vp]
@@ -201,6 +202,17 @@ def dedup_ids(ids, V: int, scratch, uniq, slot, count, status=None, stream=None)
     """mole_dedup_ids: all tensors int32 on the device; scratch [V] must be zero on entry."""
     _check(lib().mole_dedup_ids(_ptr(ids), ids.numel(), V, _ptr(scratch), _ptr(uniq), _ptr(slot), _ptr(count),
                                 _ptr(status), _stream(stream)), "mole_dedup_ids")
+
+
+STATIC_DEDUP_MAX_V = 65536
+
+
+def dedup_ids_static(ids, V: int, uniq, slot, count, status=None, stream=None):
+    """mole_dedup_ids_static: dedup_ids without a caller-supplied scratch table, for callers that
+    cannot allocate device memory; the table is a fixed 256 KB array inside the library, shared by
+    all calls on a device (so calls must not overlap on the GPU).  V <= STATIC_DEDUP_MAX_V."""
+    _check(lib().mole_dedup_ids_static(_ptr(ids), ids.numel(), V, _ptr(uniq), _ptr(slot), _ptr(count),
+                                       _ptr(status), _stream(stream)), "mole_dedup_ids_static")
 
 
 def fetch_rows(lut_host, uniq, count, max_rows: int, staging, stream=None):

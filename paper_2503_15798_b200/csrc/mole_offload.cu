@@ -2,6 +2,7 @@
 // re-parameterised table on a storage device and moves only the looked-up rows, Sec. 3.3);
 // per step the distinct ids are found on the device, their rows are read across the host
 // link by the GPU itself into a dense staging buffer, and the fused layer gathers from there.
+#include <mutex>
 #include <new>
 #include <string.h>
 
@@ -334,3 +335,59 @@ int mole_offload_buffers(mole_offload_ctx *c, int b, const int32_t **uniq, const
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Dedup for callers that cannot allocate device memory.
+//
+// Some hosts of this library have no way to get a V-entry scratch table for mole_dedup_ids:
+// a plug-in inside an inference server whose allocator already owns all of HBM (a raw
+// cudaMalloc there fails or fragments the pool), or a decode loop that must never run into
+// cudaMalloc's device-wide synchronisation.  For them the scratch table lives in the library
+// image itself: a fixed array in device global memory that every GPU loading the library
+// carries (MOLE_STATIC_DEDUP_MAX_V * 4 bytes = 256 KB) until the process exits.
+//
+// In host code the array's name is only a stand-in symbol, not an address a kernel can use, so
+// its device address is looked up with cudaGetSymbolAddress once per device (with that device
+// current) and cached; the kernel gets that address.
+// ---------------------------------------------------------------------------------------------
+namespace mole {
+
+static __device__ __align__(256) int32_t g_static_dedup_table[MOLE_STATIC_DEDUP_MAX_V];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static int32_t *g_static_table_addr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_dedup_table on the current device (looked up on first use).
+static int static_table_for_current_device(int32_t **out)
+{
+    int dev = -1;
+    MOLE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return MOLE_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_table_addr[dev]) {
+        void *p = nullptr;
+        MOLE_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_dedup_table));
+        if (!p) return MOLE_ERR_CUDA;
+        g_static_table_addr[dev] = static_cast<int32_t *>(p);
+    }
+    *out = g_static_table_addr[dev];
+    return MOLE_OK;
+}
+
+}  // namespace mole
+
+extern "C" int mole_dedup_ids_static(const int32_t *ids, int M, int V, int32_t *uniq, int32_t *slot, int32_t *count,
+                                     uint32_t *status, void *stream)
+{
+    if (M < 0 || V < 1) return MOLE_ERR_INVALID_ARG;
+    if (V > MOLE_STATIC_DEDUP_MAX_V) return MOLE_ERR_TOO_LARGE;  // the built-in table has no room for this vocabulary
+    if (M > MOLE_DEDUP_MAX_TOKENS) return MOLE_ERR_TOO_LARGE;
+    if (!count || (M > 0 && (!ids || !uniq || !slot))) return MOLE_ERR_INVALID_ARG;
+    int32_t *table = nullptr;
+    int rc = static_table_for_current_device(&table);
+    if (rc != MOLE_OK) return rc;
+    // The table is zero when the library is loaded and every run of the kernel zeroes the
+    // entries it touched before it ends, so nothing has to be cleared here.
+    return launch_dedup(ids, M, V, table, uniq, slot, count, status, static_cast<cudaStream_t>(stream));
+}
