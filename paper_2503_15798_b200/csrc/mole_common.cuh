@@ -24,33 +24,42 @@ void set_cuda_error(cudaError_t e);  // remembers the text for mole_last_cuda_er
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int elem_bytes(int dtype) { return dtype == MOLE_DTYPE_BF16 ? 2 : 4; }
 
-// Launch description of the fused layer kernel (filled by plan_layer, pure host arithmetic).
-struct LayerPlan {
-    int d_split;   // blocks per token
-    int dc;        // columns per block
-    int threads;   // threads per block
-    int smem;      // dynamic shared memory, bytes
-    int variant;   // MOLE_VARIANT_REPLICATE or MOLE_VARIANT_CLUSTER (d_split == 1 => REPLICATE)
-    int n_fast;    // N if the unrolled router path exists for it, else 0
+// Launch description of the fused kernel (filled by plan_step, pure host arithmetic).
+// A block owns one slice of dc = d / d_split columns of a token; it walks over its tokens and,
+// for every token, over the L layers, pulling the table rows of each (token, layer) item
+// through a ring of `stages` shared-memory slots.
+struct StepPlan {
+    int d_split;        // blocks per token (a cluster when > 1)
+    int dc;             // columns per block
+    int consumers;      // threads that compute (a multiple of 32); one more warp issues the copies
+    int threads;        // consumers + 32
+    int stages;         // ring depth
+    int slot_bytes;     // one ring slot: rows [+ router slice] + hidden slice, padded to 128
+    int wr_in_ring;     // 1: the router slice travels with every item (L > 1); 0: loaded once per block
+    int smem;           // dynamic shared memory, bytes
+    int blocks_per_sm;  // resident blocks per SM the shared memory allows
+    int n_fast;         // N if the unrolled router path exists for it, else 0
 };
-int plan_layer(long long M, int N, int d, int dtype, int variant, int d_split, LayerPlan *plan);
+int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan);
 
-// One fused-layer launch; `row_index` is ids (resident mode) or slot (offload mode) and
-// `rows` the number of rows of `lut` that may be addressed.
-struct LayerLaunch {
+// One launch of the fused kernel over L chained layers (L == 1: a single layer).
+// `row_index` is ids (resident mode) or slot (offload mode); `rows` the number of table rows
+// that may be addressed.
+struct StepLaunch {
     const void *hidden, *residual, *row_index, *lut, *w_router;
     void *out;
     float *gates_out;
     uint32_t *status;
+    long long lut_stride, wr_stride;  // bytes between consecutive layers
     long long M;
-    int N, d;
+    int L, N, d;
     long long rows;
     int dtype;
     uint32_t flags;
-    int variant, d_split;
+    int d_split;
     cudaStream_t stream;
 };
-int launch_layer(const LayerLaunch &L);
+int launch_step(const StepLaunch &a);
 
 #ifdef __CUDACC__
 // ---- device side ---------------------------------------------------------------------------
@@ -106,6 +115,44 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     return false;
 }
 
+// Phase completion of an mbarrier that remote blocks of the cluster signal (st.async below).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Address of the same shared-memory location in block `cta` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t cta)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(cta));
+    return remote;
+}
+// Store one float into another block's shared memory and credit 4 bytes to that block's mbarrier.
+__device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint32_t remote_bar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote_addr),
+                 "r"(__float_as_uint(v)), "r"(remote_bar)
+                 : "memory");
+}
+// Barrier over a subset of the block's warps (id 1..15, count a multiple of 32).
+__device__ __forceinline__ void named_bar_sync(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
 // programmatic dependent launch
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -119,12 +166,6 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
 }
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-__device__ __forceinline__ void st_cluster_f32(uint32_t local_smem_addr, uint32_t cta, float v)
-{
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(cta));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
 
 // 16-byte vectors of the two storage types
 template <typename T>
