@@ -1,0 +1,190 @@
+// The fused MoLE kernel for sm_100a (Eq. 4 and Eq. 8 of arXiv 2503.15798): router dot products,
+// softmax over all N experts, gather of the token's N table rows, fp32 weighted sum, residual
+// add -- for one layer or for L chained layers in one launch.
+//
+// Work decomposition.  A block owns one slice of dc = d / S columns (S blocks of a token form
+// a thread-block cluster when S > 1).  It walks over its tokens t = c, c + C, c + 2C, ... and,
+// per token, over the layers l = 0 .. L-1; one (token, layer) pair is an "item".  The chain
+// h_{l+1} = h_l + sum_j g_j(h_l) LUT_l[id][j] of a token never leaves the block: the running
+// hidden slice stays in shared memory, rounded to the storage type after every layer exactly as
+// a layer-by-layer execution would round it.
+//
+// Data movement.  Everything an item needs is pulled into a ring of shared-memory slots by bulk
+// asynchronous copies (TMA engine, untiled, no multicast) that one extra "producer" warp issues
+// `stages` items ahead: the N row pieces (they depend only on the id, so they run ahead of the
+// arithmetic and, in a chained launch, ahead of the previous kernel), the router slice of the
+// layer when L > 1, and the token's hidden slice for its first layer.  Completion is counted on
+// one mbarrier per slot ("full"); the consumer warps hand a slot back through a second one
+// ("empty").
+//
+// Arithmetic per item (consumer warps): a conflict-free linear sweep over the router slice in
+// shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp,
+// shared memory over the warps and -- when S > 1 -- st.async into every peer's shared memory
+// over the cluster; every warp then evaluates the softmax redundantly (fp32, expf, true
+// division) and combines the rows it owns in expert order.
+#pragma once
+
+#include <math.h>
+
+#include "mole_common.cuh"
+
+namespace mole {
+
+constexpr int kMaxN = 64;            // experts
+constexpr int kMaxSplit = 8;         // blocks per token
+constexpr int kMaxConsumers = 256;   // compute threads per block
+constexpr int kMaxStages = 8;        // ring depth
+constexpr int kConsumerBarrier = 1;  // named barrier of the consumer warps
+constexpr uint32_t kWaitPolls = 1u << 24;   // >= 1 s of polling before a wait gives up
+constexpr uint32_t kDrainPolls = 1u << 14;  // after a failure: short waits for copies still in flight
+
+struct StepParams {
+    const void *hidden, *residual, *row_index, *lut, *w_router;
+    void *out;
+    float *gates_out;
+    uint32_t *status;
+    long long lut_stride, wr_stride;  // bytes between layers
+    long long M, rows;
+    int N, d, S, dc, L;
+    int stages, slot_bytes, wr_in_ring, consumers;
+    uint32_t flags;
+};
+
+// Shared-memory map, computed the same way on the host (for the size) and in the kernel.
+struct SmemMap {
+    uint32_t rows_bytes, wr_bytes, hid_bytes;  // per item: row pieces, router slice, hidden slice
+    uint32_t slot_wr, slot_hid;                // offsets inside a slot
+    uint32_t slot_bytes;
+    uint32_t off_wr, off_hid, off_partial, off_xchg, off_gates, off_meta, off_bars, total;
+};
+__host__ __device__ inline uint32_t up128(uint32_t x) { return (x + 127u) & ~127u; }
+__host__ __device__ inline SmemMap smem_map(int N, int dc, int eb, int S, int stages, int wr_in_ring, int consumers)
+{
+    SmemMap m;
+    m.rows_bytes = static_cast<uint32_t>(N) * dc * eb;
+    m.wr_bytes = static_cast<uint32_t>(dc) * N * eb;
+    m.hid_bytes = static_cast<uint32_t>(dc) * eb;
+    m.slot_wr = m.rows_bytes;
+    m.slot_hid = m.rows_bytes + (wr_in_ring ? m.wr_bytes : 0u);
+    m.slot_bytes = up128(m.slot_hid + m.hid_bytes);
+    const uint32_t warps = consumers / 32;
+    m.off_wr = stages * m.slot_bytes;
+    m.off_hid = m.off_wr + (wr_in_ring ? 0u : up128(m.wr_bytes));
+    m.off_partial = m.off_hid + up128(m.hid_bytes);
+    m.off_xchg = m.off_partial + up128(2u * warps * N * 4);
+    m.off_gates = m.off_xchg + up128(2u * S * N * 4);
+    m.off_meta = m.off_gates + up128(warps * N * 4);
+    m.off_bars = m.off_meta + up128((kMaxStages + 3) * 4);
+    m.total = m.off_bars + (2 * kMaxStages + 3) * 8;
+    return m;
+}
+
+#ifdef __CUDACC__
+
+// Sum n per-lane values over the lanes that differ in bits o, o/2, .., omin: every step halves
+// the number of values a lane still carries (n - 1 + a few shuffles instead of log2 * n).  On
+// return a[0 .. left) hold the totals of values base .. base + left - 1; lanes that end up with
+// the same values hold identical copies.
+template <int NTOT, int n, int o, int omin>
+__device__ __forceinline__ void lane_reduce_scatter(float (&a)[NTOT], int lane, int &base)
+{
+    if constexpr (o >= omin) {
+        if constexpr (n > 1) {
+            constexpr int half = n / 2;
+            const bool up = (lane & o) != 0;
+#pragma unroll
+            for (int i = 0; i < half; ++i) {
+                const float send = up ? a[i] : a[i + half];
+                const float keep = up ? a[i + half] : a[i];
+                a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
+            if (up) base += half;
+            lane_reduce_scatter<NTOT, half, o / 2, omin>(a, lane, base);
+        } else {
+            a[0] += __shfl_xor_sync(0xffffffffu, a[0], o);
+            lane_reduce_scatter<NTOT, 1, o / 2, omin>(a, lane, base);
+        }
+    }
+}
+// number of values a lane is left with after lane_reduce_scatter<.., n, o, omin>
+template <int n, int o, int omin>
+struct ReduceScatterLeft {
+    static constexpr int value = (o >= omin && n > 1) ? ReduceScatterLeft<n / 2, o / 2, omin>::value : n;
+};
+template <int n, int omin>
+struct ReduceScatterLeft<n, 0, omin> {
+    static constexpr int value = n;
+};
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Bounded wait shared by producer and consumers.  `dead` (shared memory) is raised by whoever
+// gives up first; everyone else then stops waiting at once.
+__device__ __forceinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
+                                                bool cluster_scope)
+{
+    for (uint32_t i = 0; i < polls; ++i) {
+        if (cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if (i > 64) {
+            __nanosleep(64);
+            if ((i & 127u) == 0 && *dead) return false;
+        }
+    }
+    return false;
+}
+
+// Partial router logits of one item over this block's dc columns, fast path (N a power of two
+// the kernel is compiled for).  The router slice [dc][N] is swept linearly, 16 bytes per lane,
+// so a warp reads 512 consecutive bytes per step (no bank conflicts for any N).  A 16-byte
+// vector holds either VEC consecutive experts of one column (N >= VEC) or VEC / N whole columns
+// (N < VEC); since the sweep stride is a multiple of 32 vectors, a lane always meets the same
+// experts and keeps only min(VEC, N) accumulators.
+template <typename T, int NFAST>
+__device__ __forceinline__ void router_partial_fast(const unsigned char *wptr, const unsigned char *hptr, int dc,
+                                                    int tid, int lane, int nc, float *partial_warp)
+{
+    using E = Elem<T>;
+    constexpr int VEC = E::VEC;
+    constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
+    constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
+    constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
+    float acc[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+    const int nvec = dc * NFAST / VEC;
+    const uint4 *wv = reinterpret_cast<const uint4 *>(wptr);
+    for (int u = tid; u < nvec; u += nc) {
+        float wf[VEC];
+        E::unpack(wv[u], wf);
+        if constexpr (NFAST >= VEC) {
+            const float h = E::scalar(hptr, u / QL);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) acc[i] = fmaf(h, wf[i], acc[i]);
+        } else {
+#pragma unroll
+            for (int cc = 0; cc < CPV; ++cc) {
+                const float h = E::scalar(hptr, u * CPV + cc);
+#pragma unroll
+                for (int i = 0; i < NFAST; ++i) acc[i] = fmaf(h, wf[cc * NFAST + i], acc[i]);
+            }
+        }
+    }
+    int base = 0;
+    lane_reduce_scatter<NV, NV, 16, QL>(acc, lane, base);
+    constexpr int left = ReduceScatterLeft<NV, 16, QL>::value;
+    const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
+#pragma unroll
+    for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
+}
+
