@@ -188,3 +188,142 @@ __device__ __forceinline__ void router_partial_fast(const unsigned char *wptr, c
     for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
 }
 
+// T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
+template <typename T, int NFAST>
+__global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const StepParams p)
+{
+    using E = Elem<T>;
+    constexpr int VEC = E::VEC;
+    constexpr int EB = static_cast<int>(sizeof(T));
+    extern __shared__ __align__(128) unsigned char smem[];
+
+    pdl_launch_dependents();
+
+    const int N = NFAST > 0 ? NFAST : p.N;
+    const int S = p.S, dc = p.dc, d = p.d, L = p.L, stages = p.stages, nc = p.consumers;
+    const SmemMap m = smem_map(N, dc, EB, S, stages, p.wr_in_ring, nc);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long C = gridDim.x / S, c = blockIdx.x / S;  // clusters in the grid, this block's cluster
+    const int s = static_cast<int>(blockIdx.x % S);         // column slice == rank in the cluster
+    const long long ntok = c < p.M ? (p.M - c + C - 1) / C : 0;
+    const long long nitems = ntok * L;
+
+    volatile int *meta = reinterpret_cast<volatile int *>(smem + m.off_meta);  // [stages] row valid
+    volatile int *dead = meta + kMaxStages;        // somebody gave up waiting
+    volatile int *issued = meta + kMaxStages + 1;  // items whose copies have been issued
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + m.off_bars);
+    uint64_t *full = bars, *empty = bars + kMaxStages, *xbar = bars + 2 * kMaxStages, *wrbar = xbar + 2;
+
+    if (tid == 0) {
+        for (int st = 0; st < stages; ++st) {
+            mbar_init(full + st, 1);
+            mbar_init(empty + st, nc / 32);
+        }
+        mbar_init(xbar, 1);
+        mbar_init(xbar + 1, 1);
+        mbar_init(wrbar, 1);
+        *dead = 0;
+        *issued = 0;
+        meta[kMaxStages + 2] = 0;  // a flag nobody raises: lets the drain waits run their full (short) course
+        mbar_init_fence();
+    }
+    if (S > 1) {  // peers may write into this block's shared memory only once its barriers exist
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    } else {
+        __syncthreads();
+    }
+
+    if (tid >= nc) {
+        // ================= producer warp: issues every copy, `stages` items ahead =================
+        const bool ids64 = (p.flags & MOLE_FLAG_IDS_INT64) != 0;
+        long long k = 0, batch = -1, row = -1;
+        int l = 0;
+        if (!p.wr_in_ring && nitems > 0 && lane == 0) {
+            mbar_expect_tx(wrbar, m.wr_bytes);
+            bulk_g2s(smem + m.off_wr, static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(s) * m.wr_bytes,
+                     m.wr_bytes, wrbar);
+        }
+        // Everything of item `it` except (optionally) the hidden slice.
+        auto issue = [&](long long it, bool with_hidden) {
+            if (l == 0) {
+                if ((k & 31) == 0) {  // ids of the next 32 tokens of this block, one per lane
+                    const long long kk = k + lane;
+                    batch = -1;
+                    if (kk < ntok) {
+                        const long long t = c + kk * C;
+                        batch = ids64 ? __ldg(static_cast<const long long *>(p.row_index) + t)
+                                      : static_cast<long long>(__ldg(static_cast<const int *>(p.row_index) + t));
+                    }
+                }
+                row = __shfl_sync(0xffffffffu, batch, static_cast<int>(k & 31));
+            }
+            const bool valid = row >= 0 && row < p.rows;
+            const int st = static_cast<int>(it % stages);
+            unsigned char *slot = smem + static_cast<size_t>(st) * m.slot_bytes;
+            if (lane == 0) {
+                meta[st] = valid ? 1 : 0;
+                if (!valid && l == 0 && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
+                mbar_expect_tx(full + st, m.slot_hid + (l == 0 ? m.hid_bytes : 0u));
+                *issued = static_cast<int>(it + 1 < 0x7fffffff ? it + 1 : 0x7fffffff);
+            }
+            __syncwarp();
+            // an id outside the table gathers row 0 (always present); its routed term is dropped later
+            const unsigned char *src = static_cast<const unsigned char *>(p.lut) + static_cast<size_t>(l) * p.lut_stride +
+                                       (static_cast<size_t>(valid ? row : 0) * N * d + static_cast<size_t>(s) * dc) * EB;
+            if (S == 1) {
+                if (lane == 0) bulk_g2s(slot, src, m.rows_bytes, full + st);  // the N rows of an id are contiguous
+            } else {
+                const uint32_t piece = static_cast<uint32_t>(dc) * EB;
+                for (int j = lane; j < N; j += 32)
+                    bulk_g2s(slot + static_cast<size_t>(j) * piece, src + static_cast<size_t>(j) * d * EB, piece, full + st);
+            }
+            if (p.wr_in_ring && lane == 31)
+                bulk_g2s(slot + m.slot_wr,
+                         static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(l) * p.wr_stride +
+                             static_cast<size_t>(s) * m.wr_bytes,
+                         m.wr_bytes, full + st);
+            if (with_hidden && l == 0 && lane == 30) {
+                const long long t = c + k * C;
+                bulk_g2s(slot + m.slot_hid,
+                         static_cast<const unsigned char *>(p.hidden) +
+                             (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB,
+                         m.hid_bytes, full + st);
+            }
+            if (++l == L) {
+                l = 0;
+                ++k;
+            }
+        };
+        // The first `stages` items need no free slot and -- except for hidden, which the previous
+        // kernel of a chained launch writes -- nothing upstream: issue them before the grid
+        // dependency is waited for.
+        const long long pre = nitems < stages ? nitems : stages;
+        for (long long it = 0; it < pre; ++it) issue(it, false);
+        pdl_wait();
+        fence_proxy_async_global();
+        if (lane == 30) {
+            for (long long it = 0; it < pre; it += L) {  // the items with l == 0
+                const long long t = c + (it / L) * C;
+                const int st = static_cast<int>(it % stages);
+                bulk_g2s(smem + static_cast<size_t>(st) * m.slot_bytes + m.slot_hid,
+                         static_cast<const unsigned char *>(p.hidden) +
+                             (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB,
+                         m.hid_bytes, full + st);
+            }
+        }
+        for (long long it = pre; it < nitems; ++it) {
+            int ok = 1;
+            if (lane == 0) {
+                const int st = static_cast<int>(it % stages);
+                ok = wait_or_give_up(empty + st, static_cast<uint32_t>((it / stages - 1) & 1), dead, kWaitPolls, false);
+                if (!ok) {
+                    if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                    *dead = 1;
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            issue(it, true);
+        }
+    } else {
