@@ -327,3 +327,163 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             issue(it, true);
         }
     } else {
+        // ================= consumer warps: router, softmax, combine ================================
+        pdl_wait();  // out may still be read, and hidden / residual written, by the previous kernel
+        const int nwarps = nc / 32;
+        const int ngrp = dc / VEC;  // 16-byte column groups of this block's slice
+        float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [2][nwarps][N]
+        float *xchg = reinterpret_cast<float *>(smem + m.off_xchg);        // [2][S][N]
+        float *my_gates = reinterpret_cast<float *>(smem + m.off_gates) + warp * N;
+        unsigned char *hid = smem + m.off_hid;  // running hidden slice between layers
+        bool alive = true;
+
+        auto give_up = [&]() {
+            if (lane == 0) {
+                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                *dead = 1;
+            }
+            alive = false;
+        };
+        if (!p.wr_in_ring && nitems > 0) {
+            const bool got = wait_or_give_up(wrbar, 0, dead, kWaitPolls, false);
+            if (!__all_sync(0xffffffffu, got)) give_up();
+        }
+
+        long long k = 0;
+        int l = 0;
+        for (long long it = 0; it < nitems; ++it) {
+            const int st = static_cast<int>(it % stages);
+            const uint32_t ph = static_cast<uint32_t>((it / stages) & 1);
+            const int par = static_cast<int>(it & 1);
+            const long long t = c + k * C;
+            unsigned char *slot = smem + static_cast<size_t>(st) * m.slot_bytes;
+            float *part = partial + par * nwarps * N;
+            float *xch = xchg + par * S * N;
+
+            if (alive) {
+                if (S > 1 && tid == 0) mbar_expect_tx(xbar + par, static_cast<uint32_t>(S) * N * 4u);
+                const bool got = wait_or_give_up(full + st, ph, dead, kWaitPolls, false);
+                if (!__all_sync(0xffffffffu, got)) give_up();
+            } else if (it < *issued) {
+                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls, false);  // let copies in flight land
+            }
+
+            const unsigned char *hptr = (l == 0) ? slot + m.slot_hid : hid;
+            int nparts = nwarps;
+            if (alive) {
+                const unsigned char *wptr = p.wr_in_ring ? slot + m.slot_wr : smem + m.off_wr;
+                if constexpr (NFAST > 0) {
+                    router_partial_fast<T, NFAST>(wptr, hptr, dc, tid, lane, nc, part + warp * N);
+                } else {
+                    // any N: one warp per expert, lanes stride over the columns
+                    for (int j = warp; j < N; j += nwarps) {
+                        float z = 0.f;
+                        for (int cc = lane; cc < dc; cc += 32)
+                            z = fmaf(E::scalar(hptr, cc), E::scalar(wptr, static_cast<long long>(cc) * N + j), z);
+                        z = warp_sum(z);
+                        if (lane == 0) part[j] = z;
+                    }
+                    nparts = 1;
+                }
+            }
+            named_bar_sync(kConsumerBarrier, nc);
+
+            if (alive) {
+                const int j0 = lane, j1 = lane + 32;
+                float z0 = -INFINITY, z1 = -INFINITY;
+                if (S > 1) {
+                    // block totals go to every block of the cluster (this one included), then the
+                    // S partial logits are summed in slice order by everybody
+                    if (warp == 0) {
+                        const uint32_t dst = smem_u32(xch + s * N), bar = smem_u32(xbar + par);
+                        for (int j = lane; j < N; j += 32) {
+                            float zc = 0.f;
+                            for (int w = 0; w < nparts; ++w) zc += part[w * N + j];
+                            for (int q = 0; q < S; ++q) st_async_f32(map_to_cta(dst + j * 4, q), zc, map_to_cta(bar, q));
+                        }
+                    }
+                    const bool got = wait_or_give_up(xbar + par, static_cast<uint32_t>((it >> 1) & 1), dead, kWaitPolls, true);
+                    if (!__all_sync(0xffffffffu, got)) give_up();
+                    if (j0 < N) {
+                        z0 = 0.f;
+                        for (int q = 0; q < S; ++q) z0 += xch[q * N + j0];
+                    }
+                    if (j1 < N) {
+                        z1 = 0.f;
+                        for (int q = 0; q < S; ++q) z1 += xch[q * N + j1];
+                    }
+                } else {
+                    if (j0 < N) {
+                        z0 = 0.f;
+                        for (int w = 0; w < nparts; ++w) z0 += part[w * N + j0];
+                    }
+                    if (j1 < N) {
+                        z1 = 0.f;
+                        for (int w = 0; w < nparts; ++w) z1 += part[w * N + j1];
+                    }
+                }
+                // softmax over all N experts (Eq. 4), every warp its own copy
+                const float zmax = warp_max(fmaxf(z0, z1));
+                const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
+                const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
+                const float esum = warp_sum(e0 + e1);
+                if (j0 < N) my_gates[j0] = e0 / esum;
+                if (j1 < N) my_gates[j1] = e1 / esum;
+                if (p.gates_out && s == 0 && warp == 0) {
+                    if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
+                    if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
+                }
+                __syncwarp();
+            }
+
+            if (alive) {
+                // weighted sum over the experts in expert order, residual add, one rounding (Eq. 8)
+                const bool valid = meta[st] != 0;
+                const uint4 *rows_vec = reinterpret_cast<const uint4 *>(slot);
+                const uint4 *h_vec = reinterpret_cast<const uint4 *>(hptr);
+                const size_t gvec = static_cast<size_t>(t) * (d / VEC) + static_cast<size_t>(s) * ngrp;
+                for (int grp = tid; grp < ngrp; grp += nc) {
+                    uint4 res = p.residual ? __ldcg(reinterpret_cast<const uint4 *>(p.residual) + gvec + grp) : h_vec[grp];
+                    if (valid) {
+                        float acc[VEC];
+#pragma unroll
+                        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+#pragma unroll 4
+                        for (int j = 0; j < N; ++j) {
+                            float vf[VEC];
+                            E::unpack(rows_vec[j * ngrp + grp], vf);
+                            const float g = my_gates[j];
+#pragma unroll
+                            for (int i = 0; i < VEC; ++i) acc[i] = fmaf(g, vf[i], acc[i]);
+                        }
+                        float rf[VEC];
+                        E::unpack(res, rf);
+#pragma unroll
+                        for (int i = 0; i < VEC; ++i) acc[i] = rf[i] + acc[i];
+                        res = E::pack(acc);
+                    }
+                    if (l == L - 1) reinterpret_cast<uint4 *>(p.out)[gvec + grp] = res;
+                    else reinterpret_cast<uint4 *>(hid)[grp] = res;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + st);  // this warp is done with the slot
+            // the next layer's router reads the hidden slice that all warps have just written
+            if (L > 1) named_bar_sync(kConsumerBarrier, nc);
+            if (++l == L) {
+                l = 0;
+                ++k;
+            }
+        }
+    }
+    // No block of a cluster may leave while a peer can still write into its shared memory.
+    if (S > 1) {
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace mole
