@@ -261,3 +261,175 @@ static int check_common(const void *hidden, const void *ids, const void *lut, co
 
 using namespace mole;
 
+extern "C" {
+
+int mole_layer_forward_ex(const mole_args *a)
+{
+    if (!a || a->struct_size != sizeof(mole_args)) return MOLE_ERR_INVALID_ARG;
+    if (a->flags & ~(MOLE_FLAG_IDS_INT64 | MOLE_FLAG_CHAIN)) return MOLE_ERR_INVALID_ARG;
+    if (a->reserved != 0) return MOLE_ERR_INVALID_ARG;
+    int rc = check_common(a->hidden, a->ids, a->lut, a->w_router, a->out, a->residual, a->B, a->T, a->N, a->d, a->V,
+                          a->dtype);
+    if (rc != MOLE_OK) return rc;
+    const uintptr_t id_align = (a->flags & MOLE_FLAG_IDS_INT64) ? 7u : 3u;
+    if (reinterpret_cast<uintptr_t>(a->ids) & id_align) return MOLE_ERR_INVALID_ARG;
+    if (a->residual && a->residual != a->hidden && a->residual == a->out) return MOLE_ERR_INVALID_ARG;
+    StepLaunch s;
+    s.hidden = a->hidden;
+    s.residual = a->residual;
+    s.row_index = a->ids;
+    s.lut = a->lut;
+    s.w_router = a->w_router;
+    s.out = a->out;
+    s.gates_out = a->gates_out;
+    s.status = a->status;
+    s.lut_stride = 0;
+    s.wr_stride = 0;
+    s.M = static_cast<long long>(a->B) * a->T;
+    s.L = 1;
+    s.N = a->N;
+    s.d = a->d;
+    s.rows = a->V;
+    s.dtype = a->dtype;
+    s.flags = a->flags;
+    s.d_split = a->d_split;
+    s.stream = static_cast<cudaStream_t>(a->stream);
+    return launch_step(s);
+}
+
+int mole_layer_forward(const void *hidden, const int32_t *ids, const void *lut, const void *w_router, void *out, int B,
+                       int T, int N, int d, int V, void *stream)
+{
+    mole_args a;
+    memset(&a, 0, sizeof a);
+    a.struct_size = sizeof a;
+    a.hidden = hidden;
+    a.ids = ids;
+    a.lut = lut;
+    a.w_router = w_router;
+    a.out = out;
+    a.B = B;
+    a.T = T;
+    a.N = N;
+    a.d = d;
+    a.V = V;
+    a.dtype = MOLE_DTYPE_BF16;
+    a.stream = stream;
+    return mole_layer_forward_ex(&a);
+}
+
+int mole_decode_step_ex(const void *hidden_in, const int32_t *ids, const void *lut_base, int64_t lut_layer_stride_bytes,
+                        const void *w_router_base, int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status,
+                        int L, int B, int T, int N, int d, int V, int dtype, int mode, int d_split, void *stream)
+{
+    if (L < 1 || mode < MOLE_STEP_AUTO || mode > MOLE_STEP_CHAINED) return MOLE_ERR_INVALID_ARG;
+    int rc = check_common(hidden_in, ids, lut_base, w_router_base, out, nullptr, B, T, N, d, V, dtype);
+    if (rc != MOLE_OK) return rc;
+    const long long M = static_cast<long long>(B) * T;
+    if (M == 0) return MOLE_OK;
+    if ((lut_layer_stride_bytes & 15) || (wr_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if (mode == MOLE_STEP_AUTO) mode = (L > 1 && M > kFusedMaxTokens) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
+
+    StepLaunch a;
+    a.residual = nullptr;
+    a.row_index = ids;
+    a.gates_out = nullptr;
+    a.status = status;
+    a.lut_stride = lut_layer_stride_bytes;
+    a.wr_stride = wr_layer_stride_bytes;
+    a.M = M;
+    a.N = N;
+    a.d = d;
+    a.rows = V;
+    a.dtype = dtype;
+    a.d_split = d_split;
+    a.stream = static_cast<cudaStream_t>(stream);
+    if (mode == MOLE_STEP_FUSED) {
+        // one launch: every block walks its tokens through all L layers
+        a.hidden = hidden_in;
+        a.lut = lut_base;
+        a.w_router = w_router_base;
+        a.out = out;
+        a.L = L;
+        a.flags = 0;
+        return launch_step(a);
+    }
+    if (L > 1 && (!tmp || !aligned16(tmp) || out == hidden_in || tmp == hidden_in || tmp == out))
+        return MOLE_ERR_INVALID_ARG;
+    // L launches; ping-pong so that the last layer writes `out` and hidden_in is never written
+    const void *src = hidden_in;
+    for (int l = 0; l < L; ++l) {
+        void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
+        a.hidden = src;
+        a.lut = static_cast<const unsigned char *>(lut_base) + static_cast<int64_t>(l) * lut_layer_stride_bytes;
+        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
+        a.out = dst;
+        a.L = 1;
+        a.flags = MOLE_FLAG_CHAIN;
+        rc = launch_step(a);
+        if (rc != MOLE_OK) return rc;
+        src = dst;
+    }
+    return MOLE_OK;
+}
+
+int mole_decode_step(const void *hidden_in, const int32_t *ids, const void *lut_base, int64_t lut_layer_stride_bytes,
+                     const void *w_router_base, int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status,
+                     int L, int B, int T, int N, int d, int V, int dtype, void *stream)
+{
+    return mole_decode_step_ex(hidden_in, ids, lut_base, lut_layer_stride_bytes, w_router_base, wr_layer_stride_bytes, out,
+                               tmp, status, L, B, T, N, d, V, dtype, MOLE_STEP_AUTO, 0, stream);
+}
+
+int mole_decode_step_host(const void *hidden_host, const int32_t *ids_host, void *out_host, void *dev_hidden,
+                          int32_t *dev_ids, void *dev_out, void *dev_tmp, const void *lut_base,
+                          int64_t lut_layer_stride_bytes, const void *w_router_base, int64_t wr_layer_stride_bytes,
+                          uint32_t *status, int L, int B, int T, int N, int d, int V, int dtype, void *stream)
+{
+    if (B < 0 || T < 0 || (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32)) return MOLE_ERR_INVALID_ARG;
+    const long long M = static_cast<long long>(B) * T;
+    if (M == 0) return MOLE_OK;
+    if (!hidden_host || !ids_host || !out_host || !dev_hidden || !dev_ids || !dev_out) return MOLE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t act_bytes = static_cast<size_t>(M) * d * elem_bytes(dtype);
+    MOLE_CUDA_TRY(cudaMemcpyAsync(dev_ids, ids_host, static_cast<size_t>(M) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    MOLE_CUDA_TRY(cudaMemcpyAsync(dev_hidden, hidden_host, act_bytes, cudaMemcpyHostToDevice, st));
+    int rc = mole_decode_step(dev_hidden, dev_ids, lut_base, lut_layer_stride_bytes, w_router_base, wr_layer_stride_bytes,
+                              dev_out, dev_tmp, status, L, B, T, N, d, V, dtype, stream);
+    if (rc != MOLE_OK) return rc;
+    MOLE_CUDA_TRY(cudaMemcpyAsync(out_host, dev_out, act_bytes, cudaMemcpyDeviceToHost, st));
+    return MOLE_OK;
+}
+
+int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads, int *out_smem_bytes,
+              int *out_stages, int *out_blocks_per_sm)
+{
+    StepPlan plan;
+    int rc = plan_step(M, L, N, d, dtype, d_split, &plan);
+    if (rc != MOLE_OK) return rc;
+    if (out_d_split) *out_d_split = plan.d_split;
+    if (out_threads) *out_threads = plan.threads;
+    if (out_smem_bytes) *out_smem_bytes = plan.smem;
+    if (out_stages) *out_stages = plan.stages;
+    if (out_blocks_per_sm) *out_blocks_per_sm = plan.blocks_per_sm;
+    return MOLE_OK;
+}
+
+const char *mole_status_string(int code)
+{
+    switch (code) {
+        case MOLE_OK: return "ok";
+        case MOLE_ERR_INVALID_ARG: return "invalid argument";
+        case MOLE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case MOLE_ERR_CUDA: return "CUDA runtime error";
+        case MOLE_ERR_NOMEM: return "out of memory";
+        case MOLE_ERR_TOO_LARGE: return "size beyond the stated maximum";
+        default: return "unknown status";
+    }
+}
+
+const char *mole_last_cuda_error(void) { return g_cuda_error; }
+
+int mole_version(void) { return MOLE_VERSION; }
+
+}  // extern "C"
