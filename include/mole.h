@@ -46,7 +46,7 @@
 extern "C" {
 #endif
 
-#define MOLE_VERSION 100
+#define MOLE_VERSION 200
 
 /* every entry point is exported from the shared library with default visibility */
 #if defined(__GNUC__)
@@ -79,10 +79,10 @@ extern "C" {
                                   after it has.  Only valid if ids, lut and w_router are not       \
                                   written by that previous kernel. */
 
-/* mole_args.variant: how a token's d columns are spread over thread blocks */
-#define MOLE_VARIANT_AUTO 0    /* chosen from M, N, d */
-#define MOLE_VARIANT_REPLICATE 1 /* each of d_split blocks recomputes the full router */
-#define MOLE_VARIANT_CLUSTER 2 /* d_split blocks form a cluster and exchange partial logits */
+/* mole_decode_step_ex mode: how the L layers of a step are launched */
+#define MOLE_STEP_AUTO 0    /* fused unless the batch is large (then chained) */
+#define MOLE_STEP_FUSED 1   /* ONE launch: every block walks its tokens through all L layers */
+#define MOLE_STEP_CHAINED 2 /* L launches chained with programmatic dependent launch */
 
 /*
  * mole_layer_forward -- the fused layer, bf16, Eq. 4 + Eq. 8 (router, softmax over all N
@@ -117,8 +117,9 @@ typedef struct mole_args {
     uint32_t *status;      /* device status word (MOLE_STATUS_* bits OR-ed in), or NULL */
     int32_t B, T, N, d, V;
     int32_t dtype;         /* MOLE_DTYPE_* */
-    int32_t variant;       /* MOLE_VARIANT_* */
-    int32_t d_split;       /* blocks per token (1, 2, 4 or 8; d/d_split must stay a multiple of the vector width); 0 = auto */
+    int32_t reserved;      /* must be 0 */
+    int32_t d_split;       /* blocks per token (1, 2, 4 or 8; d/d_split must stay a multiple of the vector width); 0 = auto.
+                              The d_split blocks of a token form a thread-block cluster and exchange partial logits. */
     void *stream;          /* cudaStream_t */
 } mole_args;
 
@@ -128,17 +129,33 @@ MOLE_API int mole_layer_forward_ex(const mole_args *args);
  * mole_decode_step -- L layers back to back (Eq. 8 applied layer after layer; the attention
  * and shared-expert blocks that a full model runs in between are not part of this library).
  * Layer l reads table lut_base + l*lut_layer_stride_bytes and router w_router_base +
- * l*wr_layer_stride_bytes; its output is the next layer's hidden.  Launches are chained with
- * programmatic dependent launch, so layer l+1's row gathers (which depend only on ids) are in
- * flight while layer l finishes.
- *   hidden_in device [M][d], read only      out device [M][d] final result (may be == hidden_in
- *   tmp       device [M][d] scratch for the ping-pong (may be NULL when L == 1)   only if L == 1)
+ * l*wr_layer_stride_bytes; its output, rounded to the storage type, is the next layer's hidden.
+ *   hidden_in device [M][d], read only (FUSED mode also accepts out == hidden_in)
+ *   out       device [M][d] final result
+ *   tmp       device [M][d] scratch for the ping-pong of CHAINED mode (may be NULL when L == 1
+ *             or when the mode is MOLE_STEP_FUSED)
  * dtype as MOLE_DTYPE_*.  status (device, may be NULL) as in mole_args.
+ *
+ * Two ways to run it, with bit-identical results for equal d_split:
+ *  - FUSED: tokens are independent and a token's chain h_0 -> h_1 -> ... -> h_L needs nothing
+ *    but its own rows, so one launch lets each block keep a token's running hidden slice in
+ *    shared memory across all L layers while the rows of later layers (which depend only on
+ *    the id) are already streaming in.  No hidden state travels through global memory between
+ *    layers and there are no L-1 launch boundaries.
+ *  - CHAINED: L launches of the single-layer kernel with programmatic dependent launch; layer
+ *    l+1's first row gathers are in flight while layer l finishes.  This is what a model that
+ *    runs other work between the layers gets by calling mole_layer_forward_ex per layer.
+ * mole_decode_step picks FUSED up to 4096 tokens and CHAINED above; _ex lets the caller choose
+ * and force d_split (0 = auto).
  */
 MOLE_API int mole_decode_step(const void *hidden_in, const int32_t *ids, const void *lut_base,
                      int64_t lut_layer_stride_bytes, const void *w_router_base,
                      int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status, int L, int B,
                      int T, int N, int d, int V, int dtype, void *stream);
+MOLE_API int mole_decode_step_ex(const void *hidden_in, const int32_t *ids, const void *lut_base,
+                     int64_t lut_layer_stride_bytes, const void *w_router_base,
+                     int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status, int L, int B,
+                     int T, int N, int d, int V, int dtype, int mode, int d_split, void *stream);
 
 /*
  * mole_decode_step_host -- mole_decode_step for a caller whose activations live in HOST
@@ -254,10 +271,11 @@ MOLE_API const char *mole_status_string(int code);
 MOLE_API const char *mole_last_cuda_error(void);
 MOLE_API int mole_version(void);
 
-/* launch shape mole_layer_forward_ex would pick (for tests and benchmarks): blocks per token,
- * threads per block, dynamic shared memory, variant.  Pure host arithmetic, no CUDA call. */
-MOLE_API int mole_plan(int M, int N, int d, int dtype, int variant, int d_split, int *out_d_split, int *out_threads,
-              int *out_smem_bytes, int *out_variant);
+/* launch shape the library would pick for M tokens and L layers in one launch (L = 1: a single
+ * layer): blocks per token, threads per block, dynamic shared memory, depth of the row ring,
+ * resident blocks per SM.  Pure host arithmetic, no CUDA call. */
+MOLE_API int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads,
+              int *out_smem_bytes, int *out_stages, int *out_blocks_per_sm);
 
 #ifdef __cplusplus
 }

@@ -20,11 +20,11 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, ERR_NOMEM, ERR_TOO_LARGE =
 STATUS_BAD_ID, STATUS_TIMEOUT = 1, 2
 DTYPE_BF16, DTYPE_F32 = 0, 1
 FLAG_IDS_INT64, FLAG_CHAIN = 1, 2
-VARIANT_AUTO, VARIANT_REPLICATE, VARIANT_CLUSTER = 0, 1, 2
+STEP_AUTO, STEP_FUSED, STEP_CHAINED = 0, 1, 2
 
 # every symbol include/mole.h declares
 EXPORTS = (
-    "mole_layer_forward", "mole_layer_forward_ex", "mole_decode_step", "mole_decode_step_host",
+    "mole_layer_forward", "mole_layer_forward_ex", "mole_decode_step", "mole_decode_step_ex", "mole_decode_step_host",
     "mole_dedup_ids", "mole_dedup_ids_static", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
     "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_buffers",
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan",
@@ -37,7 +37,7 @@ class MoleArgs(ctypes.Structure):
         ("hidden", c_void_p), ("ids", c_void_p), ("lut", c_void_p), ("w_router", c_void_p), ("out", c_void_p),
         ("residual", c_void_p), ("gates_out", c_void_p), ("status", c_void_p),
         ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
-        ("dtype", c_int32), ("variant", c_int32), ("d_split", c_int32),
+        ("dtype", c_int32), ("reserved", c_int32), ("d_split", c_int32),
         ("stream", c_void_p),
     ]
 
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.mole_layer_forward_ex.argtypes = [POINTER(MoleArgs)]
         L.mole_decode_step.argtypes = [vp, ip, vp, c_int64, vp, c_int64, vp, vp, vp, c_int, c_int, c_int, c_int,
                                        c_int, c_int, c_int, vp]
+        L.mole_decode_step_ex.argtypes = [vp, ip, vp, c_int64, vp, c_int64, vp, vp, vp, c_int, c_int, c_int, c_int,
+                                          c_int, c_int, c_int, c_int, c_int, vp]
         L.mole_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, c_int64, vp, c_int64, vp, c_int, c_int,
                                             c_int, c_int, c_int, c_int, c_int, vp]
         L.mole_dedup_ids.argtypes = [ip, c_int, c_int, ip, ip, ip, ip, vp, vp]
@@ -87,7 +89,7 @@ def lib() -> ctypes.CDLL:
         L.mole_last_cuda_error.restype = c_char_p
         L.mole_version.argtypes = []
         L.mole_plan.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
-                                POINTER(c_int), POINTER(c_int)]
+                                POINTER(c_int), POINTER(c_int), POINTER(c_int)]
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is not c_char_p:
@@ -127,7 +129,7 @@ def _dev(t: torch.Tensor, name: str):
 
 
 def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_out=None, status=None,
-                  variant: int = VARIANT_AUTO, d_split: int = 0, chain: bool = False, stream=None, B=None, T=None):
+                  d_split: int = 0, chain: bool = False, stream=None, B=None, T=None):
     """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d],
     w_router [d][N]; returns out (allocated like hidden if not given)."""
     for name, t in (("hidden", hidden), ("ids", ids), ("lut", lut), ("w_router", w_router)):
@@ -157,7 +159,7 @@ def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_
     a.hidden, a.ids, a.lut, a.w_router, a.out = _ptr(hidden), _ptr(ids), _ptr(lut), _ptr(w_router), _ptr(out)
     a.residual, a.gates_out, a.status = _ptr(residual), _ptr(gates_out), _ptr(status)
     a.B, a.T, a.N, a.d, a.V = B, T, N, d, V
-    a.dtype, a.variant, a.d_split = tag, variant, d_split
+    a.dtype, a.reserved, a.d_split = tag, 0, d_split
     a.stream = _stream(stream)
     _check(lib().mole_layer_forward_ex(ctypes.byref(a)), "mole_layer_forward_ex")
     return out
@@ -172,8 +174,22 @@ def layer_forward_basic(hidden, ids, lut, w_router, out, stream=None):
     return out
 
 
-def decode_step(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None):
-    """mole_decode_step: luts [L][V][N][d], w_routers [L][d][N]; returns out."""
+def decode_step(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None, mode: int = STEP_AUTO,
+                d_split: int = 0):
+    """mole_decode_step_ex: luts [L][V][N][d], w_routers [L][d][N]; returns out.  mode: STEP_AUTO,
+    STEP_FUSED (one launch over all layers) or STEP_CHAINED (L launches, needs tmp when L > 1)."""
+    L, V, N, d = luts.shape
+    M = ids.numel()
+    tag = _dtype_tag(hidden_in)
+    _check(lib().mole_decode_step_ex(_ptr(hidden_in), _ptr(ids), _ptr(luts), luts.stride(0) * luts.element_size(),
+                                     _ptr(w_routers), w_routers.stride(0) * w_routers.element_size(), _ptr(out),
+                                     _ptr(tmp), _ptr(status), L, M, 1, N, d, V, tag, mode, d_split, _stream(stream)),
+           "mole_decode_step_ex")
+    return out
+
+
+def decode_step_basic(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None):
+    """mole_decode_step, the plain entry point (mode and split chosen by the library)."""
     L, V, N, d = luts.shape
     M = ids.numel()
     tag = _dtype_tag(hidden_in)
@@ -303,12 +319,13 @@ class OffloadContext:
             pass
 
 
-def plan(M: int, N: int, d: int, dtype: int = DTYPE_BF16, variant: int = VARIANT_AUTO, d_split: int = 0):
-    """mole_plan: (d_split, threads, smem_bytes, variant) the launch would use."""
-    a, b, c, e = c_int(), c_int(), c_int(), c_int()
-    _check(lib().mole_plan(M, N, d, dtype, variant, d_split, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
-                           ctypes.byref(e)), "mole_plan")
-    return a.value, b.value, c.value, e.value
+def plan(M: int, N: int, d: int, dtype: int = DTYPE_BF16, d_split: int = 0, L: int = 1):
+    """mole_plan: (d_split, threads, smem_bytes, stages, blocks_per_sm) of a launch over M tokens
+    and L layers (L = 1: a single layer)."""
+    a, b, c, e, f = c_int(), c_int(), c_int(), c_int(), c_int()
+    _check(lib().mole_plan(M, L, N, d, dtype, d_split, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                           ctypes.byref(e), ctypes.byref(f)), "mole_plan")
+    return a.value, b.value, c.value, e.value, f.value
 
 
 def version() -> int:

@@ -226,8 +226,8 @@ int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, in
     if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
     if (max_tokens < 1 || n_buffers < 1 || n_buffers > 16) return MOLE_ERR_INVALID_ARG;
     if (max_tokens > 65535) return MOLE_ERR_TOO_LARGE;
-    LayerPlan plan;
-    int rc = plan_layer(max_tokens, N, d, dtype, MOLE_VARIANT_AUTO, 0, &plan);
+    StepPlan plan;
+    int rc = plan_step(max_tokens, 1, N, d, dtype, 0, &plan);
     if (rc != MOLE_OK) return rc;
     if (V < 1) return MOLE_ERR_UNSUPPORTED_SHAPE;
     mole_offload_ctx *c = new (std::nothrow) mole_offload_ctx;
@@ -299,7 +299,7 @@ int mole_layer_forward_offload(mole_offload_ctx *c, int b, const void *hidden, c
         return MOLE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     MOLE_CUDA_TRY(cudaStreamWaitEvent(st, B.ready, 0));
-    LayerLaunch a;
+    StepLaunch a;
     a.hidden = hidden;
     a.residual = nullptr;
     a.row_index = B.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
@@ -308,16 +308,18 @@ int mole_layer_forward_offload(mole_offload_ctx *c, int b, const void *hidden, c
     a.out = out;
     a.gates_out = nullptr;
     a.status = status;
+    a.lut_stride = 0;
+    a.wr_stride = 0;
     a.M = M;
+    a.L = 1;
     a.N = c->N;
     a.d = c->d;
     a.rows = c->max_tokens;
     a.dtype = c->dtype;
     a.flags = 0;
-    a.variant = MOLE_VARIANT_AUTO;
     a.d_split = 0;
     a.stream = st;
-    int rc = launch_layer(a);
+    int rc = launch_step(a);
     if (rc != MOLE_OK) return rc;
     MOLE_CUDA_TRY(cudaEventRecord(B.consumed, st));
     return MOLE_OK;
