@@ -33,7 +33,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert lib.mole_version() == 100
+    assert lib.mole_version() == 200
     seen = {lib.mole_status_string(c).decode() for c in range(6)}
     assert len(seen) == 6 and "ok" in seen
     assert lib.mole_status_string(99).decode() == "unknown status"
@@ -46,20 +46,27 @@ def test_args_struct_layout_matches_header(lib):
 
 def test_plan_shapes():
     P = binding.plan
-    # large batches: one block per token while a token's rows fit beside other blocks
-    assert P(16384, 16, 1024)[0] == 1 and P(16384, 16, 768)[0] == 1
+    # large batches, single layer: one block per token, a ring of slots, one producer warp
+    for d in (768, 1024):
+        s, threads, smem, stages, per_sm = P(16384, 16, d)
+        assert s == 1 and 2 <= stages <= 8 and smem <= 227 * 1024 and threads == d // 8 + 32
+        assert per_sm * smem <= 228 * 1024 and per_sm * stages >= 4
     # the 1B-shaped rows (128 KB per token) are always split
-    s, threads, smem, variant = P(16384, 32, 2048)
-    assert s >= 4 and smem <= 48 * 1024 and variant == binding.VARIANT_CLUSTER
+    s, threads, smem, stages, per_sm = P(16384, 32, 2048)
+    assert s >= 2 and stages >= 2 and smem <= 227 * 1024
     # few tokens: split to occupy the SMs
     assert P(64, 16, 768)[0] >= 2 and P(1, 16, 768)[0] >= 2
-    # explicit split and variant are honoured
-    assert P(64, 16, 768, binding.DTYPE_BF16, binding.VARIANT_REPLICATE, 4)[0::3] == (4, binding.VARIANT_REPLICATE)
-    # a split of one needs no cluster
-    assert P(64, 16, 768, binding.DTYPE_BF16, binding.VARIANT_CLUSTER, 1)[3] == binding.VARIANT_REPLICATE
+    # an explicit split is honoured
+    assert P(64, 16, 768, binding.DTYPE_BF16, 4)[0] == 4 and P(64, 16, 768, binding.DTYPE_BF16, 1)[0] == 1
+    # a fused 12-layer step carries the router slice in every slot: slots about twice as large
+    one = P(256, 16, 768, binding.DTYPE_BF16, 1, 1)
+    fused = P(256, 16, 768, binding.DTYPE_BF16, 1, 12)
+    assert fused[3] >= 2 and fused[2] <= 227 * 1024 and fused[2] / fused[3] > 1.5 * (one[2] - 16 * 768 * 2) / one[3]
+    # never a deeper ring than the items a block will see
+    assert P(1, 16, 768, binding.DTYPE_BF16, 1, 1)[3] == 2 and P(1, 16, 768, binding.DTYPE_BF16, 1, 3)[3] == 3
     # fp32 tiny shape
-    s, threads, smem, variant = P(64, 4, 64, binding.DTYPE_F32)
-    assert s == 1 and threads == 32 and smem >= 4 * 64 * 4
+    s, threads, smem, stages, per_sm = P(64, 4, 64, binding.DTYPE_F32)
+    assert threads == 64 and smem >= 2 * 4 * (64 // s) * 4
 
 
 def test_plan_rejects_bad_shapes():
@@ -71,10 +78,13 @@ def test_plan_rejects_bad_shapes():
         binding.plan(64, 16, 768, 7)
     assert e.value.code == binding.ERR_INVALID_ARG
     with pytest.raises(binding.MoleError) as e:
-        binding.plan(64, 16, 768, binding.DTYPE_BF16, 0, 3)
+        binding.plan(64, 16, 768, binding.DTYPE_BF16, 3)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.MoleError) as e:
+        binding.plan(64, 16, 768, binding.DTYPE_BF16, 0, 0)  # zero layers
     assert e.value.code == binding.ERR_INVALID_ARG
     with pytest.raises(binding.MoleError) as e:  # 768 / 16 columns is not a whole number of vectors
-        binding.plan(64, 16, 40, binding.DTYPE_BF16, 0, 8)
+        binding.plan(64, 16, 40, binding.DTYPE_BF16, 8)
     assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
 
 
@@ -115,7 +125,7 @@ def test_ex_rejects_bad_struct(lib):
     a.residual = good + 0x100
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
     a.residual = None
-    a.variant = 9
+    a.reserved = 9
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
 
 
@@ -124,9 +134,13 @@ def test_decode_step_and_offload_argument_checks(lib):
     ds = lib.mole_decode_step
     assert ds(good, good, good, 16, good, 16, good + 0x100, None, None, 0, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
     assert ds(good, good, good, 8, good, 16, good + 0x100, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
-    assert ds(good, good, good, 16, good, 16, good + 0x100, None, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
-    assert ds(good, good, good, 16, good, 16, good, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, None) == binding.ERR_INVALID_ARG
     assert ds(None, None, None, 16, None, 16, None, None, None, 2, 0, 1, 16, 768, 100, 0, None) == binding.OK
+    dx = lib.mole_decode_step_ex
+    CH = binding.STEP_CHAINED
+    # chained launches need a scratch buffer and cannot run in place
+    assert dx(good, good, good, 16, good, 16, good + 0x100, None, None, 2, 4, 1, 16, 768, 100, 0, CH, 0, None) == binding.ERR_INVALID_ARG
+    assert dx(good, good, good, 16, good, 16, good, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, CH, 0, None) == binding.ERR_INVALID_ARG
+    assert dx(good, good, good, 16, good, 16, good + 0x100, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, 7, 0, None) == binding.ERR_INVALID_ARG
     dd = lib.mole_dedup_ids
     assert dd(good, -1, 10, good, good, good, good, None, None) == binding.ERR_INVALID_ARG
     assert dd(good, (1 << 20) + 1, 10, good, good, good, good, None, None) == binding.ERR_TOO_LARGE

@@ -47,7 +47,7 @@ def test_tiny_config_fp32_two_layers_every_element():
         h_ref = out.cpu().numpy()  # feed the oracle the bytes the next GPU layer sees
 
 
-# ---- bf16 parity over shapes, splits and variants ---------------------------------------------------
+# ---- bf16 parity over shapes and splits ---------------------------------------------------------------
 
 CASES = [
     # M, N, d, V
@@ -63,6 +63,8 @@ CASES = [
     (9, 33, 256, 30),
     (4, 1, 64, 8),
     (6, 12, 2560, 16),      # d-groups (320) beyond 256 threads: strided loops
+    (1500, 16, 768, 900),   # more tokens than resident blocks: every block loops over several tokens
+    (2100, 8, 256, 64),
 ]
 
 
@@ -76,16 +78,15 @@ def test_bf16_parity_auto_plan(M, N, d, V):
     check_gates(gates, gref)
 
 
-@pytest.mark.parametrize("variant", [mole.VARIANT_REPLICATE, mole.VARIANT_CLUSTER])
 @pytest.mark.parametrize("split", [1, 2, 4, 8])
-@pytest.mark.parametrize("N,d", [(16, 768), (32, 2048), (5, 512), (4, 64)])
-def test_bf16_parity_every_split_and_variant(variant, split, N, d):
+@pytest.mark.parametrize("N,d", [(16, 768), (32, 2048), (5, 512), (4, 64), (8, 256), (64, 512)])
+def test_bf16_parity_every_split(split, N, d):
     if d % (split * 8) != 0:
         pytest.skip("column slice would not be a whole number of 16-byte vectors")
     M, V = 37, 211
     hidden, ids, lut, wr = rand_case(M, N, d, V, seed=d + N + split)
     ref, gref, _ = oracle_layer(hidden, ids, lut, wr)
-    out, gates, status = run_gpu(hidden, ids, lut, wr, variant=variant, d_split=split)
+    out, gates, status = run_gpu(hidden, ids, lut, wr, d_split=split)
     assert status == 0
     check_out(out, ref)
     check_gates(gates, gref)
@@ -95,8 +96,9 @@ def test_fp32_parity_splits():
     M, N, d, V = 21, 8, 256, 50
     hidden, ids, lut, wr = rand_case(M, N, d, V, seed=5, dtype=torch.float32)
     ref, gref, _ = oracle.layer_lookup(hidden.numpy(), ids.numpy(), lut.numpy(), wr.numpy())
-    for variant, split in ((0, 0), (1, 2), (2, 4), (2, 8)):
-        out, gates, status = run_gpu(hidden, ids, lut, wr, variant=variant, d_split=split)
+    for split in (0, 1, 2, 4, 8):
+        out, gates, status = run_gpu(hidden, ids, lut, wr, d_split=split)
+        assert status == 0
         check_out(out, ref, torch.float32)
         check_gates(gates, gref)
 
@@ -141,8 +143,8 @@ def _encoded_table_bits(V, N, d, kind):
 
 
 @pytest.mark.parametrize("kind", ["hash", "id_lo", "id_hi", "expert", "col_lo", "col_hi"])
-@pytest.mark.parametrize("N,d,split,variant", [(16, 768, 0, 0), (16, 768, 4, 1), (32, 2048, 0, 0), (5, 512, 2, 2)])
-def test_gather_bit_exact_with_one_hot_gates(kind, N, d, split, variant):
+@pytest.mark.parametrize("N,d,split", [(16, 768, 0), (16, 768, 4), (16, 768, 1), (32, 2048, 0), (5, 512, 2)])
+def test_gather_bit_exact_with_one_hot_gates(kind, N, d, split):
     V, M = 300, 40
     tb = _encoded_table_bits(V, N, d, kind)
     lut = torch.from_numpy(tb.view(np.int16)).view(torch.bfloat16)
@@ -151,7 +153,7 @@ def test_gather_bit_exact_with_one_hot_gates(kind, N, d, split, variant):
     zeros = torch.zeros(M, d, dtype=torch.bfloat16)
     for jstar in sorted({0, N // 2, N - 1}):
         hidden, wr = _one_hot_inputs(M, N, d, jstar, c0=(3 * jstar + 1) % d)
-        out, gates, status = run_gpu(hidden, ids, lut, wr, residual=zeros, variant=variant, d_split=split)
+        out, gates, status = run_gpu(hidden, ids, lut, wr, residual=zeros, d_split=split)
         want_g = np.zeros((M, N), dtype=np.float32)
         want_g[:, jstar] = 1.0
         assert np.array_equal(gates.cpu().numpy(), want_g)
@@ -200,16 +202,15 @@ def test_token_permutation_and_batch_size_do_not_change_a_token():
     M, N, d, V = 96, 16, 768, 500
     hidden, ids, lut, wr = rand_case(M, N, d, V, seed=11, ids_kind="zipf")
     lut_d, wr_d = lut.to(DEV), wr.to(DEV)
-    base = mole.layer_forward(hidden.to(DEV), ids.to(DEV), lut_d, wr_d, variant=mole.VARIANT_CLUSTER, d_split=2)
+    base = mole.layer_forward(hidden.to(DEV), ids.to(DEV), lut_d, wr_d, d_split=2)
     perm = torch.randperm(M, generator=torch.Generator().manual_seed(1))
-    permuted = mole.layer_forward(hidden[perm].to(DEV), ids[perm].to(DEV), lut_d, wr_d, variant=mole.VARIANT_CLUSTER,
-                                  d_split=2)
+    permuted = mole.layer_forward(hidden[perm].to(DEV), ids[perm].to(DEV), lut_d, wr_d, d_split=2)
     assert torch.equal(permuted, base[perm.to(DEV)])
     for t in (0, 17, 95):  # the same token alone, same launch shape
         one = mole.layer_forward(hidden[t:t + 1].to(DEV), ids[t:t + 1].to(DEV), lut_d, wr_d,
-                                 variant=mole.VARIANT_CLUSTER, d_split=2)
+                                 d_split=2)
         assert torch.equal(one[0], base[t])
-    again = mole.layer_forward(hidden.to(DEV), ids.to(DEV), lut_d, wr_d, variant=mole.VARIANT_CLUSTER, d_split=2)
+    again = mole.layer_forward(hidden.to(DEV), ids.to(DEV), lut_d, wr_d, d_split=2)
     assert torch.equal(again, base)  # run-to-run deterministic
 
 
@@ -226,17 +227,12 @@ def test_in_place_output_and_separate_residual():
     M, N, d, V = 70, 16, 768, 90
     hidden, ids, lut, wr = rand_case(M, N, d, V, seed=13)
     ref, _, _ = oracle_layer(hidden, ids, lut, wr)
-    for variant, split in ((0, 0), (0, 1), (2, 4)):
+    for split in (0, 1, 2, 4):
         h = hidden.to(DEV).clone()
-        out = mole.layer_forward(h, ids.to(DEV), lut.to(DEV), wr.to(DEV), out=h, variant=variant, d_split=split)
+        out = mole.layer_forward(h, ids.to(DEV), lut.to(DEV), wr.to(DEV), out=h, d_split=split)
         torch.cuda.synchronize()
         assert out.data_ptr() == h.data_ptr()
         check_out(h, ref)
-    # replicated routers cannot run in place: the call is refused, nothing is launched
-    h = hidden.to(DEV).clone()
-    with pytest.raises(mole.MoleError) as e:
-        mole.layer_forward(h, ids.to(DEV), lut.to(DEV), wr.to(DEV), out=h, variant=mole.VARIANT_REPLICATE, d_split=2)
-    assert e.value.code == mole.ERR_INVALID_ARG
     res = torch.empty(M, d).normal_(0, 1, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
     ref_r, _, _ = oracle_layer(hidden, ids, lut, wr, residual=res)
     out, _, _ = run_gpu(hidden, ids, lut, wr, residual=res)
@@ -260,8 +256,8 @@ def test_bad_ids_leave_the_residual_and_raise_the_status_bit():
     ids[3], ids[8] = -1, V
     ref, gref, bad = oracle_layer(hidden, ids, lut, wr)
     assert bad == 2
-    for variant, split in ((0, 0), (1, 2), (2, 2)):
-        out, gates, status = run_gpu(hidden, ids, lut, wr, variant=variant, d_split=split)
+    for split in (0, 1, 2):
+        out, gates, status = run_gpu(hidden, ids, lut, wr, d_split=split)
         assert status & mole.STATUS_BAD_ID and not status & mole.STATUS_TIMEOUT
         check_out(out, ref)
         assert np.array_equal(bits(out)[3], bits(hidden)[3]) and np.array_equal(bits(out)[8], bits(hidden)[8])
@@ -289,28 +285,67 @@ def test_maximum_sizes_N64_and_wide_d():
 
 # ---- chained layers ------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("M,N,d,L", [(64, 16, 768, 5), (3, 16, 1024, 4), (40, 32, 2048, 3), (300, 16, 768, 2), (8, 4, 64, 1)])
-def test_decode_step_equals_layer_after_layer(M, N, d, L):
-    V = 400
+def _step_case(M, N, d, L, V=400):
     g = torch.Generator().manual_seed(M + L)
     luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16).to(DEV)
     wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
     hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
     ids = torch.from_numpy(inputs.zipf_ids(M, V, seed=4)).to(DEV)
-    out = torch.empty_like(hidden)
-    tmp = torch.empty_like(hidden)
+    return luts, wrs, hidden, ids
+
+
+@pytest.mark.parametrize("M,N,d,L,split", [(64, 16, 768, 5, 1), (64, 16, 768, 5, 2), (3, 16, 1024, 4, 4), (40, 32, 2048, 3, 8),
+                                           (300, 16, 768, 2, 1), (8, 4, 64, 1, 1), (9, 5, 512, 3, 2), (700, 8, 256, 3, 1),
+                                           (1300, 16, 768, 2, 2)])
+def test_decode_step_fused_and_chained_equal_layer_after_layer(M, N, d, L, split):
+    luts, wrs, hidden, ids = _step_case(M, N, d, L)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     keep = hidden.clone()
-    mole.decode_step(hidden, ids, luts, wrs, out, tmp, status=status)
+    fused = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), None, status=status,
+                             mode=mole.STEP_FUSED, d_split=split)
+    chained = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status,
+                               mode=mole.STEP_CHAINED, d_split=split)
     h = hidden
-    for l in range(L):  # single layers, each already checked against the oracle above
+    for l in range(L):  # single layers, each checked against the oracle
         ref, _, _ = oracle_layer(h, ids, luts[l], wrs[l])
-        h = mole.layer_forward(h, ids, luts[l], wrs[l])
+        h = mole.layer_forward(h, ids, luts[l], wrs[l], d_split=split)
         check_out(h, ref)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    assert torch.equal(out, h)
+    assert torch.equal(fused, h) and torch.equal(chained, h)  # same split => same bits
     assert torch.equal(hidden, keep)  # the input is never written
+
+
+@pytest.mark.parametrize("M,N,d,L", [(64, 16, 768, 12), (256, 16, 1024, 6), (16, 32, 2048, 4), (1, 16, 768, 12)])
+def test_decode_step_auto_plan_against_the_oracle_chain(M, N, d, L):
+    luts, wrs, hidden, ids = _step_case(M, N, d, L, V=300)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = mole.decode_step_basic(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # the oracle, layer after layer, each layer fed the storage-type rounding of the previous one
+    h = hidden
+    for l in range(L):
+        ref, _, _ = oracle_layer(h, ids, luts[l], wrs[l])
+        h = torch.from_numpy(ref).to(torch.bfloat16)
+    # rounding decisions may differ from the oracle's by one ulp per layer and then propagate
+    err = np.abs(as_f64(out) - as_f64(h))
+    assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(as_f64(h)))).all(), float(err.max())
+
+
+def test_decode_step_fused_in_place_and_bad_ids():
+    M, N, d, L = 50, 16, 768, 4
+    luts, wrs, hidden, ids = _step_case(M, N, d, L)
+    ids[7], ids[31] = -2, 400
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    want = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status,
+                            mode=mole.STEP_CHAINED, d_split=1)
+    h = hidden.clone()
+    mole.decode_step(h, ids, luts, wrs, h, None, status=status, mode=mole.STEP_FUSED, d_split=1)
+    torch.cuda.synchronize()
+    assert int(status.item()) == mole.STATUS_BAD_ID
+    assert torch.equal(h, want)
+    assert torch.equal(h[7], hidden[7]) and torch.equal(h[31], hidden[31])  # no routed term in any layer
 
 
 def test_decode_step_host_round_trip():
