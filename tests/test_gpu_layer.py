@@ -84,6 +84,11 @@ def test_bf16_parity_every_split(split, N, d):
     if d % (split * 8) != 0:
         pytest.skip("column slice would not be a whole number of 16-byte vectors")
     M, V = 37, 211
+    try:
+        mole.plan(M, N, d, mole.DTYPE_BF16, split)
+    except mole.MoleError as e:  # two ring slots of this split do not fit in shared memory
+        assert e.code == mole.ERR_UNSUPPORTED_SHAPE and N * (d // split) * 2 * 3 > 227 * 1024
+        pytest.skip("this split does not fit")
     hidden, ids, lut, wr = rand_case(M, N, d, V, seed=d + N + split)
     ref, gref, _ = oracle_layer(hidden, ids, lut, wr)
     out, gates, status = run_gpu(hidden, ids, lut, wr, d_split=split)
