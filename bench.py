@@ -35,6 +35,9 @@ METRIC = "MoLE layer tokens/s (L-layer decode step) and achieved HBM GB/s"
 UNIT = "tokens/s"
 N_BATCHES = 32          # distinct id batches the steps rotate through
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
+TRAFFIC = {}
 
 
 def parse_args():
@@ -209,7 +212,7 @@ def workload_config(sh, L, M, args):
 class StepGraphs:
     """One CUDA graph per id batch; a graph holds the L chained layer launches of one step."""
 
-    def __init__(self, mole, luts, wrs, hidden, id_batches):
+    def __init__(self, mole, luts, wrs, hidden, id_batches, mode=0):
         import torch
 
         self.torch, self.graphs = torch, []
@@ -220,13 +223,13 @@ class StepGraphs:
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
             for ids in id_batches:  # warm-up launches outside capture (sets kernel attributes)
-                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status)
+                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status, mode=mode)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         for ids in id_batches:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status)
+                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status, mode=mode)
             self.graphs.append(g)
 
     def run(self, k0, k1):
@@ -289,8 +292,9 @@ def run_mole(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- headline: K steps of the L-layer chained step ---------------------------------------------------
+    # ---- headline: K steps of the L-layer decode step, as mole_decode_step runs it ------------------------
     hidden = hidden_all[:M].contiguous()
+    fused = not (L > 1 and M > 4096)  # mole_decode_step's own choice: one fused launch up to 4096 tokens
     graphs = StepGraphs(mole, luts, wrs, hidden, batches_for(M))
     graphs.run(0, max(args.warmup, 3))
     barrier()
@@ -304,9 +308,9 @@ def run_mole(args):
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * M * args.steps / (ms * 1e-3)
-    launches = args.steps * L
-    layer_bytes = sh.layer_bytes(M)
-    achieved = layer_bytes / (ms * 1e-3 / launches) / 1e9
+    launches = args.steps * (1 if fused else L)
+    launch_bytes = sh.step_bytes(M, L) if fused else sh.layer_bytes(M)
+    achieved = launch_bytes / (ms * 1e-3 / launches) / 1e9
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -315,8 +319,9 @@ def run_mole(args):
         "tokens_per_s_per_layer": value * L,
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "kernel": "mole_layer_kernel", "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": layer_bytes, "us_per_launch": ms * 1e3 / launches},
+                     "traffic": TRAFFIC.get((sh.name, M, L)), "kernel": "mole_step_kernel", "peak_source": peak_src,
+                     "launch": ("one fused launch per step (all %d layers)" % L) if fused else "one launch per layer, chained",
+                     "algorithmic_bytes_per_launch": launch_bytes, "us_per_launch": ms * 1e3 / launches},
         "clocks": clocks.summary(),
     }
 
@@ -360,11 +365,19 @@ def run_mole(args):
             hid = hidden_all[:m].contiguous()
             bl = batches_for(m)
             steps_m = max(50, min(args.steps, int(2e6 // max(m, 64))))
-            g = StepGraphs(mole, luts, wrs, hid, bl)
+            g = StepGraphs(mole, luts, wrs, hid, bl, mode=mole.STEP_CHAINED)
             g.run(0, 20)
             torch.cuda.synchronize()
             ms_m = timed_ms(torch, lambda: g.run(0, steps_m))
             us_layer = ms_m * 1e3 / (steps_m * L)
+            del g
+            us_fused = None
+            if m <= 4096:
+                g = StepGraphs(mole, luts, wrs, hid, bl, mode=mole.STEP_FUSED)
+                g.run(0, 20)
+                torch.cuda.synchronize()
+                us_fused = timed_ms(torch, lambda: g.run(0, steps_m)) * 1e3 / steps_m
+                del g
             # isolated single launches of layer 0: steady (rotating ids) and cold (L2 flushed before each)
             out = torch.empty_like(hid)
             reps = 200 if m <= 1024 else 20
@@ -377,14 +390,19 @@ def run_mole(args):
                     ts.append(timed_ms(torch, lambda: mole.layer_forward(hid, bl[r % N_BATCHES], luts[0], wrs[0], out)))
                 iso.append(statistics.median(ts) * 1e3)
             nbytes = sh.layer_bytes(m)
+            fb = sh.step_bytes(m, L)
             sweep.append({
-                "batch": m, "chained_us_per_layer": us_layer, "tokens_per_s_all_layers": m / (us_layer * L * 1e-6),
+                "batch": m,
+                "fused_us_per_step": us_fused, "fused_tokens_per_s_all_layers": (m / (us_fused * 1e-6)) if us_fused else None,
+                "fused_GBps": (fb / us_fused / 1e3) if us_fused else None,
+                "fused_frac_of_peak": (fb / us_fused / 1e3 / peak) if us_fused else None,
+                "chained_us_per_layer": us_layer, "tokens_per_s_all_layers": m / (us_layer * L * 1e-6),
                 "tokens_per_s_per_layer": m / (us_layer * 1e-6), "chained_GBps": nbytes / us_layer / 1e3,
                 "chained_frac_of_peak": nbytes / us_layer / 1e3 / peak,
                 "isolated_steady_us": iso[0], "isolated_cold_us": iso[1],
-                "isolated_cold_GBps": nbytes / iso[1] / 1e3, "plan": mole.plan(m, sh.N, sh.d),
+                "isolated_cold_GBps": nbytes / iso[1] / 1e3,
+                "plan_layer": mole.plan(m, sh.N, sh.d), "plan_fused": mole.plan(m, sh.N, sh.d, mole.DTYPE_BF16, 0, L),
             })
-            del g
         line["sweep"] = sweep
         del flush
 

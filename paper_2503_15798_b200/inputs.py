@@ -50,6 +50,13 @@ class Shape:
         e = self.elem_bytes
         return M * self.N * self.d * e + 2 * M * self.d * e + self.d * self.N * e
 
+    def step_bytes(self, M: int, L: int) -> int:
+        """Algorithmic bytes of L chained layers run as ONE launch: per layer the gathered rows
+        and the router weights, plus hidden in and out once (between layers the hidden state
+        never leaves the chip)."""
+        e = self.elem_bytes
+        return L * (M * self.N * self.d * e + self.d * self.N * e) + 2 * M * self.d * e
+
 
 SHAPES = {
     "tiny": Shape("tiny", V=512, d=64, N=4, L=2, dtype="f32", batches=(64,), D=256),
