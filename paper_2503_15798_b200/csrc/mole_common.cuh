@@ -167,6 +167,45 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
+// Explicit shared-space accesses (32-bit shared addresses): the hot loops index slots of the
+// ring through run-time offsets, and these keep every access on the shared-memory path.
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, const uint4 &v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t a, const uint2 &v)
+{
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+
 // 16-byte vectors of the two storage types
 template <typename T>
 struct Elem;
@@ -201,12 +240,8 @@ struct Elem<__nv_bfloat16> {
     {
         return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p)[i]);
     }
-    // L2-only load: for data another kernel wrote shortly before (never served from a stale L1 line)
-    static __device__ __forceinline__ float scalar_cg(const void *p, long long i)
-    {
-        const uint32_t bits = __ldcg(reinterpret_cast<const unsigned short *>(p) + i);
-        return __uint_as_float(bits << 16);
-    }
+    // element i of an array in shared memory (32-bit shared address)
+    static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds16(base + 2 * i) << 16); }
 };
 template <>
 struct Elem<float> {
@@ -231,10 +266,7 @@ struct Elem<float> {
     {
         return reinterpret_cast<const float *>(p)[i];
     }
-    static __device__ __forceinline__ float scalar_cg(const void *p, long long i)
-    {
-        return __ldcg(reinterpret_cast<const float *>(p) + i);
-    }
+    static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds32(base + 4 * i)); }
 };
 #endif  // __CUDACC__
 

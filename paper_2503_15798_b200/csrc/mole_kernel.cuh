@@ -21,7 +21,7 @@
 // shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp,
 // shared memory over the warps and -- when S > 1 -- st.async into every peer's shared memory
 // over the cluster; every warp then evaluates the softmax redundantly (fp32, expf, true
-// division) and combines the rows it owns in expert order.
+// division) and combines the rows of the column groups it owns.
 #pragma once
 
 #include <math.h>
@@ -47,6 +47,7 @@ struct StepParams {
     long long M, rows;
     int N, d, S, dc, L;
     int stages, slot_bytes, wr_in_ring, consumers;
+    int P;  // lanes that share one 16-byte column group in the combine (1, 2 or 4)
     uint32_t flags;
 };
 
@@ -151,32 +152,46 @@ __device__ __forceinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, 
 // (N < VEC); since the sweep stride is a multiple of 32 vectors, a lane always meets the same
 // experts and keeps only min(VEC, N) accumulators.
 template <typename T, int NFAST>
-__device__ __forceinline__ void router_partial_fast(const unsigned char *wptr, const unsigned char *hptr, int dc,
-                                                    int tid, int lane, int nc, float *partial_warp)
+__device__ __forceinline__ void router_partial_fast(uint32_t waddr, uint32_t haddr, int dc, int tid, int lane, int nc,
+                                                    float *partial_warp)
 {
     using E = Elem<T>;
     constexpr int VEC = E::VEC;
     constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
     constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
     constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
+    constexpr int UNR = 4;                               // vectors in flight per lane
     float acc[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) acc[i] = 0.f;
     const int nvec = dc * NFAST / VEC;
-    const uint4 *wv = reinterpret_cast<const uint4 *>(wptr);
-    for (int u = tid; u < nvec; u += nc) {
-        float wf[VEC];
-        E::unpack(wv[u], wf);
-        if constexpr (NFAST >= VEC) {
-            const float h = E::scalar(hptr, u / QL);
+    for (int u0 = tid; u0 < nvec; u0 += UNR * nc) {
+        uint4 wv[UNR];
+        float hv[UNR][CPV];
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) acc[i] = fmaf(h, wf[i], acc[i]);
-        } else {
+        for (int r = 0; r < UNR; ++r) {  // all loads first, then the arithmetic
+            const int u = u0 + r * nc;
+            const bool ok = u < nvec;
+            const int ui = ok ? u : u0;
+            wv[r] = lds128(waddr + 16u * ui);
 #pragma unroll
             for (int cc = 0; cc < CPV; ++cc) {
-                const float h = E::scalar(hptr, u * CPV + cc);
+                const float h = E::lds_scalar(haddr, NFAST >= VEC ? ui / QL : ui * CPV + cc);
+                hv[r][cc] = ok ? h : 0.f;  // past the end: contributes nothing
+            }
+        }
 #pragma unroll
-                for (int i = 0; i < NFAST; ++i) acc[i] = fmaf(h, wf[cc * NFAST + i], acc[i]);
+        for (int r = 0; r < UNR; ++r) {
+            float wf[VEC];
+            E::unpack(wv[r], wf);
+            if constexpr (NFAST >= VEC) {
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) acc[i] = fmaf(hv[r][0], wf[i], acc[i]);
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < CPV; ++cc)
+#pragma unroll
+                    for (int i = 0; i < NFAST; ++i) acc[i] = fmaf(hv[r][cc], wf[cc * NFAST + i], acc[i]);
             }
         }
     }
@@ -186,6 +201,111 @@ __device__ __forceinline__ void router_partial_fast(const unsigned char *wptr, c
     const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
 #pragma unroll
     for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
+}
+
+// Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over this block's dc columns.
+// A warp covers 32 / P column groups of 16 bytes; the P lanes that share a group (lane bits
+// above log2(32 / P), so that the 8 lanes of a quarter warp read 8 different groups and never
+// collide on a bank) each sum a contiguous chunk of the experts, a shuffle reduce-scatter adds
+// the P partial sums and leaves every lane with VEC / P finished columns, to which it adds the
+// residual, rounds once and stores 16 / P bytes (to global memory, or to the running hidden
+// slice in shared memory when dst_g is null).
+template <typename T, int P>
+__device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint32_t gates, const unsigned char *residual_g,
+                                             unsigned char *dst_g, uint32_t dst_s, int N, int ngrp, bool valid, int warp,
+                                             int lane, int nwarps)
+{
+    using E = Elem<T>;
+    constexpr int VEC = E::VEC;
+    constexpr int GPW = 32 / P;   // column groups per warp
+    constexpr int W = 4 / P;      // 32-bit words a lane finishes
+    constexpr int VPW = VEC / 4;  // values per word: 2 (bf16) or 1 (fp32)
+    constexpr int UNR = 4;        // rows in flight per lane
+    const int part = lane / GPW, gl = lane % GPW;
+    const int chunk = (N + P - 1) / P;
+    const int jb = part * chunk, je = (jb + chunk < N) ? jb + chunk : N;
+    for (int g0 = warp * GPW; g0 < ngrp; g0 += nwarps * GPW) {
+        const int grp = g0 + gl;
+        const bool in = grp < ngrp;
+        const int gg = in ? grp : ngrp - 1;
+        float acc[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+        if (valid) {
+            for (int j0 = jb; j0 < je; j0 += UNR) {
+                uint4 rv[UNR];
+                float gv[UNR];
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) {
+                    const bool ok = j0 + r < je;
+                    const int j = ok ? j0 + r : j0;
+                    rv[r] = lds128(rows + 16u * (j * ngrp + gg));
+                    const float g = __uint_as_float(lds32(gates + 4u * j));
+                    gv[r] = ok ? g : 0.f;
+                }
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) {
+                    float vf[VEC];
+                    E::unpack(rv[r], vf);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
+                }
+            }
+        }
+        int base = 0;
+        if constexpr (P > 1) lane_reduce_scatter<VEC, VEC, 16, GPW>(acc, lane, base);
+        const int word = gg * 4 + base / VPW;  // first 32-bit word of this lane's columns
+        uint32_t rw[W];
+        if (residual_g) {
+            const uint32_t *rsrc = reinterpret_cast<const uint32_t *>(residual_g) + word;
+            if constexpr (W == 4) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(rsrc));
+                rw[0] = v.x, rw[1] = v.y, rw[2] = v.z, rw[3] = v.w;
+            } else if constexpr (W == 2) {
+                const uint2 v = __ldcg(reinterpret_cast<const uint2 *>(rsrc));
+                rw[0] = v.x, rw[1] = v.y;
+            } else {
+                rw[0] = __ldcg(rsrc);
+            }
+        } else {
+            const uint32_t rsrc = haddr + 4u * word;
+            if constexpr (W == 4) {
+                const uint4 v = lds128(rsrc);
+                rw[0] = v.x, rw[1] = v.y, rw[2] = v.z, rw[3] = v.w;
+            } else if constexpr (W == 2) {
+                const uint2 v = lds64(rsrc);
+                rw[0] = v.x, rw[1] = v.y;
+            } else {
+                rw[0] = lds32(rsrc);
+            }
+        }
+        if (valid) {
+#pragma unroll
+            for (int w = 0; w < W; ++w) {
+                if constexpr (VPW == 2) {
+                    const float lo = __uint_as_float(rw[w] << 16) + acc[2 * w];
+                    const float hi = __uint_as_float(rw[w] & 0xffff0000u) + acc[2 * w + 1];
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+                    rw[w] = *reinterpret_cast<const uint32_t *>(&b);
+                } else {
+                    rw[w] = __float_as_uint(__uint_as_float(rw[w]) + acc[w]);
+                }
+            }
+        }
+        if (in) {
+            if (dst_g) {
+                uint32_t *o = reinterpret_cast<uint32_t *>(dst_g) + word;
+                if constexpr (W == 4) *reinterpret_cast<uint4 *>(o) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+                else if constexpr (W == 2) *reinterpret_cast<uint2 *>(o) = make_uint2(rw[0], rw[1]);
+                else *o = rw[0];
+            } else {
+                const uint32_t o = dst_s + 4u * word;
+                if constexpr (W == 4) sts128(o, make_uint4(rw[0], rw[1], rw[2], rw[3]));
+                else if constexpr (W == 2) sts64(o, make_uint2(rw[0], rw[1]));
+                else sts32(o, rw[0]);
+            }
+        }
+    }
 }
 
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
@@ -238,7 +358,8 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         // ================= producer warp: issues every copy, `stages` items ahead =================
         const bool ids64 = (p.flags & MOLE_FLAG_IDS_INT64) != 0;
         long long k = 0, batch = -1, row = -1;
-        int l = 0;
+        int l = 0, pst = 0;       // layer and ring slot of the next item to issue
+        uint32_t pph = 1;         // parity of the `empty` phase that frees that slot (first reuse: phase 0 done)
         if (!p.wr_in_ring && nitems > 0 && lane == 0) {
             mbar_expect_tx(wrbar, m.wr_bytes);
             bulk_g2s(smem + m.off_wr, static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(s) * m.wr_bytes,
@@ -259,7 +380,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 row = __shfl_sync(0xffffffffu, batch, static_cast<int>(k & 31));
             }
             const bool valid = row >= 0 && row < p.rows;
-            const int st = static_cast<int>(it % stages);
+            const int st = pst;
             unsigned char *slot = smem + static_cast<size_t>(st) * m.slot_bytes;
             if (lane == 0) {
                 meta[st] = valid ? 1 : 0;
@@ -294,6 +415,10 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 l = 0;
                 ++k;
             }
+            if (++pst == stages) {
+                pst = 0;
+                pph ^= 1u;
+            }
         };
         // The first `stages` items need no free slot and -- except for hidden, which the previous
         // kernel of a chained launch writes -- nothing upstream: issue them before the grid
@@ -315,8 +440,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         for (long long it = pre; it < nitems; ++it) {
             int ok = 1;
             if (lane == 0) {
-                const int st = static_cast<int>(it % stages);
-                ok = wait_or_give_up(empty + st, static_cast<uint32_t>((it / stages - 1) & 1), dead, kWaitPolls, false);
+                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, false);
                 if (!ok) {
                     if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
                     *dead = 1;
@@ -334,7 +458,6 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [2][nwarps][N]
         float *xchg = reinterpret_cast<float *>(smem + m.off_xchg);        // [2][S][N]
         float *my_gates = reinterpret_cast<float *>(smem + m.off_gates) + warp * N;
-        unsigned char *hid = smem + m.off_hid;  // running hidden slice between layers
         bool alive = true;
 
         auto give_up = [&]() {
@@ -349,14 +472,15 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             if (!__all_sync(0xffffffffu, got)) give_up();
         }
 
-        long long k = 0;
-        int l = 0;
+        const uint32_t smem_base = smem_u32(smem);
+        const uint32_t hid_s = smem_base + m.off_hid;
+        const uint32_t gates_s = smem_u32(my_gates);
+        long long t = c;  // token of the current item
+        int l = 0, st = 0;
+        uint32_t ph = 0;  // ring slot of the current item and the parity of its use
         for (long long it = 0; it < nitems; ++it) {
-            const int st = static_cast<int>(it % stages);
-            const uint32_t ph = static_cast<uint32_t>((it / stages) & 1);
             const int par = static_cast<int>(it & 1);
-            const long long t = c + k * C;
-            unsigned char *slot = smem + static_cast<size_t>(st) * m.slot_bytes;
+            const uint32_t slot_s = smem_base + static_cast<uint32_t>(st) * m.slot_bytes;
             float *part = partial + par * nwarps * N;
             float *xch = xchg + par * S * N;
 
@@ -368,18 +492,18 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls, false);  // let copies in flight land
             }
 
-            const unsigned char *hptr = (l == 0) ? slot + m.slot_hid : hid;
+            const uint32_t haddr = (l == 0) ? slot_s + m.slot_hid : hid_s;
             int nparts = nwarps;
             if (alive) {
-                const unsigned char *wptr = p.wr_in_ring ? slot + m.slot_wr : smem + m.off_wr;
+                const uint32_t waddr = p.wr_in_ring ? slot_s + m.slot_wr : smem_base + m.off_wr;
                 if constexpr (NFAST > 0) {
-                    router_partial_fast<T, NFAST>(wptr, hptr, dc, tid, lane, nc, part + warp * N);
+                    router_partial_fast<T, NFAST>(waddr, haddr, dc, tid, lane, nc, part + warp * N);
                 } else {
                     // any N: one warp per expert, lanes stride over the columns
                     for (int j = warp; j < N; j += nwarps) {
                         float z = 0.f;
                         for (int cc = lane; cc < dc; cc += 32)
-                            z = fmaf(E::scalar(hptr, cc), E::scalar(wptr, static_cast<long long>(cc) * N + j), z);
+                            z = fmaf(E::lds_scalar(haddr, cc), E::lds_scalar(waddr, cc * N + j), z);
                         z = warp_sum(z);
                         if (lane == 0) part[j] = z;
                     }
@@ -437,34 +561,17 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             }
 
             if (alive) {
-                // weighted sum over the experts in expert order, residual add, one rounding (Eq. 8)
                 const bool valid = meta[st] != 0;
-                const uint4 *rows_vec = reinterpret_cast<const uint4 *>(slot);
-                const uint4 *h_vec = reinterpret_cast<const uint4 *>(hptr);
-                const size_t gvec = static_cast<size_t>(t) * (d / VEC) + static_cast<size_t>(s) * ngrp;
-                for (int grp = tid; grp < ngrp; grp += nc) {
-                    uint4 res = p.residual ? __ldcg(reinterpret_cast<const uint4 *>(p.residual) + gvec + grp) : h_vec[grp];
-                    if (valid) {
-                        float acc[VEC];
-#pragma unroll
-                        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
-#pragma unroll 4
-                        for (int j = 0; j < N; ++j) {
-                            float vf[VEC];
-                            E::unpack(rows_vec[j * ngrp + grp], vf);
-                            const float g = my_gates[j];
-#pragma unroll
-                            for (int i = 0; i < VEC; ++i) acc[i] = fmaf(g, vf[i], acc[i]);
-                        }
-                        float rf[VEC];
-                        E::unpack(res, rf);
-#pragma unroll
-                        for (int i = 0; i < VEC; ++i) acc[i] = rf[i] + acc[i];
-                        res = E::pack(acc);
-                    }
-                    if (l == L - 1) reinterpret_cast<uint4 *>(p.out)[gvec + grp] = res;
-                    else reinterpret_cast<uint4 *>(hid)[grp] = res;
-                }
+                const size_t gbyte = (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB;
+                const unsigned char *res_g =
+                    p.residual ? static_cast<const unsigned char *>(p.residual) + gbyte : nullptr;
+                unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + gbyte : nullptr;
+                if (p.P == 4)
+                    combine_item<T, 4>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
+                else if (p.P == 2)
+                    combine_item<T, 2>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
+                else
+                    combine_item<T, 1>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty + st);  // this warp is done with the slot
@@ -472,7 +579,11 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             if (L > 1) named_bar_sync(kConsumerBarrier, nc);
             if (++l == L) {
                 l = 0;
-                ++k;
+                t += C;
+            }
+            if (++st == stages) {
+                st = 0;
+                ph ^= 1u;
             }
         }
     }

@@ -2,6 +2,7 @@
 // for a single layer and for a chained L-layer decode step (Eq. 4 and Eq. 8 of arXiv
 // 2503.15798).  The kernel itself is in mole_kernel.cuh.
 #include <atomic>
+#include <stdlib.h>
 #include <string.h>
 
 #include "mole_kernel.cuh"
@@ -25,10 +26,17 @@ constexpr int kSmemPerBlockMax = 227 * 1024;  // opt-in limit per block
 constexpr int kSmemPerSM = 228 * 1024;        // per SM, of which every resident block reserves 1 KB
 constexpr long long kFusedMaxTokens = 4096;   // above this a step runs as L chained launches
 
-static int consumers_for(int dc, int vec)
+// Lanes per 16-byte column group in the combine: as many (up to 4) as keep the block within
+// kMaxConsumers threads.
+static int lanes_per_group(int dc, int vec)
 {
     const int groups = dc / vec;
-    return round_up(groups < kMaxConsumers ? groups : kMaxConsumers, 32);
+    return groups * 4 <= kMaxConsumers ? 4 : (groups * 2 <= kMaxConsumers ? 2 : 1);
+}
+static int consumers_for(int dc, int vec)
+{
+    const int lanes = (dc / vec) * lanes_per_group(dc, vec);
+    return round_up(lanes < kMaxConsumers ? lanes : kMaxConsumers, 32);
 }
 
 int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan)
@@ -86,6 +94,10 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     const long long items = blocks > 0 ? ((M * S + blocks - 1) / blocks) * L : 1;
     if (stages > items) stages = items < 2 ? 2 : static_cast<int>(items);
     while (stages > 2 && !fits(S, stages)) --stages;
+    if (const char *f = getenv("MOLE_FORCE_STAGES")) {  // debugging aid: ring depth, if it fits
+        const int v = atoi(f);
+        if (v >= 2 && v <= kMaxStages && fits(S, v)) stages = v;
+    }
     const SmemMap m = smem_map(N, dc, eb, S, stages, in_ring, consumers);
     plan->d_split = S;
     plan->dc = dc;
@@ -184,8 +196,18 @@ int launch_step(const StepLaunch &a)
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
+    StepKernel k = pick_kernel(a.dtype, plan.n_fast);
+    rc = ensure_smem(k, plan.smem);
+    if (rc != MOLE_OK) return rc;
     // a persistent grid: as many blocks as fit at once (whole clusters), never more than the work
-    long long grid = static_cast<long long>(plan.blocks_per_sm) * sms / plan.d_split * plan.d_split;
+    int per_sm = 0;
+    MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, plan.threads, plan.smem));
+    if (per_sm < 1) per_sm = 1;
+    if (const char *f = getenv("MOLE_FORCE_BLOCKS_PER_SM")) {  // debugging aid
+        const int v = atoi(f);
+        if (v >= 1 && v < per_sm) per_sm = v;
+    }
+    long long grid = static_cast<long long>(per_sm) * sms / plan.d_split * plan.d_split;
     if (grid < plan.d_split) grid = plan.d_split;
     if (grid > a.M * plan.d_split) grid = a.M * plan.d_split;
 
@@ -211,11 +233,8 @@ int launch_step(const StepLaunch &a)
     p.slot_bytes = plan.slot_bytes;
     p.wr_in_ring = plan.wr_in_ring;
     p.consumers = plan.consumers;
+    p.P = lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype));
     p.flags = a.flags;
-
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast);
-    rc = ensure_smem(k, plan.smem);
-    if (rc != MOLE_OK) return rc;
 
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
