@@ -47,7 +47,6 @@ struct StepParams {
     long long M, rows;
     int N, d, S, dc, L;
     int stages, slot_bytes, wr_in_ring, consumers;
-    int P;  // lanes that share one 16-byte column group in the combine (1, 2 or 4)
     uint32_t flags;
 };
 
@@ -203,7 +202,10 @@ __device__ __forceinline__ void router_partial_fast(uint32_t waddr, uint32_t had
     for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
 }
 
-// Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over this block's dc columns.
+// Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over this block's dc columns,
+// with g_j = e_j / sum_k e_k given as the un-normalised e_j: the lanes add up the e_j of their
+// experts next to the rows, so the normalisation costs no reduction of its own -- one reciprocal
+// and one multiply per column at the end.
 // A warp covers 32 / P column groups of 16 bytes; the P lanes that share a group (lane bits
 // above log2(32 / P), so that the 8 lanes of a quarter warp read 8 different groups and never
 // collide on a bank) each sum a contiguous chunk of the experts, a shuffle reduce-scatter adds
@@ -229,6 +231,7 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
         const bool in = grp < ngrp;
         const int gg = in ? grp : ngrp - 1;
         float acc[VEC];
+        float esum = 0.f;
 #pragma unroll
         for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
         if (valid) {
@@ -247,13 +250,19 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
                 for (int r = 0; r < UNR; ++r) {
                     float vf[VEC];
                     E::unpack(rv[r], vf);
+                    esum += gv[r];
 #pragma unroll
                     for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
                 }
             }
         }
         int base = 0;
-        if constexpr (P > 1) lane_reduce_scatter<VEC, VEC, 16, GPW>(acc, lane, base);
+        if constexpr (P > 1) {
+            lane_reduce_scatter<VEC, VEC, 16, GPW>(acc, lane, base);
+#pragma unroll
+            for (int o = 16; o >= GPW; o >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, o);
+        }
+        const float inv = __frcp_rn(esum);
         const int word = gg * 4 + base / VPW;  // first 32-bit word of this lane's columns
         uint32_t rw[W];
         if (residual_g) {
@@ -283,12 +292,12 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
 #pragma unroll
             for (int w = 0; w < W; ++w) {
                 if constexpr (VPW == 2) {
-                    const float lo = __uint_as_float(rw[w] << 16) + acc[2 * w];
-                    const float hi = __uint_as_float(rw[w] & 0xffff0000u) + acc[2 * w + 1];
+                    const float lo = fmaf(acc[2 * w], inv, __uint_as_float(rw[w] << 16));
+                    const float hi = fmaf(acc[2 * w + 1], inv, __uint_as_float(rw[w] & 0xffff0000u));
                     const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
                     rw[w] = *reinterpret_cast<const uint32_t *>(&b);
                 } else {
-                    rw[w] = __float_as_uint(__uint_as_float(rw[w]) + acc[w]);
+                    rw[w] = __float_as_uint(fmaf(acc[w], inv, __uint_as_float(rw[w])));
                 }
             }
         }
@@ -309,7 +318,8 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
 }
 
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
-template <typename T, int NFAST>
+// P: lanes that share one 16-byte column group in the combine.
+template <typename T, int NFAST, int P>
 __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const StepParams p)
 {
     using E = Elem<T>;
@@ -539,21 +549,28 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 } else {
                     if (j0 < N) {
                         z0 = 0.f;
+#pragma unroll 8
                         for (int w = 0; w < nparts; ++w) z0 += part[w * N + j0];
                     }
                     if (j1 < N) {
                         z1 = 0.f;
+#pragma unroll 8
                         for (int w = 0; w < nparts; ++w) z1 += part[w * N + j1];
                     }
                 }
-                // softmax over all N experts (Eq. 4), every warp its own copy
-                const float zmax = warp_max(fmaxf(z0, z1));
+                // softmax over all N experts (Eq. 4), every warp its own copy.  Only the numerators
+                // e_j = exp(z_j - m) are formed here; the combine divides by their sum.  Any shift
+                // m gives the same gates, so the (shuffle-heavy) maximum is taken only when some
+                // logit is large enough for exp to leave the comfortable range.
+                const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
+                float zmax = 0.f;
+                if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(z0, z1));
                 const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
                 const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
-                const float esum = warp_sum(e0 + e1);
-                if (j0 < N) my_gates[j0] = e0 / esum;
-                if (j1 < N) my_gates[j1] = e1 / esum;
+                if (j0 < N) my_gates[j0] = e0;
+                if (j1 < N) my_gates[j1] = e1;
                 if (p.gates_out && s == 0 && warp == 0) {
+                    const float esum = warp_sum(e0 + e1);
                     if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
                     if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
                 }
@@ -566,12 +583,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 const unsigned char *res_g =
                     p.residual ? static_cast<const unsigned char *>(p.residual) + gbyte : nullptr;
                 unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + gbyte : nullptr;
-                if (p.P == 4)
-                    combine_item<T, 4>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
-                else if (p.P == 2)
-                    combine_item<T, 2>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
-                else
-                    combine_item<T, 1>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
+                combine_item<T, P>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty + st);  // this warp is done with the slot

@@ -118,22 +118,28 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
 
 typedef void (*StepKernel)(const StepParams);
 
-template <typename T>
+template <typename T, int P>
 static StepKernel pick_n(int n_fast)
 {
     switch (n_fast) {
-        case 4: return mole_step_kernel<T, 4>;
-        case 8: return mole_step_kernel<T, 8>;
-        case 16: return mole_step_kernel<T, 16>;
-        case 32: return mole_step_kernel<T, 32>;
-        case 64: return mole_step_kernel<T, 64>;
-        default: return mole_step_kernel<T, 0>;
+        case 4: return mole_step_kernel<T, 4, P>;
+        case 8: return mole_step_kernel<T, 8, P>;
+        case 16: return mole_step_kernel<T, 16, P>;
+        case 32: return mole_step_kernel<T, 32, P>;
+        case 64: return mole_step_kernel<T, 64, P>;
+        default: return mole_step_kernel<T, 0, P>;
     }
 }
 
-static StepKernel pick_kernel(int dtype, int n_fast)
+template <typename T>
+static StepKernel pick_p(int n_fast, int lanes)
 {
-    return dtype == MOLE_DTYPE_BF16 ? pick_n<__nv_bfloat16>(n_fast) : pick_n<float>(n_fast);
+    return lanes == 4 ? pick_n<T, 4>(n_fast) : (lanes == 2 ? pick_n<T, 2>(n_fast) : pick_n<T, 1>(n_fast));
+}
+
+static StepKernel pick_kernel(int dtype, int n_fast, int lanes)
+{
+    return dtype == MOLE_DTYPE_BF16 ? pick_p<__nv_bfloat16>(n_fast, lanes) : pick_p<float>(n_fast, lanes);
 }
 
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
@@ -196,7 +202,7 @@ int launch_step(const StepLaunch &a)
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast);
+    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)));
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
     // a persistent grid: as many blocks as fit at once (whole clusters), never more than the work
@@ -233,7 +239,6 @@ int launch_step(const StepLaunch &a)
     p.slot_bytes = plan.slot_bytes;
     p.wr_in_ring = plan.wr_in_ring;
     p.consumers = plan.consumers;
-    p.P = lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype));
     p.flags = a.flags;
 
     cudaLaunchConfig_t cfg;
