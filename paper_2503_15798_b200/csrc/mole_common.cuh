@@ -206,6 +206,35 @@ __device__ __forceinline__ void sts32(uint32_t a, uint32_t v)
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
 }
 
+// Two fp32 values in one 64-bit register and the packed fused multiply-add of sm_100
+// (two independent IEEE fmas per instruction: same results as two scalar fmaf).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
+    return r;
+}
+__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // 16-byte vectors of the two storage types
 template <typename T>
 struct Elem;
@@ -222,6 +251,14 @@ struct Elem<__nv_bfloat16> {
         f[5] = __uint_as_float(v.z & 0xffff0000u);
         f[6] = __uint_as_float(v.w << 16);
         f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    // the 8 values as 4 fp32 pairs (columns 0-1, 2-3, 4-5, 6-7)
+    static __device__ __forceinline__ void unpack_pairs(const uint4 &v, f32x2 (&p)[4])
+    {
+        p[0] = pack2u(v.x << 16, v.x & 0xffff0000u);
+        p[1] = pack2u(v.y << 16, v.y & 0xffff0000u);
+        p[2] = pack2u(v.z << 16, v.z & 0xffff0000u);
+        p[3] = pack2u(v.w << 16, v.w & 0xffff0000u);
     }
     static __device__ __forceinline__ uint4 pack(const float (&f)[8])
     {
@@ -252,6 +289,11 @@ struct Elem<float> {
         f[1] = __uint_as_float(v.y);
         f[2] = __uint_as_float(v.z);
         f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ void unpack_pairs(const uint4 &v, f32x2 (&p)[2])
+    {
+        p[0] = pack2u(v.x, v.y);
+        p[1] = pack2u(v.z, v.w);
     }
     static __device__ __forceinline__ uint4 pack(const float (&f)[4])
     {

@@ -131,9 +131,10 @@ __device__ __forceinline__ float warp_sum(float v)
 
 // Bounded wait shared by producer and consumers.  `dead` (shared memory) is raised by whoever
 // gives up first; everyone else then stops waiting at once.
-__device__ __forceinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
+__device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
                                                 bool cluster_scope)
 {
+#pragma unroll 1
     for (uint32_t i = 0; i < polls; ++i) {
         if (cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if (i > 64) {
@@ -159,47 +160,56 @@ __device__ __forceinline__ void router_partial_fast(uint32_t waddr, uint32_t had
     constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
     constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
     constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
+    constexpr int PPC = NV / 2;                          // fp32 pairs per column of a vector
     constexpr int UNR = 4;                               // vectors in flight per lane
-    float acc[NV];
+    f32x2 acc[NV / 2];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+    for (int i = 0; i < NV / 2; ++i) acc[i] = 0ull;
     const int nvec = dc * NFAST / VEC;
-    for (int u0 = tid; u0 < nvec; u0 += UNR * nc) {
+    // One vector: its VEC values, as fp32 pairs, times the hidden value(s) of its column(s).
+    auto mac = [&](const uint4 &w, const float (&h)[CPV]) {
+        f32x2 wp[VEC / 2];
+        E::unpack_pairs(w, wp);
+#pragma unroll
+        for (int cc = 0; cc < CPV; ++cc) {
+            const f32x2 hh = pack2(h[cc], h[cc]);
+#pragma unroll
+            for (int i = 0; i < PPC; ++i) acc[i] = fma2(hh, wp[cc * PPC + i], acc[i]);
+        }
+    };
+    auto hidden_of = [&](int u, float (&h)[CPV]) {
+#pragma unroll
+        for (int cc = 0; cc < CPV; ++cc) h[cc] = E::lds_scalar(haddr, NFAST >= VEC ? u / QL : u * CPV + cc);
+    };
+    int u0 = tid;
+#pragma unroll 1
+    for (; u0 + (UNR - 1) * nc < nvec; u0 += UNR * nc) {  // full batches: all loads first, then the arithmetic
         uint4 wv[UNR];
         float hv[UNR][CPV];
 #pragma unroll
-        for (int r = 0; r < UNR; ++r) {  // all loads first, then the arithmetic
-            const int u = u0 + r * nc;
-            const bool ok = u < nvec;
-            const int ui = ok ? u : u0;
-            wv[r] = lds128(waddr + 16u * ui);
-#pragma unroll
-            for (int cc = 0; cc < CPV; ++cc) {
-                const float h = E::lds_scalar(haddr, NFAST >= VEC ? ui / QL : ui * CPV + cc);
-                hv[r][cc] = ok ? h : 0.f;  // past the end: contributes nothing
-            }
-        }
-#pragma unroll
         for (int r = 0; r < UNR; ++r) {
-            float wf[VEC];
-            E::unpack(wv[r], wf);
-            if constexpr (NFAST >= VEC) {
-#pragma unroll
-                for (int i = 0; i < VEC; ++i) acc[i] = fmaf(hv[r][0], wf[i], acc[i]);
-            } else {
-#pragma unroll
-                for (int cc = 0; cc < CPV; ++cc)
-#pragma unroll
-                    for (int i = 0; i < NFAST; ++i) acc[i] = fmaf(hv[r][cc], wf[cc * NFAST + i], acc[i]);
-            }
+            wv[r] = lds128(waddr + 16u * (u0 + r * nc));
+            hidden_of(u0 + r * nc, hv[r]);
         }
+#pragma unroll
+        for (int r = 0; r < UNR; ++r) mac(wv[r], hv[r]);
     }
+#pragma unroll 1
+    for (; u0 < nvec; u0 += nc) {  // tail
+        float h[CPV];
+        const uint4 w = lds128(waddr + 16u * u0);
+        hidden_of(u0, h);
+        mac(w, h);
+    }
+    float a[NV];
+#pragma unroll
+    for (int i = 0; i < NV / 2; ++i) unpack2(acc[i], a[2 * i], a[2 * i + 1]);
     int base = 0;
-    lane_reduce_scatter<NV, NV, 16, QL>(acc, lane, base);
+    lane_reduce_scatter<NV, NV, 16, QL>(a, lane, base);
     constexpr int left = ReduceScatterLeft<NV, 16, QL>::value;
     const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
 #pragma unroll
-    for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
+    for (int i = 0; i < left; ++i) partial_warp[first + i] = a[i];
 }
 
 // Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over this block's dc columns,
@@ -226,36 +236,51 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     const int part = lane / GPW, gl = lane % GPW;
     const int chunk = (N + P - 1) / P;
     const int jb = part * chunk, je = (jb + chunk < N) ? jb + chunk : N;
+#pragma unroll 1
     for (int g0 = warp * GPW; g0 < ngrp; g0 += nwarps * GPW) {
         const int grp = g0 + gl;
         const bool in = grp < ngrp;
         const int gg = in ? grp : ngrp - 1;
-        float acc[VEC];
+        f32x2 accp[VEC / 2];
         float esum = 0.f;
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+        for (int i = 0; i < VEC / 2; ++i) accp[i] = 0ull;
         if (valid) {
-            for (int j0 = jb; j0 < je; j0 += UNR) {
+            int j0 = jb;
+#pragma unroll 1
+            for (; j0 + UNR <= je; j0 += UNR) {  // full batches: all loads first
                 uint4 rv[UNR];
                 float gv[UNR];
 #pragma unroll
                 for (int r = 0; r < UNR; ++r) {
-                    const bool ok = j0 + r < je;
-                    const int j = ok ? j0 + r : j0;
-                    rv[r] = lds128(rows + 16u * (j * ngrp + gg));
-                    const float g = __uint_as_float(lds32(gates + 4u * j));
-                    gv[r] = ok ? g : 0.f;
+                    rv[r] = lds128(rows + 16u * ((j0 + r) * ngrp + gg));
+                    gv[r] = __uint_as_float(lds32(gates + 4u * (j0 + r)));
                 }
 #pragma unroll
                 for (int r = 0; r < UNR; ++r) {
-                    float vf[VEC];
-                    E::unpack(rv[r], vf);
+                    f32x2 vp[VEC / 2];
+                    E::unpack_pairs(rv[r], vp);
+                    const f32x2 g2 = pack2(gv[r], gv[r]);
                     esum += gv[r];
 #pragma unroll
-                    for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
+                    for (int i = 0; i < VEC / 2; ++i) accp[i] = fma2(g2, vp[i], accp[i]);
                 }
             }
+#pragma unroll 1
+            for (; j0 < je; ++j0) {  // tail
+                const uint4 rv = lds128(rows + 16u * (j0 * ngrp + gg));
+                const float g = __uint_as_float(lds32(gates + 4u * j0));
+                f32x2 vp[VEC / 2];
+                E::unpack_pairs(rv, vp);
+                const f32x2 g2 = pack2(g, g);
+                esum += g;
+#pragma unroll
+                for (int i = 0; i < VEC / 2; ++i) accp[i] = fma2(g2, vp[i], accp[i]);
+            }
         }
+        float acc[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC / 2; ++i) unpack2(accp[i], acc[2 * i], acc[2 * i + 1]);
         int base = 0;
         if constexpr (P > 1) {
             lane_reduce_scatter<VEC, VEC, 16, GPW>(acc, lane, base);
@@ -488,6 +513,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         long long t = c;  // token of the current item
         int l = 0, st = 0;
         uint32_t ph = 0;  // ring slot of the current item and the parity of its use
+#pragma unroll 1
         for (long long it = 0; it < nitems; ++it) {
             const int par = static_cast<int>(it & 1);
             const uint32_t slot_s = smem_base + static_cast<uint32_t>(st) * m.slot_bytes;
