@@ -20,8 +20,8 @@
 // Arithmetic per item (consumer warps): a conflict-free linear sweep over the router slice in
 // shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp,
 // shared memory over the warps and -- when S > 1 -- st.async into every peer's shared memory
-// over the cluster; every warp then evaluates the softmax redundantly (fp32, expf, true
-// division) and combines the rows of the column groups it owns.
+// over the cluster; warp 0 evaluates the softmax numerators (fp32, expf) for the block, and every
+// warp combines the rows of the column groups it owns, dividing by the sum of the numerators.
 #pragma once
 
 #include <math.h>
@@ -34,7 +34,9 @@ constexpr int kMaxN = 64;            // experts
 constexpr int kMaxSplit = 8;         // blocks per token
 constexpr int kMaxConsumers = 256;   // compute threads per block
 constexpr int kMaxStages = 8;        // ring depth
-constexpr int kConsumerBarrier = 1;  // named barrier of the consumer warps
+constexpr int kBarLogits = 1;  // named barriers of the consumer warps: partial logits written,
+constexpr int kBarGates = 2;   // softmax numerators written,
+constexpr int kBarHidden = 3;  // running hidden slice written
 constexpr uint32_t kWaitPolls = 1u << 24;   // >= 1 s of polling before a wait gives up
 constexpr uint32_t kDrainPolls = 1u << 14;  // after a failure: short waits for copies still in flight
 
@@ -73,7 +75,7 @@ __host__ __device__ inline SmemMap smem_map(int N, int dc, int eb, int S, int st
     m.off_partial = m.off_hid + up128(m.hid_bytes);
     m.off_xchg = m.off_partial + up128(2u * warps * N * 4);
     m.off_gates = m.off_xchg + up128(2u * S * N * 4);
-    m.off_meta = m.off_gates + up128(warps * N * 4);
+    m.off_meta = m.off_gates + up128(N * 4);
     m.off_bars = m.off_meta + up128((kMaxStages + 3) * 4);
     m.total = m.off_bars + (2 * kMaxStages + 3) * 8;
     return m;
@@ -131,13 +133,15 @@ __device__ __forceinline__ float warp_sum(float v)
 
 // Bounded wait shared by producer and consumers.  `dead` (shared memory) is raised by whoever
 // gives up first; everyone else then stops waiting at once.
+// `patient`: sleep after every failed poll (the producer, which runs several items ahead and
+// must not take issue slots from the warps that compute).
 __device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
-                                                bool cluster_scope)
+                                             bool cluster_scope, bool patient = false)
 {
 #pragma unroll 1
     for (uint32_t i = 0; i < polls; ++i) {
         if (cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-        if (i > 64) {
+        if (patient || i > 64) {
             __nanosleep(64);
             if ((i & 127u) == 0 && *dead) return false;
         }
@@ -475,7 +479,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         for (long long it = pre; it < nitems; ++it) {
             int ok = 1;
             if (lane == 0) {
-                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, false);
+                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, false, true);
                 if (!ok) {
                     if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
                     *dead = 1;
@@ -492,7 +496,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         const int ngrp = dc / VEC;  // 16-byte column groups of this block's slice
         float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [2][nwarps][N]
         float *xchg = reinterpret_cast<float *>(smem + m.off_xchg);        // [2][S][N]
-        float *my_gates = reinterpret_cast<float *>(smem + m.off_gates) + warp * N;
+        float *gates = reinterpret_cast<float *>(smem + m.off_gates);  // [N] softmax numerators of the current item
         bool alive = true;
 
         auto give_up = [&]() {
@@ -509,7 +513,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
 
         const uint32_t smem_base = smem_u32(smem);
         const uint32_t hid_s = smem_base + m.off_hid;
-        const uint32_t gates_s = smem_u32(my_gates);
+        const uint32_t gates_s = smem_u32(gates);
         long long t = c;  // token of the current item
         int l = 0, st = 0;
         uint32_t ph = 0;  // ring slot of the current item and the parity of its use
@@ -521,7 +525,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             float *xch = xchg + par * S * N;
 
             if (alive) {
-                if (S > 1 && tid == 0) mbar_expect_tx(xbar + par, static_cast<uint32_t>(S) * N * 4u);
+                if (S > 1 && tid == 0) mbar_expect_tx(xbar + par, static_cast<uint32_t>(S) * N * 4u);  // tid 0 is in warp 0
                 const bool got = wait_or_give_up(full + st, ph, dead, kWaitPolls, false);
                 if (!__all_sync(0xffffffffu, got)) give_up();
             } else if (it < *issued) {
@@ -546,62 +550,58 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                     nparts = 1;
                 }
             }
-            named_bar_sync(kConsumerBarrier, nc);
-
-            if (alive) {
-                const int j0 = lane, j1 = lane + 32;
-                float z0 = -INFINITY, z1 = -INFINITY;
-                if (S > 1) {
-                    // block totals go to every block of the cluster (this one included), then the
-                    // S partial logits are summed in slice order by everybody
-                    if (warp == 0) {
-                        const uint32_t dst = smem_u32(xch + s * N), bar = smem_u32(xbar + par);
-                        for (int j = lane; j < N; j += 32) {
-                            float zc = 0.f;
-                            for (int w = 0; w < nparts; ++w) zc += part[w * N + j];
-                            for (int q = 0; q < S; ++q) st_async_f32(map_to_cta(dst + j * 4, q), zc, map_to_cta(bar, q));
-                        }
-                    }
-                    const bool got = wait_or_give_up(xbar + par, static_cast<uint32_t>((it >> 1) & 1), dead, kWaitPolls, true);
-                    if (!__all_sync(0xffffffffu, got)) give_up();
+            // warp 0 turns the partial logits into softmax numerators for everybody
+            if (warp != 0) {
+                named_bar_arrive(kBarLogits, nc);
+            } else {
+                named_bar_sync(kBarLogits, nc);
+                if (alive) {
+                    const int j0 = lane, j1 = lane + 32;
+                    float z0 = 0.f, z1 = 0.f;
                     if (j0 < N) {
-                        z0 = 0.f;
-                        for (int q = 0; q < S; ++q) z0 += xch[q * N + j0];
-                    }
-                    if (j1 < N) {
-                        z1 = 0.f;
-                        for (int q = 0; q < S; ++q) z1 += xch[q * N + j1];
-                    }
-                } else {
-                    if (j0 < N) {
-                        z0 = 0.f;
 #pragma unroll 8
                         for (int w = 0; w < nparts; ++w) z0 += part[w * N + j0];
                     }
                     if (j1 < N) {
-                        z1 = 0.f;
 #pragma unroll 8
                         for (int w = 0; w < nparts; ++w) z1 += part[w * N + j1];
                     }
+                    if (S > 1) {
+                        // block totals go to every block of the cluster (this one included), then
+                        // the S partial logits are summed in slice order by everybody
+                        const uint32_t dst = smem_u32(xch + s * N), bar = smem_u32(xbar + par);
+                        for (int q = 0; q < S; ++q) {
+                            if (j0 < N) st_async_f32(map_to_cta(dst + j0 * 4, q), z0, map_to_cta(bar, q));
+                            if (j1 < N) st_async_f32(map_to_cta(dst + j1 * 4, q), z1, map_to_cta(bar, q));
+                        }
+                        const bool got =
+                            wait_or_give_up(xbar + par, static_cast<uint32_t>((it >> 1) & 1), dead, kWaitPolls, true);
+                        if (!__all_sync(0xffffffffu, got)) give_up();
+                        z0 = 0.f, z1 = 0.f;
+                        if (j0 < N)
+                            for (int q = 0; q < S; ++q) z0 += xch[q * N + j0];
+                        if (j1 < N)
+                            for (int q = 0; q < S; ++q) z1 += xch[q * N + j1];
+                    }
+                    // softmax over all N experts (Eq. 4).  Only the numerators e_j = exp(z_j - m)
+                    // are formed here; the combine divides by their sum.  Any shift m gives the same
+                    // gates, so the (shuffle-heavy) maximum is taken only when some logit is large
+                    // enough for exp to leave the comfortable range.
+                    const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
+                    float zmax = 0.f;
+                    if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(j0 < N ? z0 : -INFINITY, j1 < N ? z1 : -INFINITY));
+                    const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
+                    const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
+                    if (j0 < N) gates[j0] = e0;
+                    if (j1 < N) gates[j1] = e1;
+                    if (p.gates_out && s == 0) {
+                        const float esum = warp_sum(e0 + e1);
+                        if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
+                        if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
+                    }
                 }
-                // softmax over all N experts (Eq. 4), every warp its own copy.  Only the numerators
-                // e_j = exp(z_j - m) are formed here; the combine divides by their sum.  Any shift
-                // m gives the same gates, so the (shuffle-heavy) maximum is taken only when some
-                // logit is large enough for exp to leave the comfortable range.
-                const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
-                float zmax = 0.f;
-                if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(z0, z1));
-                const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
-                const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
-                if (j0 < N) my_gates[j0] = e0;
-                if (j1 < N) my_gates[j1] = e1;
-                if (p.gates_out && s == 0 && warp == 0) {
-                    const float esum = warp_sum(e0 + e1);
-                    if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
-                    if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
-                }
-                __syncwarp();
             }
+            named_bar_sync(kBarGates, nc);
 
             if (alive) {
                 const bool valid = meta[st] != 0;
@@ -614,7 +614,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             __syncwarp();
             if (lane == 0) mbar_arrive(empty + st);  // this warp is done with the slot
             // the next layer's router reads the hidden slice that all warps have just written
-            if (L > 1) named_bar_sync(kConsumerBarrier, nc);
+            if (L > 1) named_bar_sync(kBarHidden, nc);
             if (++l == L) {
                 l = 0;
                 t += C;
