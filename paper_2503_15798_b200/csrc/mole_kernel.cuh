@@ -2,26 +2,28 @@
 // softmax over all N experts, gather of the token's N table rows, fp32 weighted sum, residual
 // add -- for one layer or for L chained layers in one launch.
 //
-// Work decomposition.  A block owns one slice of dc = d / S columns (S blocks of a token form
-// a thread-block cluster when S > 1).  It walks over its tokens t = c, c + C, c + 2C, ... and,
-// per token, over the layers l = 0 .. L-1; one (token, layer) pair is an "item".  The chain
-// h_{l+1} = h_l + sum_j g_j(h_l) LUT_l[id][j] of a token never leaves the block: the running
-// hidden slice stays in shared memory, rounded to the storage type after every layer exactly as
-// a layer-by-layer execution would round it.
+// Work decomposition.  A block owns whole tokens: it walks over its tokens t = b, b + G, b + 2G,
+// ... (G blocks in the grid) and, per token, over the layers l = 0 .. L-1; one (token, layer)
+// pair is an "item".  The chain h_{l+1} = h_l + sum_j g_j(h_l) LUT_l[id][j] of a token never
+// leaves the block: the running hidden state stays in shared memory, rounded to the storage
+// type after every layer exactly as a layer-by-layer execution would round it.  There is no
+// communication between blocks.
 //
-// Data movement.  Everything an item needs is pulled into a ring of shared-memory slots by bulk
+// Data movement.  An item is cut into K column chunks of dcc = d / K columns.  Everything it
+// needs is pulled through a ring of shared-memory slots, one chunk per slot, by bulk
 // asynchronous copies (TMA engine, untiled, no multicast) that one extra "producer" warp issues
-// `stages` items ahead: the N row pieces (they depend only on the id, so they run ahead of the
-// arithmetic and, in a chained launch, ahead of the previous kernel), the router slice of the
-// layer when L > 1, and the token's hidden slice for its first layer.  Completion is counted on
-// one mbarrier per slot ("full"); the consumer warps hand a slot back through a second one
-// ("empty").
+// `stages` chunks ahead: first (when L > 1) the K chunks [dcc][N] of the layer's router matrix,
+// then the K chunks [N][dcc] of the token's table rows.  The rows depend only on the id, so they
+// run ahead of the arithmetic and, in a chained launch, ahead of the previous kernel.  The
+// token's hidden state arrives with its first chunk in a small ring of its own.  Completion is
+// counted on one mbarrier per slot ("full"); the consumer warps hand a slot back through a
+// second one ("empty").  With L == 1 the router matrix is loaded once per block instead.
 //
-// Arithmetic per item (consumer warps): a conflict-free linear sweep over the router slice in
-// shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp,
-// shared memory over the warps and -- when S > 1 -- st.async into every peer's shared memory
-// over the cluster; warp 0 evaluates the softmax numerators (fp32, expf) for the block, and every
-// warp combines the rows of the column groups it owns, dividing by the sum of the numerators.
+// Arithmetic per item (consumer warps): a conflict-free linear sweep over the router chunks in
+// shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp
+// and shared memory over the warps; warp 0 evaluates the softmax numerators (fp32, expf) for
+// the block, and every warp combines the row chunks of the column groups it owns, dividing by
+// the sum of the numerators.
 #pragma once
 
 #include <math.h>
@@ -30,13 +32,13 @@
 
 namespace mole {
 
-constexpr int kMaxN = 64;            // experts
-constexpr int kMaxSplit = 8;         // blocks per token
-constexpr int kMaxConsumers = 256;   // compute threads per block
-constexpr int kMaxStages = 8;        // ring depth
-constexpr int kBarLogits = 1;  // named barriers of the consumer warps: partial logits written,
-constexpr int kBarGates = 2;   // softmax numerators written,
-constexpr int kBarHidden = 3;  // running hidden slice written
+constexpr int kMaxN = 64;           // experts
+constexpr int kMaxChunks = 16;      // column chunks per token
+constexpr int kMaxConsumers = 256;  // compute threads per block
+constexpr int kMaxStages = 8;       // ring depth
+constexpr int kBarLogits = 1;       // named barriers of the consumer warps: partial logits written,
+constexpr int kBarGates = 2;        // softmax numerators written,
+constexpr int kBarHidden = 3;       // running hidden state written
 constexpr uint32_t kWaitPolls = 1u << 24;   // >= 1 s of polling before a wait gives up
 constexpr uint32_t kDrainPolls = 1u << 14;  // after a failure: short waits for copies still in flight
 
@@ -47,37 +49,33 @@ struct StepParams {
     uint32_t *status;
     long long lut_stride, wr_stride;  // bytes between layers
     long long M, rows;
-    int N, d, S, dc, L;
-    int stages, slot_bytes, wr_in_ring, consumers;
+    int N, d, K, dcc, L;
+    int stages, hring, wr_in_ring, consumers;
     uint32_t flags;
 };
 
 // Shared-memory map, computed the same way on the host (for the size) and in the kernel.
 struct SmemMap {
-    uint32_t rows_bytes, wr_bytes, hid_bytes;  // per item: row pieces, router slice, hidden slice
-    uint32_t slot_wr, slot_hid;                // offsets inside a slot
-    uint32_t slot_bytes;
-    uint32_t off_wr, off_hid, off_partial, off_xchg, off_gates, off_meta, off_bars, total;
+    uint32_t chunk_bytes;  // one ring slot: a [dcc][N] router chunk or an [N][dcc] rows chunk
+    uint32_t hid_bytes;    // one hidden state: d elements
+    uint32_t off_wr, off_hring, off_hid, off_partial, off_gates, off_meta, off_bars, total;
 };
 __host__ __device__ inline uint32_t up128(uint32_t x) { return (x + 127u) & ~127u; }
-__host__ __device__ inline SmemMap smem_map(int N, int dc, int eb, int S, int stages, int wr_in_ring, int consumers)
+__host__ __device__ inline SmemMap smem_map(int N, int d, int dcc, int eb, int stages, int hring, int wr_in_ring,
+                                            int consumers)
 {
     SmemMap m;
-    m.rows_bytes = static_cast<uint32_t>(N) * dc * eb;
-    m.wr_bytes = static_cast<uint32_t>(dc) * N * eb;
-    m.hid_bytes = static_cast<uint32_t>(dc) * eb;
-    m.slot_wr = m.rows_bytes;
-    m.slot_hid = m.rows_bytes + (wr_in_ring ? m.wr_bytes : 0u);
-    m.slot_bytes = up128(m.slot_hid + m.hid_bytes);
+    m.chunk_bytes = static_cast<uint32_t>(N) * dcc * eb;
+    m.hid_bytes = static_cast<uint32_t>(d) * eb;
     const uint32_t warps = consumers / 32;
-    m.off_wr = stages * m.slot_bytes;
-    m.off_hid = m.off_wr + (wr_in_ring ? 0u : up128(m.wr_bytes));
+    m.off_wr = stages * up128(m.chunk_bytes);                                             // resident router matrix (L == 1)
+    m.off_hring = m.off_wr + (wr_in_ring ? 0u : up128(static_cast<uint32_t>(d) * N * eb));  // hidden states of the tokens in flight
+    m.off_hid = m.off_hring + hring * up128(m.hid_bytes);                                 // running hidden state between layers
     m.off_partial = m.off_hid + up128(m.hid_bytes);
-    m.off_xchg = m.off_partial + up128(2u * warps * N * 4);
-    m.off_gates = m.off_xchg + up128(2u * S * N * 4);
+    m.off_gates = m.off_partial + up128(warps * N * 4);
     m.off_meta = m.off_gates + up128(N * 4);
     m.off_bars = m.off_meta + up128((kMaxStages + 3) * 4);
-    m.total = m.off_bars + (2 * kMaxStages + 3) * 8;
+    m.total = m.off_bars + (2 * kMaxStages + 1) * 8;
     return m;
 }
 
@@ -149,29 +147,31 @@ __device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, vol
     return false;
 }
 
-// Partial router logits of one item over this block's dc columns, fast path (N a power of two
-// the kernel is compiled for).  The router slice [dc][N] is swept linearly, 16 bytes per lane,
-// so a warp reads 512 consecutive bytes per step (no bank conflicts for any N).  A 16-byte
-// vector holds either VEC consecutive experts of one column (N >= VEC) or VEC / N whole columns
-// (N < VEC); since the sweep stride is a multiple of 32 vectors, a lane always meets the same
-// experts and keeps only min(VEC, N) accumulators.
+// Partial router logits over one chunk of columns, fast path (N a power of two the kernel is
+// compiled for).  The router chunk [ncols][N] is swept linearly, 16 bytes per lane, so a warp
+// reads 512 consecutive bytes per step (no bank conflicts for any N).  A 16-byte vector holds
+// either VEC consecutive experts of one column (N >= VEC) or VEC / N whole columns (N < VEC);
+// since the sweep stride is a multiple of 32 vectors, a lane always meets the same experts and
+// keeps only min(VEC, N) accumulators, as fp32 pairs, across all chunks of an item.
 template <typename T, int NFAST>
-__device__ __forceinline__ void router_partial_fast(uint32_t waddr, uint32_t haddr, int dc, int tid, int lane, int nc,
-                                                    float *partial_warp)
-{
+struct Sweep {
     using E = Elem<T>;
-    constexpr int VEC = E::VEC;
-    constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
-    constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
-    constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
-    constexpr int PPC = NV / 2;                          // fp32 pairs per column of a vector
-    constexpr int UNR = 4;                               // vectors in flight per lane
+    static constexpr int VEC = E::VEC;
+    static constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
+    static constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
+    static constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
+    static constexpr int PPC = NV / 2;                          // fp32 pairs per column of a vector
+    static constexpr int UNR = 4;                               // vectors in flight per lane
     f32x2 acc[NV / 2];
+
+    __device__ __forceinline__ void clear()
+    {
 #pragma unroll
-    for (int i = 0; i < NV / 2; ++i) acc[i] = 0ull;
-    const int nvec = dc * NFAST / VEC;
-    // One vector: its VEC values, as fp32 pairs, times the hidden value(s) of its column(s).
-    auto mac = [&](const uint4 &w, const float (&h)[CPV]) {
+        for (int i = 0; i < NV / 2; ++i) acc[i] = 0ull;
+    }
+    // one vector: its VEC values, as fp32 pairs, times the hidden value(s) of its column(s)
+    __device__ __forceinline__ void mac(const uint4 &w, const float (&h)[CPV])
+    {
         f32x2 wp[VEC / 2];
         E::unpack_pairs(w, wp);
 #pragma unroll
@@ -180,43 +180,69 @@ __device__ __forceinline__ void router_partial_fast(uint32_t waddr, uint32_t had
 #pragma unroll
             for (int i = 0; i < PPC; ++i) acc[i] = fma2(hh, wp[cc * PPC + i], acc[i]);
         }
-    };
-    auto hidden_of = [&](int u, float (&h)[CPV]) {
+    }
+    static __device__ __forceinline__ void hidden_of(uint32_t haddr, int u, float (&h)[CPV])
+    {
 #pragma unroll
         for (int cc = 0; cc < CPV; ++cc) h[cc] = E::lds_scalar(haddr, NFAST >= VEC ? u / QL : u * CPV + cc);
-    };
-    int u0 = tid;
+    }
+    // waddr: the chunk in shared memory; haddr: the hidden values of the chunk's first column on
+    __device__ __forceinline__ void chunk(uint32_t waddr, uint32_t haddr, int ncols, int tid, int nc)
+    {
+        const int nvec = ncols * NFAST / VEC;
+        int u0 = tid;
 #pragma unroll 1
-    for (; u0 + (UNR - 1) * nc < nvec; u0 += UNR * nc) {  // full batches: all loads first, then the arithmetic
-        uint4 wv[UNR];
-        float hv[UNR][CPV];
+        for (; u0 + (UNR - 1) * nc < nvec; u0 += UNR * nc) {  // full batches: all loads first
+            uint4 wv[UNR];
+            float hv[UNR][CPV];
 #pragma unroll
-        for (int r = 0; r < UNR; ++r) {
-            wv[r] = lds128(waddr + 16u * (u0 + r * nc));
-            hidden_of(u0 + r * nc, hv[r]);
+            for (int r = 0; r < UNR; ++r) {
+                wv[r] = lds128(waddr + 16u * (u0 + r * nc));
+                hidden_of(haddr, u0 + r * nc, hv[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < UNR; ++r) mac(wv[r], hv[r]);
         }
-#pragma unroll
-        for (int r = 0; r < UNR; ++r) mac(wv[r], hv[r]);
-    }
 #pragma unroll 1
-    for (; u0 < nvec; u0 += nc) {  // tail
-        float h[CPV];
-        const uint4 w = lds128(waddr + 16u * u0);
-        hidden_of(u0, h);
-        mac(w, h);
+        for (; u0 < nvec; u0 += nc) {  // tail
+            float h[CPV];
+            const uint4 w = lds128(waddr + 16u * u0);
+            hidden_of(haddr, u0, h);
+            mac(w, h);
+        }
     }
-    float a[NV];
+    // sum over the lanes of the warp; partial_warp[j] = this warp's share of logit j
+    __device__ __forceinline__ void finish(int lane, float *partial_warp)
+    {
+        float a[NV];
 #pragma unroll
-    for (int i = 0; i < NV / 2; ++i) unpack2(acc[i], a[2 * i], a[2 * i + 1]);
-    int base = 0;
-    lane_reduce_scatter<NV, NV, 16, QL>(a, lane, base);
-    constexpr int left = ReduceScatterLeft<NV, 16, QL>::value;
-    const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
+        for (int i = 0; i < NV / 2; ++i) unpack2(acc[i], a[2 * i], a[2 * i + 1]);
+        int base = 0;
+        lane_reduce_scatter<NV, NV, 16, QL>(a, lane, base);
+        constexpr int left = ReduceScatterLeft<NV, 16, QL>::value;
+        const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
 #pragma unroll
-    for (int i = 0; i < left; ++i) partial_warp[first + i] = a[i];
-}
+        for (int i = 0; i < left; ++i) partial_warp[first + i] = a[i];
+    }
+};
+// any N <= 64: one warp per expert, lanes stride over the columns; partial[j] accumulates over chunks
+template <typename T>
+struct Sweep<T, 0> {
+    using E = Elem<T>;
+    __device__ __forceinline__ void clear() {}
+    __device__ __forceinline__ void chunk_any(uint32_t waddr, uint32_t haddr, int ncols, int N, int warp, int lane,
+                                              int nwarps, bool first, float *partial)
+    {
+        for (int j = warp; j < N; j += nwarps) {
+            float z = 0.f;
+            for (int cc = lane; cc < ncols; cc += 32) z = fmaf(E::lds_scalar(haddr, cc), E::lds_scalar(waddr, cc * N + j), z);
+            z = warp_sum(z);
+            if (lane == 0) partial[j] = first ? z : partial[j] + z;
+        }
+    }
+};
 
-// Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over this block's dc columns,
+// Weighted sum of one item (Eq. 8): out = res + sum_j g_j * row_j over one chunk of columns,
 // with g_j = e_j / sum_k e_k given as the un-normalised e_j: the lanes add up the e_j of their
 // experts next to the rows, so the normalisation costs no reduction of its own -- one reciprocal
 // and one multiply per column at the end.
