@@ -372,6 +372,13 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     }
 }
 
+// Wait for a phase of a ring barrier: one inline poll, then the bounded slow path.
+__device__ __forceinline__ bool wait_ring(uint64_t *bar, uint32_t parity, volatile int *dead)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_or_give_up(bar, parity, dead, kWaitPolls, false);
+}
+
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
 // P: lanes that share one 16-byte column group in the combine.
 template <typename T, int NFAST, int P>
@@ -385,124 +392,124 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
     pdl_launch_dependents();
 
     const int N = NFAST > 0 ? NFAST : p.N;
-    const int S = p.S, dc = p.dc, d = p.d, L = p.L, stages = p.stages, nc = p.consumers;
-    const SmemMap m = smem_map(N, dc, EB, S, stages, p.wr_in_ring, nc);
+    const int K = p.K, dcc = p.dcc, d = p.d, L = p.L, stages = p.stages, nc = p.consumers, HR = p.hring;
+    const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, p.wr_in_ring, nc);
+    const uint32_t slot_bytes = up128(m.chunk_bytes), hid_stride = up128(m.hid_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const long long C = gridDim.x / S, c = blockIdx.x / S;  // clusters in the grid, this block's cluster
-    const int s = static_cast<int>(blockIdx.x % S);         // column slice == rank in the cluster
-    const long long ntok = c < p.M ? (p.M - c + C - 1) / C : 0;
-    const long long nitems = ntok * L;
+    const long long G = gridDim.x, b0 = blockIdx.x;
+    const int ntok = b0 < p.M ? static_cast<int>((p.M - b0 + G - 1) / G) : 0;  // tokens of this block
+    const int cpi = (p.wr_in_ring ? 2 : 1) * K;                                // chunks per item
 
     volatile int *meta = reinterpret_cast<volatile int *>(smem + m.off_meta);  // [stages] row valid
     volatile int *dead = meta + kMaxStages;        // somebody gave up waiting
-    volatile int *issued = meta + kMaxStages + 1;  // items whose copies have been issued
+    volatile int *issued = meta + kMaxStages + 1;  // chunks whose copies have been issued
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + m.off_bars);
-    uint64_t *full = bars, *empty = bars + kMaxStages, *xbar = bars + 2 * kMaxStages, *wrbar = xbar + 2;
+    uint64_t *full = bars, *empty = bars + kMaxStages, *wrbar = bars + 2 * kMaxStages;
 
     if (tid == 0) {
         for (int st = 0; st < stages; ++st) {
             mbar_init(full + st, 1);
             mbar_init(empty + st, nc / 32);
         }
-        mbar_init(xbar, 1);
-        mbar_init(xbar + 1, 1);
         mbar_init(wrbar, 1);
         *dead = 0;
         *issued = 0;
         meta[kMaxStages + 2] = 0;  // a flag nobody raises: lets the drain waits run their full (short) course
         mbar_init_fence();
     }
-    if (S > 1) {  // peers may write into this block's shared memory only once its barriers exist
-        cluster_arrive_release();
-        cluster_wait_acquire();
-    } else {
-        __syncthreads();
-    }
+    __syncthreads();
 
     if (tid >= nc) {
-        // ================= producer warp: issues every copy, `stages` items ahead =================
+        // ================= producer warp: issues every copy, `stages` chunks ahead ================
         const bool ids64 = (p.flags & MOLE_FLAG_IDS_INT64) != 0;
-        long long k = 0, batch = -1, row = -1;
-        int l = 0, pst = 0;       // layer and ring slot of the next item to issue
+        long long batch = -1, row = -1;
+        int k = 0, l = 0, q = 0;  // token of this block, layer, chunk of the item: the next chunk to issue
+        int pst = 0, he = 0;      // its ring slot; hidden-ring entry of token k
         uint32_t pph = 1;         // parity of the `empty` phase that frees that slot (first reuse: phase 0 done)
-        if (!p.wr_in_ring && nitems > 0 && lane == 0) {
-            mbar_expect_tx(wrbar, m.wr_bytes);
-            bulk_g2s(smem + m.off_wr, static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(s) * m.wr_bytes,
-                     m.wr_bytes, wrbar);
+        const long long total = static_cast<long long>(ntok) * L * cpi;
+        if (!p.wr_in_ring && ntok > 0 && lane == 0) {
+            const uint32_t wr_bytes = static_cast<uint32_t>(d) * N * EB;
+            mbar_expect_tx(wrbar, wr_bytes);
+            bulk_g2s(smem + m.off_wr, p.w_router, wr_bytes, wrbar);
         }
-        // Everything of item `it` except (optionally) the hidden slice.
-        auto issue = [&](long long it, bool with_hidden) {
-            if (l == 0) {
+        auto hidden_copy = [&](int tok, int entry, int st) {
+            const long long t = b0 + static_cast<long long>(tok) * G;
+            bulk_g2s(smem + m.off_hring + static_cast<size_t>(entry) * hid_stride,
+                     static_cast<const unsigned char *>(p.hidden) + static_cast<size_t>(t) * d * EB, m.hid_bytes, full + st);
+        };
+        // Issue the next chunk; the hidden state (first chunk of a token) only if with_hidden.
+        auto issue = [&](long long ci, bool with_hidden) {
+            if (l == 0 && q == 0) {
                 if ((k & 31) == 0) {  // ids of the next 32 tokens of this block, one per lane
-                    const long long kk = k + lane;
+                    const int kk = k + lane;
                     batch = -1;
                     if (kk < ntok) {
-                        const long long t = c + kk * C;
+                        const long long t = b0 + static_cast<long long>(kk) * G;
                         batch = ids64 ? __ldg(static_cast<const long long *>(p.row_index) + t)
                                       : static_cast<long long>(__ldg(static_cast<const int *>(p.row_index) + t));
                     }
                 }
-                row = __shfl_sync(0xffffffffu, batch, static_cast<int>(k & 31));
+                row = __shfl_sync(0xffffffffu, batch, k & 31);
             }
             const bool valid = row >= 0 && row < p.rows;
+            const bool first = l == 0 && q == 0;
             const int st = pst;
-            unsigned char *slot = smem + static_cast<size_t>(st) * m.slot_bytes;
+            unsigned char *slot = smem + static_cast<size_t>(st) * slot_bytes;
             if (lane == 0) {
                 meta[st] = valid ? 1 : 0;
-                if (!valid && l == 0 && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
-                mbar_expect_tx(full + st, m.slot_hid + (l == 0 ? m.hid_bytes : 0u));
-                *issued = static_cast<int>(it + 1 < 0x7fffffff ? it + 1 : 0x7fffffff);
+                if (!valid && first && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
+                mbar_expect_tx(full + st, m.chunk_bytes + (first ? m.hid_bytes : 0u));
+                *issued = static_cast<int>(ci + 1 < 0x7fffffff ? ci + 1 : 0x7fffffff);
             }
             __syncwarp();
-            // an id outside the table gathers row 0 (always present); its routed term is dropped later
-            const unsigned char *src = static_cast<const unsigned char *>(p.lut) + static_cast<size_t>(l) * p.lut_stride +
-                                       (static_cast<size_t>(valid ? row : 0) * N * d + static_cast<size_t>(s) * dc) * EB;
-            if (S == 1) {
-                if (lane == 0) bulk_g2s(slot, src, m.rows_bytes, full + st);  // the N rows of an id are contiguous
+            if (p.wr_in_ring && q < K) {
+                // router chunk: columns q*dcc .. of W_r[l], contiguous
+                if (lane == 0)
+                    bulk_g2s(slot,
+                             static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(l) * p.wr_stride +
+                                 static_cast<size_t>(q) * m.chunk_bytes,
+                             m.chunk_bytes, full + st);
             } else {
-                const uint32_t piece = static_cast<uint32_t>(dc) * EB;
-                for (int j = lane; j < N; j += 32)
-                    bulk_g2s(slot + static_cast<size_t>(j) * piece, src + static_cast<size_t>(j) * d * EB, piece, full + st);
+                // rows chunk: columns kk*dcc .. of the N rows of the id.  An id outside the table
+                // gathers row 0 (always present); its routed term is dropped later.
+                const int kk = p.wr_in_ring ? q - K : q;
+                const unsigned char *src = static_cast<const unsigned char *>(p.lut) + static_cast<size_t>(l) * p.lut_stride +
+                                           (static_cast<size_t>(valid ? row : 0) * N * d + static_cast<size_t>(kk) * dcc) * EB;
+                if (K == 1) {
+                    if (lane == 0) bulk_g2s(slot, src, m.chunk_bytes, full + st);  // the N rows of an id are contiguous
+                } else {
+                    const uint32_t piece = static_cast<uint32_t>(dcc) * EB;
+                    for (int j = lane; j < N; j += 32)
+                        bulk_g2s(slot + static_cast<size_t>(j) * piece, src + static_cast<size_t>(j) * d * EB, piece, full + st);
+                }
             }
-            if (p.wr_in_ring && lane == 31)
-                bulk_g2s(slot + m.slot_wr,
-                         static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(l) * p.wr_stride +
-                             static_cast<size_t>(s) * m.wr_bytes,
-                         m.wr_bytes, full + st);
-            if (with_hidden && l == 0 && lane == 30) {
-                const long long t = c + k * C;
-                bulk_g2s(slot + m.slot_hid,
-                         static_cast<const unsigned char *>(p.hidden) +
-                             (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB,
-                         m.hid_bytes, full + st);
-            }
-            if (++l == L) {
-                l = 0;
-                ++k;
+            if (with_hidden && first && lane == 31) hidden_copy(k, he, st);
+            if (++q == cpi) {
+                q = 0;
+                if (++l == L) {
+                    l = 0;
+                    ++k;
+                    if (++he == HR) he = 0;
+                }
             }
             if (++pst == stages) {
                 pst = 0;
                 pph ^= 1u;
             }
         };
-        // The first `stages` items need no free slot and -- except for hidden, which the previous
+        // The first `stages` chunks need no free slot and -- except for hidden, which the previous
         // kernel of a chained launch writes -- nothing upstream: issue them before the grid
         // dependency is waited for.
-        const long long pre = nitems < stages ? nitems : stages;
-        for (long long it = 0; it < pre; ++it) issue(it, false);
+        const long long pre = total < stages ? total : stages;
+        for (long long ci = 0; ci < pre; ++ci) issue(ci, false);
         pdl_wait();
         fence_proxy_async_global();
-        if (lane == 30) {
-            for (long long it = 0; it < pre; it += L) {  // the items with l == 0
-                const long long t = c + (it / L) * C;
-                const int st = static_cast<int>(it % stages);
-                bulk_g2s(smem + static_cast<size_t>(st) * m.slot_bytes + m.slot_hid,
-                         static_cast<const unsigned char *>(p.hidden) +
-                             (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB,
-                         m.hid_bytes, full + st);
-            }
+        if (lane == 31) {
+            const int per_tok = L * cpi;  // chunk tok*per_tok is the first chunk of token tok
+            for (int tok = 0; static_cast<long long>(tok) * per_tok < pre; ++tok)
+                hidden_copy(tok, tok % HR, static_cast<int>((static_cast<long long>(tok) * per_tok) % stages));
         }
-        for (long long it = pre; it < nitems; ++it) {
+        for (long long ci = pre; ci < total; ++ci) {
             int ok = 1;
             if (lane == 0) {
                 ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, false, true);
@@ -513,152 +520,6 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
-            issue(it, true);
+            issue(ci, true);
         }
     } else {
-        // ================= consumer warps: router, softmax, combine ================================
-        pdl_wait();  // out may still be read, and hidden / residual written, by the previous kernel
-        const int nwarps = nc / 32;
-        const int ngrp = dc / VEC;  // 16-byte column groups of this block's slice
-        float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [2][nwarps][N]
-        float *xchg = reinterpret_cast<float *>(smem + m.off_xchg);        // [2][S][N]
-        float *gates = reinterpret_cast<float *>(smem + m.off_gates);  // [N] softmax numerators of the current item
-        bool alive = true;
-
-        auto give_up = [&]() {
-            if (lane == 0) {
-                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
-                *dead = 1;
-            }
-            alive = false;
-        };
-        if (!p.wr_in_ring && nitems > 0) {
-            const bool got = wait_or_give_up(wrbar, 0, dead, kWaitPolls, false);
-            if (!__all_sync(0xffffffffu, got)) give_up();
-        }
-
-        const uint32_t smem_base = smem_u32(smem);
-        const uint32_t hid_s = smem_base + m.off_hid;
-        const uint32_t gates_s = smem_u32(gates);
-        long long t = c;  // token of the current item
-        int l = 0, st = 0;
-        uint32_t ph = 0;  // ring slot of the current item and the parity of its use
-#pragma unroll 1
-        for (long long it = 0; it < nitems; ++it) {
-            const int par = static_cast<int>(it & 1);
-            const uint32_t slot_s = smem_base + static_cast<uint32_t>(st) * m.slot_bytes;
-            float *part = partial + par * nwarps * N;
-            float *xch = xchg + par * S * N;
-
-            if (alive) {
-                if (S > 1 && tid == 0) mbar_expect_tx(xbar + par, static_cast<uint32_t>(S) * N * 4u);  // tid 0 is in warp 0
-                const bool got = wait_or_give_up(full + st, ph, dead, kWaitPolls, false);
-                if (!__all_sync(0xffffffffu, got)) give_up();
-            } else if (it < *issued) {
-                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls, false);  // let copies in flight land
-            }
-
-            const uint32_t haddr = (l == 0) ? slot_s + m.slot_hid : hid_s;
-            int nparts = nwarps;
-            if (alive) {
-                const uint32_t waddr = p.wr_in_ring ? slot_s + m.slot_wr : smem_base + m.off_wr;
-                if constexpr (NFAST > 0) {
-                    router_partial_fast<T, NFAST>(waddr, haddr, dc, tid, lane, nc, part + warp * N);
-                } else {
-                    // any N: one warp per expert, lanes stride over the columns
-                    for (int j = warp; j < N; j += nwarps) {
-                        float z = 0.f;
-                        for (int cc = lane; cc < dc; cc += 32)
-                            z = fmaf(E::lds_scalar(haddr, cc), E::lds_scalar(waddr, cc * N + j), z);
-                        z = warp_sum(z);
-                        if (lane == 0) part[j] = z;
-                    }
-                    nparts = 1;
-                }
-            }
-            // warp 0 turns the partial logits into softmax numerators for everybody
-            if (warp != 0) {
-                named_bar_arrive(kBarLogits, nc);
-            } else {
-                named_bar_sync(kBarLogits, nc);
-                if (alive) {
-                    const int j0 = lane, j1 = lane + 32;
-                    float z0 = 0.f, z1 = 0.f;
-                    if (j0 < N) {
-#pragma unroll 8
-                        for (int w = 0; w < nparts; ++w) z0 += part[w * N + j0];
-                    }
-                    if (j1 < N) {
-#pragma unroll 8
-                        for (int w = 0; w < nparts; ++w) z1 += part[w * N + j1];
-                    }
-                    if (S > 1) {
-                        // block totals go to every block of the cluster (this one included), then
-                        // the S partial logits are summed in slice order by everybody
-                        const uint32_t dst = smem_u32(xch + s * N), bar = smem_u32(xbar + par);
-                        for (int q = 0; q < S; ++q) {
-                            if (j0 < N) st_async_f32(map_to_cta(dst + j0 * 4, q), z0, map_to_cta(bar, q));
-                            if (j1 < N) st_async_f32(map_to_cta(dst + j1 * 4, q), z1, map_to_cta(bar, q));
-                        }
-                        const bool got =
-                            wait_or_give_up(xbar + par, static_cast<uint32_t>((it >> 1) & 1), dead, kWaitPolls, true);
-                        if (!__all_sync(0xffffffffu, got)) give_up();
-                        z0 = 0.f, z1 = 0.f;
-                        if (j0 < N)
-                            for (int q = 0; q < S; ++q) z0 += xch[q * N + j0];
-                        if (j1 < N)
-                            for (int q = 0; q < S; ++q) z1 += xch[q * N + j1];
-                    }
-                    // softmax over all N experts (Eq. 4).  Only the numerators e_j = exp(z_j - m)
-                    // are formed here; the combine divides by their sum.  Any shift m gives the same
-                    // gates, so the (shuffle-heavy) maximum is taken only when some logit is large
-                    // enough for exp to leave the comfortable range.
-                    const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
-                    float zmax = 0.f;
-                    if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(j0 < N ? z0 : -INFINITY, j1 < N ? z1 : -INFINITY));
-                    const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
-                    const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
-                    if (j0 < N) gates[j0] = e0;
-                    if (j1 < N) gates[j1] = e1;
-                    if (p.gates_out && s == 0) {
-                        const float esum = warp_sum(e0 + e1);
-                        if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
-                        if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
-                    }
-                }
-            }
-            named_bar_sync(kBarGates, nc);
-
-            if (alive) {
-                const bool valid = meta[st] != 0;
-                const size_t gbyte = (static_cast<size_t>(t) * d + static_cast<size_t>(s) * dc) * EB;
-                const unsigned char *res_g =
-                    p.residual ? static_cast<const unsigned char *>(p.residual) + gbyte : nullptr;
-                unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + gbyte : nullptr;
-                combine_item<T, P>(slot_s, haddr, gates_s, res_g, dst, hid_s, N, ngrp, valid, warp, lane, nwarps);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty + st);  // this warp is done with the slot
-            // the next layer's router reads the hidden slice that all warps have just written
-            if (L > 1) named_bar_sync(kBarHidden, nc);
-            if (++l == L) {
-                l = 0;
-                t += C;
-            }
-            if (++st == stages) {
-                st = 0;
-                ph ^= 1u;
-            }
-        }
-    }
-    // No block of a cluster may leave while a peer can still write into its shared memory.
-    if (S > 1) {
-        __syncwarp();
-        cluster_arrive_release();
-        cluster_wait_acquire();
-    }
-}
-
-#endif  // __CUDACC__
-
-}  // namespace mole
