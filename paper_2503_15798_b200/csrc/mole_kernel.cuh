@@ -523,3 +523,150 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             issue(ci, true);
         }
     } else {
+        // ================= consumer warps: router, softmax, combine ================================
+        pdl_wait();  // out may still be read, and hidden / residual written, by the previous kernel
+        const int nwarps = nc / 32;
+        const int ngrp = dcc / VEC;  // 16-byte column groups of one chunk
+        float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [nwarps][N]
+        float *gates = reinterpret_cast<float *>(smem + m.off_gates);      // [N] softmax numerators of the current item
+        const uint32_t smem_base = smem_u32(smem);
+        const uint32_t hid_s = smem_base + m.off_hid, gates_s = smem_u32(gates);
+        const uint32_t chunk_cols_bytes = static_cast<uint32_t>(dcc) * EB;
+        bool alive = true;
+
+        auto give_up = [&]() {
+            if (lane == 0) {
+                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                *dead = 1;
+            }
+            alive = false;
+        };
+        // Make the ring slot `st` usable (its copies have landed) -- or, after a failure, give
+        // copies that were issued a short time to land so that none is in flight at exit.
+        long long ci = 0;  // chunks consumed so far
+        auto acquire = [&](int st, uint32_t ph) {
+            if (alive) {
+                if (!wait_ring(full + st, ph, dead)) give_up();
+            } else if (ci < *issued) {
+                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls, false);
+            }
+        };
+        if (!p.wr_in_ring && ntok > 0) {
+            if (!wait_or_give_up(wrbar, 0, dead, kWaitPolls, false)) give_up();
+        }
+
+        int st = 0, he = 0;  // ring slot of the next chunk, hidden-ring entry of the current token
+        uint32_t ph = 0;     // parity of the slot's current use
+        auto release = [&]() {  // hand the current slot back and move on to the next
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + st);
+            ++ci;
+            if (++st == stages) {
+                st = 0;
+                ph ^= 1u;
+            }
+        };
+        Sweep<T, NFAST> sweep;
+#pragma unroll 1
+        for (int k = 0; k < ntok; ++k) {
+            const long long t = b0 + static_cast<long long>(k) * G;
+            const size_t tbyte = static_cast<size_t>(t) * d * EB;
+#pragma unroll 1
+            for (int l = 0; l < L; ++l) {
+                // the item's hidden state: as loaded (first layer) or as left by the previous layer
+                const uint32_t haddr = (l == 0) ? smem_base + m.off_hring + static_cast<uint32_t>(he) * hid_stride : hid_s;
+
+                // ---- router: partial logits over all d columns ----
+                sweep.clear();
+                if (p.wr_in_ring) {
+#pragma unroll 1
+                    for (int q = 0; q < K; ++q) {
+                        acquire(st, ph);
+                        if (alive) {
+                            const uint32_t waddr = smem_base + static_cast<uint32_t>(st) * slot_bytes;
+                            if constexpr (NFAST > 0) sweep.chunk(waddr, haddr + q * chunk_cols_bytes, dcc, tid, nc);
+                            else sweep.chunk_any(waddr, haddr + q * chunk_cols_bytes, dcc, N, warp, lane, nwarps, q == 0, partial);
+                        }
+                        release();
+                    }
+                } else {
+                    acquire(st, ph);  // the first rows chunk brings the hidden state with it
+                    if (alive) {
+                        if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, haddr, d, tid, nc);
+                        else sweep.chunk_any(smem_base + m.off_wr, haddr, d, N, warp, lane, nwarps, true, partial);
+                    }
+                }
+                if constexpr (NFAST > 0) {
+                    if (alive) sweep.finish(lane, partial + warp * N);
+                }
+
+                // ---- warp 0 turns the partial logits into softmax numerators for everybody ----
+                if (warp != 0) {
+                    named_bar_arrive(kBarLogits, nc);
+                } else {
+                    named_bar_sync(kBarLogits, nc);
+                    if (alive) {
+                        const int j0 = lane, j1 = lane + 32;
+                        float z0 = 0.f, z1 = 0.f;
+                        if constexpr (NFAST > 0) {
+                            // fixed trip count, loads independent of one another (rows past nwarps repeat row 0, weight 0)
+#pragma unroll
+                            for (int w = 0; w < kMaxConsumers / 32; ++w) {
+                                const int ww = w < nwarps ? w : 0;
+                                const float a0 = j0 < N ? partial[ww * N + j0] : 0.f;
+                                z0 += w < nwarps ? a0 : 0.f;
+                                if constexpr (NFAST > 32) {
+                                    const float a1 = partial[ww * N + j1];
+                                    z1 += w < nwarps ? a1 : 0.f;
+                                }
+                            }
+                        } else {
+                            if (j0 < N) z0 = partial[j0];
+                            if (j1 < N) z1 = partial[j1];
+                        }
+                        // softmax over all N experts (Eq. 4).  Only the numerators e_j = exp(z_j - m)
+                        // are formed here; the combine divides by their sum.  Any shift m gives the same
+                        // gates, so the (shuffle-heavy) maximum is taken only when some logit is large
+                        // enough for exp to leave the comfortable range.
+                        const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
+                        float zmax = 0.f;
+                        if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(j0 < N ? z0 : -INFINITY, j1 < N ? z1 : -INFINITY));
+                        const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
+                        const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
+                        if (j0 < N) gates[j0] = e0;
+                        if (j1 < N) gates[j1] = e1;
+                        if (p.gates_out) {
+                            const float esum = warp_sum(e0 + e1);
+                            if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
+                            if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
+                        }
+                    }
+                }
+                named_bar_sync(kBarGates, nc);
+
+                // ---- weighted sum of the rows, chunk by chunk (Eq. 8) ----
+#pragma unroll 1
+                for (int kk = 0; kk < K; ++kk) {
+                    if (p.wr_in_ring || kk > 0) acquire(st, ph);
+                    if (alive) {
+                        const bool valid = meta[st] != 0;
+                        const uint32_t off = kk * chunk_cols_bytes;
+                        const unsigned char *res_g =
+                            p.residual ? static_cast<const unsigned char *>(p.residual) + tbyte + off : nullptr;
+                        unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + tbyte + off : nullptr;
+                        combine_item<T, P>(smem_base + static_cast<uint32_t>(st) * slot_bytes, haddr + off, gates_s, res_g, dst,
+                                           hid_s + off, N, ngrp, valid, warp, lane, nwarps);
+                    }
+                    release();
+                }
+                // the next layer's router reads the hidden state that all warps have just written
+                if (l + 1 < L) named_bar_sync(kBarHidden, nc);
+            }
+            if (++he == HR) he = 0;
+        }
+    }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace mole
