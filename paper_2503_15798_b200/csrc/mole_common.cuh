@@ -25,17 +25,18 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int elem_bytes(int dtype) { return dtype == MOLE_DTYPE_BF16 ? 2 : 4; }
 
 // Launch description of the fused kernel (filled by plan_step, pure host arithmetic).
-// A block owns one slice of dc = d / d_split columns of a token; it walks over its tokens and,
-// for every token, over the L layers, pulling the table rows of each (token, layer) item
-// through a ring of `stages` shared-memory slots.
+// A block owns whole tokens; it walks over its tokens and, for every token, over the L layers,
+// pulling the router matrix (L > 1) and the table rows of each (token, layer) item, cut into
+// d_split column chunks, through a ring of `stages` shared-memory slots.
 struct StepPlan {
-    int d_split;        // blocks per token (a cluster when > 1)
-    int dc;             // columns per block
+    int d_split;        // column chunks per token
+    int dc;             // columns per chunk
     int consumers;      // threads that compute (a multiple of 32); one more warp issues the copies
     int threads;        // consumers + 32
-    int stages;         // ring depth
-    int slot_bytes;     // one ring slot: rows [+ router slice] + hidden slice, padded to 128
-    int wr_in_ring;     // 1: the router slice travels with every item (L > 1); 0: loaded once per block
+    int stages;         // ring depth, in chunks
+    int hring;          // hidden states of tokens in flight
+    int slot_bytes;     // one ring slot
+    int wr_in_ring;     // 1: the router chunks travel through the ring; 0: router matrix loaded once per block
     int smem;           // dynamic shared memory, bytes
     int blocks_per_sm;  // resident blocks per SM the shared memory allows
     int n_fast;         // N if the unrolled router path exists for it, else 0

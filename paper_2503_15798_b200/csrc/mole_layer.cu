@@ -28,15 +28,20 @@ constexpr long long kFusedMaxTokens = 4096;   // above this a step runs as L cha
 
 // Lanes per 16-byte column group in the combine: as many (up to 4) as keep the block within
 // kMaxConsumers threads.
-static int lanes_per_group(int dc, int vec)
+static int lanes_per_group(int dcc, int vec)
 {
-    const int groups = dc / vec;
+    const int groups = dcc / vec;
     return groups * 4 <= kMaxConsumers ? 4 : (groups * 2 <= kMaxConsumers ? 2 : 1);
 }
-static int consumers_for(int dc, int vec)
+static int consumers_for(int dcc, int vec)
 {
-    const int lanes = (dc / vec) * lanes_per_group(dc, vec);
+    const int lanes = (dcc / vec) * lanes_per_group(dcc, vec);
     return round_up(lanes < kMaxConsumers ? lanes : kMaxConsumers, 32);
+}
+static int env_int(const char *name)  // debugging aids: MOLE_FORCE_* override parts of the plan
+{
+    const char *f = getenv(name);
+    return f ? atoi(f) : 0;
 }
 
 int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan)
@@ -45,66 +50,62 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     if (L < 1 || M < 0) return MOLE_ERR_INVALID_ARG;
     const int eb = elem_bytes(dtype), vec = 16 / eb;
     if (N < 1 || N > kMaxN || d < vec || d % vec != 0) return MOLE_ERR_UNSUPPORTED_SHAPE;
-    const int in_ring = L > 1 ? 1 : 0;
-    auto fits = [&](int S, int stages) {
-        const int dc = d / S;
-        return smem_map(N, dc, eb, S, stages, in_ring, consumers_for(dc, vec)).total <=
-               static_cast<uint32_t>(kSmemPerBlockMax);
+    // the router matrix stays resident only for a single layer, and only if it leaves room for the ring
+    const int in_ring = (L > 1 || static_cast<long long>(d) * N * eb > 96 * 1024) ? 1 : 0;
+    const int per_tok = L * (in_ring ? 2 : 1);  // chunks per token, per column chunk
+    auto total_smem = [&](int K, int stages) {
+        const int dcc = d / K;
+        const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
+        return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers_for(dcc, vec)).total;
     };
-    int S;
+    int K;
     if (d_split != 0) {
-        if (d_split != 1 && d_split != 2 && d_split != 4 && d_split != 8) return MOLE_ERR_INVALID_ARG;
+        if (d_split != 1 && d_split != 2 && d_split != 4 && d_split != 8 && d_split != 16) return MOLE_ERR_INVALID_ARG;
         if (d % (d_split * vec) != 0) return MOLE_ERR_UNSUPPORTED_SHAPE;
-        S = d_split;
-        if (!fits(S, 2)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        K = d_split;
+        if (total_smem(K, 2) > static_cast<uint32_t>(kSmemPerBlockMax)) return MOLE_ERR_UNSUPPORTED_SHAPE;
     } else {
-        // Split a token over more blocks while one item (rows + router slice) is too large for a
-        // ring of several slots, or while there are too few tokens to give every SM a block;
-        // stop when a row piece would drop under 512 bytes.
-        S = 1;
-        while (S < kMaxSplit && d % (2 * S * vec) == 0 && (d / (2 * S)) * eb >= 512) {
-            const long long item = static_cast<long long>(N) * (d / S) * eb * (1 + in_ring);
-            if (item > 48 * 1024 || M * S < kNumSMs) S *= 2;
-            else break;
-        }
-        while (!fits(S, 2)) {
-            if (S >= kMaxSplit || d % (2 * S * vec) != 0) return MOLE_ERR_UNSUPPORTED_SHAPE;
-            S *= 2;
+        // the fewest column chunks that keep one chunk at or under 32 KB (and a ring of two in shared memory)
+        K = 1;
+        while (static_cast<long long>(N) * (d / K) * eb > 32 * 1024 || total_smem(K, 2) > static_cast<uint32_t>(kSmemPerBlockMax)) {
+            if (K >= kMaxChunks || d % (2 * K * vec) != 0) {
+                if (total_smem(K, 2) <= static_cast<uint32_t>(kSmemPerBlockMax)) break;  // larger chunks, but they fit
+                return MOLE_ERR_UNSUPPORTED_SHAPE;
+            }
+            K *= 2;
         }
     }
-    const int dc = d / S;
-    const int consumers = consumers_for(dc, vec);
-    const SmemMap one = smem_map(N, dc, eb, S, 1, in_ring, consumers);
-    const int fixed = static_cast<int>(one.total - one.slot_bytes);
-    const int slot = static_cast<int>(one.slot_bytes);
-    // Resident blocks per SM wanted: enough to cover the work (up to 4), each with >= 2 slots.
-    long long want = (M * S + kNumSMs - 1) / kNumSMs;
-    want = want < 1 ? 1 : (want > 4 ? 4 : want);
-    int stages = 2;
-    for (; want >= 1; --want) {
-        const long long room = kSmemPerSM / want - 1024 - fixed;
-        stages = static_cast<int>(room / slot);
-        if (stages >= 2) break;
+    const int dcc = d / K;
+    const int consumers = consumers_for(dcc, vec);
+    // Resident blocks per SM aimed at: two token chains per SM once there are more tokens than SMs.
+    int want = M > kNumSMs ? 2 : 1;
+    if (env_int("MOLE_FORCE_TARGET_BLOCKS") > 0) want = env_int("MOLE_FORCE_TARGET_BLOCKS");
+    int stages = 0;
+    for (; want >= 1 && stages == 0; --want) {
+        const uint32_t budget = static_cast<uint32_t>(kSmemPerSM / want - 1024);
+        for (int s = kMaxStages; s >= 2; --s)
+            if (total_smem(K, s) <= budget && total_smem(K, s) <= static_cast<uint32_t>(kSmemPerBlockMax)) {
+                stages = s;
+                break;
+            }
     }
-    if (stages < 2) stages = 2;  // fits(S, 2) holds
-    if (stages > kMaxStages) stages = kMaxStages;
-    // no deeper than the items a block will see
+    if (stages == 0) stages = 2;  // total_smem(K, 2) fits a block (checked above)
+    // no deeper than the chunks a block will see
     const long long cap = static_cast<long long>(kNumSMs) * 4;
-    const long long blocks = M * S < cap ? M * S : cap;
-    const long long items = blocks > 0 ? ((M * S + blocks - 1) / blocks) * L : 1;
-    if (stages > items) stages = items < 2 ? 2 : static_cast<int>(items);
-    while (stages > 2 && !fits(S, stages)) --stages;
-    if (const char *f = getenv("MOLE_FORCE_STAGES")) {  // debugging aid: ring depth, if it fits
-        const int v = atoi(f);
-        if (v >= 2 && v <= kMaxStages && fits(S, v)) stages = v;
-    }
-    const SmemMap m = smem_map(N, dc, eb, S, stages, in_ring, consumers);
-    plan->d_split = S;
-    plan->dc = dc;
+    const long long blocks = M < cap ? (M > 0 ? M : 1) : cap;
+    const long long chunks = ((M + blocks - 1) / blocks) * per_tok * K;
+    if (stages > chunks) stages = chunks < 2 ? 2 : static_cast<int>(chunks);
+    const int forced = env_int("MOLE_FORCE_STAGES");
+    if (forced >= 2 && forced <= kMaxStages && total_smem(K, forced) <= static_cast<uint32_t>(kSmemPerBlockMax)) stages = forced;
+    const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
+    const SmemMap m = smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers);
+    plan->d_split = K;
+    plan->dc = dcc;
     plan->consumers = consumers;
     plan->threads = consumers + 32;
     plan->stages = stages;
-    plan->slot_bytes = static_cast<int>(m.slot_bytes);
+    plan->hring = hring;
+    plan->slot_bytes = static_cast<int>(up128(m.chunk_bytes));
     plan->wr_in_ring = in_ring;
     plan->smem = static_cast<int>(m.total);
     int per_sm = kSmemPerSM / (plan->smem + 1024);
@@ -198,7 +199,7 @@ int launch_step(const StepLaunch &a)
     StepPlan plan;
     int rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan);
     if (rc != MOLE_OK) return rc;
-    if (a.M * plan.d_split > 0x7fffffffLL) return MOLE_ERR_TOO_LARGE;
+    if (a.M * a.L > 0x3fffffffLL) return MOLE_ERR_TOO_LARGE;
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
@@ -209,13 +210,10 @@ int launch_step(const StepLaunch &a)
     int per_sm = 0;
     MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, plan.threads, plan.smem));
     if (per_sm < 1) per_sm = 1;
-    if (const char *f = getenv("MOLE_FORCE_BLOCKS_PER_SM")) {  // debugging aid
-        const int v = atoi(f);
-        if (v >= 1 && v < per_sm) per_sm = v;
-    }
-    long long grid = static_cast<long long>(per_sm) * sms / plan.d_split * plan.d_split;
-    if (grid < plan.d_split) grid = plan.d_split;
-    if (grid > a.M * plan.d_split) grid = a.M * plan.d_split;
+    if (env_int("MOLE_FORCE_BLOCKS_PER_SM") >= 1 && env_int("MOLE_FORCE_BLOCKS_PER_SM") < per_sm)
+        per_sm = env_int("MOLE_FORCE_BLOCKS_PER_SM");
+    long long grid = static_cast<long long>(per_sm) * sms;
+    if (grid > a.M) grid = a.M;
 
     StepParams p;
     p.hidden = a.hidden;
@@ -232,11 +230,11 @@ int launch_step(const StepLaunch &a)
     p.rows = a.rows;
     p.N = a.N;
     p.d = a.d;
-    p.S = plan.d_split;
-    p.dc = plan.dc;
+    p.K = plan.d_split;
+    p.dcc = plan.dc;
     p.L = a.L;
     p.stages = plan.stages;
-    p.slot_bytes = plan.slot_bytes;
+    p.hring = plan.hring;
     p.wr_in_ring = plan.wr_in_ring;
     p.consumers = plan.consumers;
     p.flags = a.flags;
@@ -247,18 +245,11 @@ int launch_step(const StepLaunch &a)
     cfg.blockDim = dim3(plan.threads, 1, 1);
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = a.stream;
-    cudaLaunchAttribute attrs[2];
+    cudaLaunchAttribute attrs[1];
     unsigned na = 0;
     if (a.flags & MOLE_FLAG_CHAIN) {
         attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attrs[na].val.programmaticStreamSerializationAllowed = 1;
-        ++na;
-    }
-    if (plan.d_split > 1) {
-        attrs[na].id = cudaLaunchAttributeClusterDimension;
-        attrs[na].val.clusterDim.x = plan.d_split;
-        attrs[na].val.clusterDim.y = 1;
-        attrs[na].val.clusterDim.z = 1;
         ++na;
     }
     cfg.attrs = attrs;

@@ -46,27 +46,24 @@ def test_args_struct_layout_matches_header(lib):
 
 def test_plan_shapes():
     P = binding.plan
-    # large batches, single layer: one block per token, a ring of slots, one producer warp
+    # rows of up to 32 KB per token travel as one chunk; a ring of slots and one producer warp
     for d in (768, 1024):
-        s, threads, smem, stages, per_sm = P(16384, 16, d)
-        assert s == 1 and 2 <= stages <= 8 and smem <= 227 * 1024 and threads == 2 * d // 8 + 32  # 2 lanes per column group
-        assert per_sm * smem <= 228 * 1024 and per_sm * stages >= 4
-    # the 1B-shaped rows (128 KB per token) are always split
-    s, threads, smem, stages, per_sm = P(16384, 32, 2048)
-    assert s >= 2 and stages >= 2 and smem <= 227 * 1024
-    # few tokens: split to occupy the SMs
-    assert P(64, 16, 768)[0] >= 2 and P(1, 16, 768)[0] >= 2
-    # an explicit split is honoured
+        k, threads, smem, stages, per_sm = P(16384, 16, d)
+        assert k == 1 and 2 <= stages <= 8 and smem <= 227 * 1024 and threads == 2 * d // 8 + 32  # 2 lanes per column group
+        assert per_sm >= 2 and per_sm * (smem + 1024) <= 228 * 1024
+    # the 1B-shaped rows (128 KB per token) are cut into column chunks of at most 32 KB
+    k, threads, smem, stages, per_sm = P(256, 32, 2048)
+    assert k == 4 and stages >= 2 and smem <= 227 * 1024
+    # few tokens: one block per SM may use all of its shared memory for a deep ring
+    B = binding.DTYPE_BF16
+    assert P(64, 16, 768, B, 0, 12)[3] > P(16384, 16, 768, B, 0, 12)[3] and P(64, 16, 768, B, 0, 12)[4] == 1
+    # an explicit number of chunks is honoured
     assert P(64, 16, 768, binding.DTYPE_BF16, 4)[0] == 4 and P(64, 16, 768, binding.DTYPE_BF16, 1)[0] == 1
-    # a fused 12-layer step carries the router slice in every slot: slots about twice as large
-    one = P(256, 16, 768, binding.DTYPE_BF16, 1, 1)
-    fused = P(256, 16, 768, binding.DTYPE_BF16, 1, 12)
-    assert fused[3] >= 2 and fused[2] <= 227 * 1024 and fused[2] / fused[3] > 1.5 * (one[2] - 16 * 768 * 2) / one[3]
-    # never a deeper ring than the items a block will see
-    assert P(1, 16, 768, binding.DTYPE_BF16, 1, 1)[3] == 2 and P(1, 16, 768, binding.DTYPE_BF16, 1, 3)[3] == 3
+    # never a deeper ring than the chunks a block will see
+    assert P(1, 16, 768, binding.DTYPE_BF16, 1, 1)[3] == 2 and P(1, 16, 768, binding.DTYPE_BF16, 1, 3)[3] == 6
     # fp32 tiny shape
-    s, threads, smem, stages, per_sm = P(64, 4, 64, binding.DTYPE_F32)
-    assert threads in (64, 96) and smem >= 2 * 4 * (64 // s) * 4
+    k, threads, smem, stages, per_sm = P(64, 4, 64, binding.DTYPE_F32)
+    assert k == 1 and threads == 96 and smem >= 2 * 4 * 64 * 4
 
 
 def test_plan_rejects_bad_shapes():
