@@ -134,11 +134,11 @@ __device__ __forceinline__ float warp_sum(float v)
 // `patient`: sleep after every failed poll (the producer, which runs several items ahead and
 // must not take issue slots from the warps that compute).
 __device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
-                                             bool cluster_scope, bool patient = false)
+                                             bool patient = false)
 {
 #pragma unroll 1
     for (uint32_t i = 0; i < polls; ++i) {
-        if (cluster_scope ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if (patient || i > 64) {
             __nanosleep(64);
             if ((i & 127u) == 0 && *dead) return false;
@@ -376,7 +376,7 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
 __device__ __forceinline__ bool wait_ring(uint64_t *bar, uint32_t parity, volatile int *dead)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return wait_or_give_up(bar, parity, dead, kWaitPolls, false);
+    return wait_or_give_up(bar, parity, dead, kWaitPolls);
 }
 
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
@@ -512,7 +512,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         for (long long ci = pre; ci < total; ++ci) {
             int ok = 1;
             if (lane == 0) {
-                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, false, true);
+                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, true);
                 if (!ok) {
                     if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
                     *dead = 1;
@@ -548,11 +548,11 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             if (alive) {
                 if (!wait_ring(full + st, ph, dead)) give_up();
             } else if (ci < *issued) {
-                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls, false);
+                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls);
             }
         };
         if (!p.wr_in_ring && ntok > 0) {
-            if (!wait_or_give_up(wrbar, 0, dead, kWaitPolls, false)) give_up();
+            if (!wait_or_give_up(wrbar, 0, dead, kWaitPolls)) give_up();
         }
 
         int st = 0, he = 0;  // ring slot of the next chunk, hidden-ring entry of the current token

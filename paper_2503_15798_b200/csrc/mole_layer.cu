@@ -206,7 +206,7 @@ int launch_step(const StepLaunch &a)
     StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)));
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
-    // a persistent grid: as many blocks as fit at once (whole clusters), never more than the work
+    // a persistent grid: as many blocks as fit at once never more than the tokens
     int per_sm = 0;
     MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, plan.threads, plan.smem));
     if (per_sm < 1) per_sm = 1;
