@@ -77,8 +77,10 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     }
     const int dcc = d / K;
     const int consumers = consumers_for(dcc, vec);
-    // Resident blocks per SM aimed at: two token chains per SM once there are more tokens than SMs.
-    int want = M > kNumSMs ? 2 : 1;
+    // Resident blocks per SM aimed at: one per token while tokens are few (each with the deepest ring
+    // that fits), up to four token chains per SM when there are many (shallower rings, more overlap).
+    int want = static_cast<int>((M + kNumSMs - 1) / kNumSMs);
+    want = want < 1 ? 1 : (want > 4 ? 4 : want);
     if (env_int("MOLE_FORCE_TARGET_BLOCKS") > 0) want = env_int("MOLE_FORCE_TARGET_BLOCKS");
     int stages = 0;
     for (; want >= 1 && stages == 0; --want) {
