@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-batch sweep and the isolated-launch rows")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--layers", type=int, default=0, help="override L (debugging; the line then says so)")
+    ap.add_argument("--offload", action="store_true",
+                    help="offload mode instead: table in pinned host memory, per-step dedup + row fetch overlapped with "
+                         "the previous layer's combine; roofline = measured host-link GB/s")
     return ap.parse_args()
 
 
@@ -130,6 +133,34 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's (all-reduce MAX; `dist` None for one process)."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, M: int, steps: int, ms: float) -> float:
+    """Replicas only (weak scaling): every rank runs its own M-token steps, so the job's rate is
+    world * M * steps over the slowest rank's time."""
+    return world * M * steps / (ms * 1e-3)
+
+
+def rank_seeds(rank: int, layer: int = 0, batch: int = 0, m: int = 0) -> dict:
+    """Per-rank seeds: every replica has its own tables, hidden states and id batches."""
+    return {"table": 1000 + layer + 100 * rank, "router": 2000 + layer, "hidden": 3000 + rank,
+            "ids": 4000 + 1000 * rank + batch + 7 * m}
+
+
+def reference_arm_runs_here(rank: int) -> bool:
+    """--impl reference under torchrun: rank 0 alone runs and prints; the others exit 0 without work."""
+    return rank == 0
+
+
 # ------------------------------------------------------------------------------------------------------
 # the CPU oracle leg (only bench.py's baseline leg and --impl reference execute oracle/)
 # ------------------------------------------------------------------------------------------------------
@@ -166,7 +197,7 @@ def run_reference(args):
     import oracle
     from paper_2503_15798_b200 import inputs
 
-    if int(os.environ.get("RANK", "0")) != 0:
+    if not reference_arm_runs_here(int(os.environ.get("RANK", "0"))):
         return
     sh = inputs.SHAPES[args.config]
     L = args.layers or sh.L
@@ -282,13 +313,13 @@ def run_mole(args):
     # ---- resident inputs: L tables, routers, hidden, rotating id batches (per-rank seeds) ----------
     luts = torch.empty((L, sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
     for l in range(L):
-        inputs.make_table(sh.V, sh.N, sh.d, seed=1000 + l + 100 * rank, device=dev, out=luts[l])
+        inputs.make_table(sh.V, sh.N, sh.d, seed=rank_seeds(rank, l)["table"], device=dev, out=luts[l])
     wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
     max_m = max([M] + ([b for b in sh.batches] if not args.no_sweep else []))
-    hidden_all = inputs.make_hidden(max_m, sh.d, seed=3000 + rank, device=dev)
+    hidden_all = inputs.make_hidden(max_m, sh.d, seed=rank_seeds(rank)["hidden"], device=dev)
 
     def batches_for(m):
-        return [inputs.make_ids(m, sh.V, seed=4000 + 1000 * rank + b + 7 * m, device=dev) for b in range(N_BATCHES)]
+        return [inputs.make_ids(m, sh.V, seed=rank_seeds(rank, 0, b, m)["ids"], device=dev) for b in range(N_BATCHES)]
 
     def barrier():
         if dist is not None:
@@ -305,12 +336,9 @@ def run_mole(args):
         ms = timed_ms(torch, lambda: graphs.run(0, args.steps))
     barrier()
     assert int(graphs.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     ms_per_step = ms / args.steps
-    value = world * M * args.steps / (ms * 1e-3)
+    value = whole_job_tokens_per_s(world, M, args.steps, ms)
     launches = args.steps * (1 if fused else L)
     launch_bytes = sh.step_bytes(M, L) if fused else sh.layer_bytes(M)
     achieved = launch_bytes / (ms * 1e-3 / launches) / 1e9
@@ -348,11 +376,8 @@ def run_mole(args):
     ms_e2e = timed_ms(torch, lambda: e2e_run(e2e_steps))
     wall_e2e = time.perf_counter() - t0
     barrier()
-    if dist is not None:
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    line["e2e"] = {"value": world * M * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
+    ms_e2e = max_over_ranks(ms_e2e, dist, dev)
+    line["e2e"] = {"value": whole_job_tokens_per_s(world, M, e2e_steps, ms_e2e), "unit": UNIT,
                    "h2d_bytes_per_step": M * sh.d * 2 + M * 4, "d2h_bytes_per_step": M * sh.d * 2,
                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
                    "how": "mole_decode_step_host: pinned host hidden+ids -> device, L chained layers, result -> "
@@ -432,8 +457,117 @@ def run_mole(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------------
+# offload mode: table in pinned host memory (410M-shaped by default), one JSON line of its own
+# ------------------------------------------------------------------------------------------------------
+
+def run_offload(args):
+    """Per decode step and layer: dedup the ids on the device, let the GPU fetch the distinct rows
+    from the pinned host table into an HBM staging buffer (side stream), combine from staging (main
+    stream); layer l+1's fetch overlaps layer l's combine through two buffers."""
+    import numpy as np
+    import torch
+
+    from paper_2503_15798_b200 import binding as mole
+    from paper_2503_15798_b200 import build as lib_build
+    from paper_2503_15798_b200 import inputs
+
+    lib_build.build()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = args.config if args.config != "160m" else "410m"
+    sh = inputs.SHAPES[cfg]
+    L = args.layers or sh.L
+    row_bytes = sh.row_bytes
+
+    # the host table, layer by layer (generated on the device, copied down once, outside any timed region)
+    host = mole.HostTable((L, sh.V, sh.N, sh.d), torch.bfloat16)
+    tmp = torch.empty((sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        inputs.make_table(sh.V, sh.N, sh.d, seed=1000 + l, device=dev, out=tmp)
+        host.tensor[l].copy_(tmp)
+    torch.cuda.synchronize()
+    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
+
+    # host link, measured: a large pinned host -> device copy, and the GPU-initiated read of the same bytes
+    nrows = 8192
+    big = torch.empty((nrows, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    src = host.tensor[0][:nrows]
+    big.copy_(src, non_blocking=True)
+    torch.cuda.synchronize()
+    ms_copy = min(timed_ms(torch, lambda: big.copy_(src, non_blocking=True)) for _ in range(5))
+    link_copy = nrows * row_bytes / ms_copy / 1e6
+    uniq_all = torch.arange(nrows, dtype=torch.int32, device=dev)
+    cnt_all = torch.tensor([nrows], dtype=torch.int32, device=dev)
+    mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)
+    torch.cuda.synchronize()
+    ms_fetch = min(timed_ms(torch, lambda: mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)) for _ in range(5))
+    link_fetch = nrows * row_bytes / ms_fetch / 1e6
+    del big
+
+    rows = []
+    side = torch.cuda.Stream()
+    for M in (1, 8, 64):
+        ctx = mole.OffloadContext(M, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
+        hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
+        bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
+        id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        uniq_rows = float(np.mean([len(np.unique(b.cpu().numpy())) for b in id_batches]))
+
+        def step(k):
+            ids = id_batches[k % N_BATCHES]
+            main = torch.cuda.current_stream()
+            side.wait_stream(main)
+            ctx.prefetch(0, ids, host.tensor[0], side)
+            h = hidden
+            for l in range(L):
+                if l + 1 < L:
+                    ctx.prefetch((l + 1) % 2, ids, host.tensor[l + 1], side)  # overlaps layer l's combine
+                out = bufs[l % 2]
+                ctx.forward(l % 2, h, wrs[l], out, status=status)
+                h = out
+
+        steps = max(20, min(args.steps, 400))
+        for k in range(max(args.warmup, 3)):
+            step(k)
+        torch.cuda.synchronize()
+        ms = timed_ms(torch, lambda: [step(k) for k in range(steps)])
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        us_step = ms * 1e3 / steps
+        link_bytes = uniq_rows * row_bytes * L  # distinct rows only cross the link
+        rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
+                     "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
+                     "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
+                     "launches_per_step": 3 * L})
+        ctx.destroy()
+    top = rows[-1]
+    line = {
+        "metric": "MoLE offload-mode tokens/s (L-layer decode step) and achieved host-link GB/s", "value": top["tokens_per_s"],
+        "unit": UNIT, "n_gpus": 1, "steps": max(20, min(args.steps, 400)), "warmup": max(args.warmup, 3),
+        "ms_per_step": top["us_per_step"] / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{sh.name}-shaped offload decode: table {sh.layer_table_bytes * L / 1e9:.2f} GB in pinned host "
+                               f"memory, L={L}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
+                   "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": 64,
+                   "l2": "rows come from host memory; 32 rotating id batches"},
+        "gpu_launches": 3 * L * max(20, min(args.steps, 400)),
+        "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": link_fetch, "unit": "GB/s",
+                     "frac": top["frac_of_link"], "traffic": None, "kernel": "mole_fetch_kernel",
+                     "peak_source": "measured in this run: GPU-initiated read of 8192 rows of the pinned table "
+                                    f"({link_fetch:.1f} GB/s; cudaMemcpyAsync of the same bytes {link_copy:.1f} GB/s)"},
+        "host_link": {"memcpy_GBps": link_copy, "gpu_read_GBps": link_fetch},
+        "sweep": rows,
+    }
+    host.free()
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.offload:
+        return run_offload(args)
     if args.impl == "reference":
         run_reference(args)
     else:
