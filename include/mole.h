@@ -118,8 +118,9 @@ typedef struct mole_args {
     int32_t B, T, N, d, V;
     int32_t dtype;         /* MOLE_DTYPE_* */
     int32_t reserved;      /* must be 0 */
-    int32_t d_split;       /* blocks per token (1, 2, 4 or 8; d/d_split must stay a multiple of the vector width); 0 = auto.
-                              The d_split blocks of a token form a thread-block cluster and exchange partial logits. */
+    int32_t d_split;       /* column chunks a token's rows are streamed in (1, 2, 4, 8 or 16; d/d_split must stay a
+                              multiple of the vector width); 0 = auto: the fewest chunks of at most 32 KB.  The
+                              chunking fixes the order of the fp32 sums: equal d_split, bit-identical results. */
     void *stream;          /* cudaStream_t */
 } mole_args;
 
@@ -272,7 +273,7 @@ MOLE_API const char *mole_last_cuda_error(void);
 MOLE_API int mole_version(void);
 
 /* launch shape the library would pick for M tokens and L layers in one launch (L = 1: a single
- * layer): blocks per token, threads per block, dynamic shared memory, depth of the row ring,
+ * layer): column chunks per token, threads per block, dynamic shared memory, depth of the ring,
  * resident blocks per SM.  Pure host arithmetic, no CUDA call. */
 MOLE_API int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads,
               int *out_smem_bytes, int *out_stages, int *out_blocks_per_sm);
