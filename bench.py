@@ -176,7 +176,7 @@ def time_oracle(table_bits, wr_bits, hidden_bits, id_batches, L, budget_s, threa
         oracle.layer_lookup(hidden_bits, id_batches[calls % len(id_batches)], table_bits, wr_bits, threads=threads)
         calls += 1
         dt = time.perf_counter() - t0
-        if dt >= budget_s or calls >= 4096:
+        if dt >= budget_s or calls >= 1000000:
             break
     M = hidden_bits.shape[0]
     return M * calls / dt / L, calls, dt
@@ -441,8 +441,8 @@ def run_mole(args):
         cores = oracle.effective_threads(len(os.sched_getaffinity(0)))
         table0 = host_bits(luts[0])
         ids_np = [b.cpu().numpy().astype(np.int64) for b in batches_for(M)]
-        v_all, calls, dt = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 8.0, cores)
-        v_one, calls1, dt1 = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 4.0, 1)
+        v_all, calls, dt = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 12.0, cores)
+        v_one, calls1, dt1 = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 5.0, 1)
         line["cpu_baseline"] = {
             "value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{calls} calls of the oracle's lookup-form layer (fp64) on a host copy of layer 0's table, "
