@@ -26,12 +26,16 @@ constexpr int kSmemPerBlockMax = 227 * 1024;  // opt-in limit per block
 constexpr int kSmemPerSM = 228 * 1024;        // per SM, of which every resident block reserves 1 KB
 constexpr long long kFusedMaxTokens = 4096;   // above this a step runs as L chained launches
 
-// Lanes per 16-byte column group in the combine: as many (up to 4) as keep the block within
-// kMaxConsumers threads.
+// Lanes per 16-byte column group in the combine (1, 2 or 4).
+static int env_int(const char *name);
 static int lanes_per_group(int dcc, int vec)
 {
     const int groups = dcc / vec;
-    return groups * 4 <= kMaxConsumers ? 4 : (groups * 2 <= kMaxConsumers ? 2 : 1);
+    const int forced = env_int("MOLE_FORCE_LANES");  // debugging aid
+    if ((forced == 1 || forced == 2 || forced == 4) && groups * forced <= kMaxConsumers) return forced;
+    // about four compute warps -- one per SM sub-partition -- measured best: more warps repeat the
+    // per-item bookkeeping, fewer lengthen the chain of an item
+    return groups * 4 <= 128 ? 4 : (groups * 2 <= 128 ? 2 : 1);
 }
 static int consumers_for(int dcc, int vec)
 {

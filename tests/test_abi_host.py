@@ -49,7 +49,7 @@ def test_plan_shapes():
     # rows of up to 32 KB per token travel as one chunk; a ring of slots and one producer warp
     for d in (768, 1024):
         k, threads, smem, stages, per_sm = P(16384, 16, d)
-        assert k == 1 and 2 <= stages <= 8 and smem <= 227 * 1024 and threads == 2 * d // 8 + 32  # 2 lanes per column group
+        assert k == 1 and 2 <= stages <= 8 and smem <= 227 * 1024 and threads == d // 8 + 32  # one lane per column group
         assert per_sm >= 2 and per_sm * (smem + 1024) <= 228 * 1024
     # the 1B-shaped rows (128 KB per token) are cut into column chunks of at most 32 KB
     k, threads, smem, stages, per_sm = P(256, 32, 2048)
@@ -63,7 +63,7 @@ def test_plan_shapes():
     assert P(1, 16, 768, binding.DTYPE_BF16, 1, 1)[3] == 2 and P(1, 16, 768, binding.DTYPE_BF16, 1, 3)[3] == 6
     # fp32 tiny shape
     k, threads, smem, stages, per_sm = P(64, 4, 64, binding.DTYPE_F32)
-    assert k == 1 and threads == 96 and smem >= 2 * 4 * 64 * 4
+    assert k == 1 and threads == 96 and smem >= 2 * 4 * 64 * 4  # 16 groups x 4 lanes + the producer warp
 
 
 def test_plan_rejects_bad_shapes():
