@@ -464,7 +464,7 @@ def run_mole(args):
 def run_offload(args):
     """Per decode step and layer: dedup the ids on the device, let the GPU fetch the distinct rows
     from the pinned host table into an HBM staging buffer (side stream), combine from staging (main
-    stream); layer l+1's fetch overlaps layer l's combine through two buffers."""
+    stream); layer l+1's fetch overlaps layer l's combine through two buffers (mole_offload_decode_step)."""
     import numpy as np
     import torch
 
@@ -515,18 +515,11 @@ def run_offload(args):
         status = torch.zeros(1, dtype=torch.int32, device=dev)
         uniq_rows = float(np.mean([len(np.unique(b.cpu().numpy())) for b in id_batches]))
 
-        def step(k):
-            ids = id_batches[k % N_BATCHES]
-            main = torch.cuda.current_stream()
-            side.wait_stream(main)
-            ctx.prefetch(0, ids, host.tensor[0], side)
-            h = hidden
-            for l in range(L):
-                if l + 1 < L:
-                    ctx.prefetch((l + 1) % 2, ids, host.tensor[l + 1], side)  # overlaps layer l's combine
-                out = bufs[l % 2]
-                ctx.forward(l % 2, h, wrs[l], out, status=status)
-                h = out
+        luts_host = host.tensor  # [L][V][N][d], pinned and device-mapped
+
+        def step(k):  # one call per step: one dedup, layer l+1's fetch under layer l's combine
+            ctx.decode_step(hidden, id_batches[k % N_BATCHES], luts_host, wrs, bufs[0], bufs[1], status=status,
+                            side_stream=side)
 
         steps = max(20, min(args.steps, 400))
         for k in range(max(args.warmup, 3)):
@@ -540,7 +533,7 @@ def run_offload(args):
         rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                      "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                      "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 3 * L})
+                     "launches_per_step": 1 + 2 * L})
         ctx.destroy()
     top = rows[-1]
     line = {
@@ -552,7 +545,7 @@ def run_offload(args):
                                f"memory, L={L}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
                    "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": 64,
                    "l2": "rows come from host memory; 32 rotating id batches"},
-        "gpu_launches": 3 * L * max(20, min(args.steps, 400)),
+        "gpu_launches": (1 + 2 * L) * max(20, min(args.steps, 400)),
         "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": link_fetch, "unit": "GB/s",
                      "frac": top["frac_of_link"], "traffic": None, "kernel": "mole_fetch_kernel",
                      "peak_source": "measured in this run: GPU-initiated read of 8192 rows of the pinned table "

@@ -262,6 +262,23 @@ MOLE_API int mole_offload_prefetch(mole_offload_ctx *ctx, int buf, const int32_t
 MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const void *hidden, const void *w_router, void *out,
                                uint32_t *status, int B, int T, void *stream);
 
+/*
+ * mole_offload_decode_step -- a whole L-layer decode step in offload mode, one call: the ids
+ * are deduplicated ONCE (they are the same for every layer), then layer l+1's distinct rows are
+ * fetched from its host table on side_stream while layer l combines on stream (the paper issues
+ * the row transfer first so that it overlaps the rest of the layer, App. A.2 listing).  Needs a
+ * context with n_buffers >= 2.
+ *   hidden_in device [M][d], read only;  out device [M][d] final result;  tmp device [M][d]
+ *   scratch (may be NULL when L == 1);  lut_host_base HOST pointer (pinned + mapped) of layer 0's
+ *   table, layer l at + l*lut_layer_stride_bytes;  w_router_base device, layer l at
+ *   + l*wr_layer_stride_bytes.
+ * Output is bit-identical to L calls of mole_layer_forward.  stream and side_stream must differ.
+ */
+MOLE_API int mole_offload_decode_step(mole_offload_ctx *ctx, const void *hidden_in, const int32_t *ids,
+                             const void *lut_host_base, int64_t lut_layer_stride_bytes, const void *w_router_base,
+                             int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status, int L, int B, int T,
+                             void *stream, void *side_stream);
+
 /* device pointers of a buffer's arrays, for inspection: uniq [max_tokens], slot [max_tokens], count [1], staging */
 MOLE_API int mole_offload_buffers(mole_offload_ctx *ctx, int buf, const int32_t **uniq, const int32_t **slot,
                          const int32_t **count, const void **staging);

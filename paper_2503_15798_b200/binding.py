@@ -26,7 +26,8 @@ STEP_AUTO, STEP_FUSED, STEP_CHAINED = 0, 1, 2
 EXPORTS = (
     "mole_layer_forward", "mole_layer_forward_ex", "mole_decode_step", "mole_decode_step_ex", "mole_decode_step_host",
     "mole_dedup_ids", "mole_dedup_ids_static", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
-    "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_buffers",
+    "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_decode_step",
+    "mole_offload_buffers",
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan",
 )
 
@@ -81,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.mole_offload_destroy.argtypes = [vp]
         L.mole_offload_prefetch.argtypes = [vp, c_int, ip, c_int, vp, vp]
         L.mole_layer_forward_offload.argtypes = [vp, c_int, vp, vp, vp, vp, c_int, c_int, vp]
+        L.mole_offload_decode_step.argtypes = [vp, vp, ip, vp, c_int64, vp, c_int64, vp, vp, vp, c_int, c_int, c_int, vp, vp]
         L.mole_offload_buffers.argtypes = [vp, c_int, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
                                            POINTER(c_void_p)]
         L.mole_status_string.argtypes = [c_int]
@@ -289,6 +291,17 @@ class OffloadContext:
         M = hidden.numel() // self.d
         _check(lib().mole_layer_forward_offload(self.handle, buf, _ptr(hidden), _ptr(w_router), _ptr(out),
                                                 _ptr(status), M, 1, _stream(stream)), "mole_layer_forward_offload")
+        return out
+
+    def decode_step(self, hidden_in, ids, luts_host, w_routers, out, tmp=None, status=None, stream=None, side_stream=None):
+        """mole_offload_decode_step: luts_host [L][V][N][d] pinned host tensor, w_routers [L][d][N] device."""
+        L = luts_host.shape[0]
+        M = ids.numel()
+        _check(lib().mole_offload_decode_step(self.handle, _ptr(hidden_in), _ptr(ids), _ptr(luts_host),
+                                              luts_host.stride(0) * luts_host.element_size(), _ptr(w_routers),
+                                              w_routers.stride(0) * w_routers.element_size(), _ptr(out), _ptr(tmp),
+                                              _ptr(status), L, M, 1, _stream(stream), _stream(side_stream)),
+               "mole_offload_decode_step")
         return out
 
     def buffers(self, buf: int):

@@ -149,6 +149,7 @@ struct mole_offload_ctx {
     int max_tokens, N, d, V, dtype, n_buffers;
     long long row_bytes;
     int32_t *table;  // [V] dedup scratch, kept all zero between kernels
+    cudaEvent_t step_begin;  // orders the side stream after the main stream at the start of a whole step
     struct Buffer {
         unsigned char *staging;  // [max_tokens][N][d]
         int32_t *uniq, *slot, *count;
@@ -214,6 +215,7 @@ int mole_offload_destroy(mole_offload_ctx *c)
         delete[] c->buf;
     }
     if (c->table) cudaFree(c->table);
+    if (c->step_begin) cudaEventDestroy(c->step_begin);
     delete c;
     (void)cudaGetLastError();
     return MOLE_OK;
@@ -248,6 +250,7 @@ int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, in
     memset(c->buf, 0, sizeof(mole_offload_ctx::Buffer) * n_buffers);
     cudaError_t e = cudaMalloc(&c->table, sizeof(int32_t) * static_cast<size_t>(V));
     if (e == cudaSuccess) e = cudaMemset(c->table, 0, sizeof(int32_t) * static_cast<size_t>(V));
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->step_begin, cudaEventDisableTiming);
     for (int b = 0; b < n_buffers && e == cudaSuccess; ++b) {
         mole_offload_ctx::Buffer &B = c->buf[b];
         e = cudaMalloc(&B.staging, static_cast<size_t>(c->row_bytes) * max_tokens);
@@ -322,6 +325,78 @@ int mole_layer_forward_offload(mole_offload_ctx *c, int b, const void *hidden, c
     int rc = launch_step(a);
     if (rc != MOLE_OK) return rc;
     MOLE_CUDA_TRY(cudaEventRecord(B.consumed, st));
+    return MOLE_OK;
+}
+
+int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const int32_t *ids, const void *lut_host_base,
+                             int64_t lut_layer_stride_bytes, const void *w_router_base, int64_t wr_layer_stride_bytes,
+                             void *out, void *tmp, uint32_t *status, int L, int B_, int T, void *stream, void *side_stream)
+{
+    if (!c || c->n_buffers < 2 || L < 1 || B_ < 0 || T < 0 || stream == side_stream) return MOLE_ERR_INVALID_ARG;
+    const long long M = static_cast<long long>(B_) * T;
+    if (M > c->max_tokens) return MOLE_ERR_TOO_LARGE;
+    if (M == 0) return MOLE_OK;
+    if (!hidden_in || !ids || !lut_host_base || !w_router_base || !out) return MOLE_ERR_INVALID_ARG;
+    if (!aligned16(hidden_in) || !aligned16(lut_host_base) || !aligned16(w_router_base) || !aligned16(out) ||
+        (lut_layer_stride_bytes & 15) || (wr_layer_stride_bytes & 15))
+        return MOLE_ERR_INVALID_ARG;
+    if (L > 1 && (!tmp || !aligned16(tmp) || out == hidden_in || tmp == hidden_in || tmp == out)) return MOLE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream), side = static_cast<cudaStream_t>(side_stream);
+    mole_offload_ctx::Buffer &B0 = c->buf[0], &B1 = c->buf[1];
+
+    // the side stream starts after whatever the caller has queued on the main stream (ids, tables) and
+    // after the previous step's layers have stopped reading the slot map and both staging areas
+    MOLE_CUDA_TRY(cudaEventRecord(c->step_begin, st));
+    MOLE_CUDA_TRY(cudaStreamWaitEvent(side, c->step_begin, 0));
+    MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B0.consumed, 0));
+    MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B1.consumed, 0));
+    // one dedup for the whole step: every layer looks up the same ids (slot map and distinct ids in buffer 0)
+    int rc = launch_dedup(ids, static_cast<int>(M), c->V, c->table, B0.uniq, B0.slot, B0.count, status, side);
+    if (rc != MOLE_OK) return rc;
+    B0.M = B1.M = static_cast<int>(M);
+
+    // fetch layer l's distinct rows into staging area l & 1 (once layer l-2 has finished with it)
+    auto fetch = [&](int l) -> int {
+        mole_offload_ctx::Buffer &Bl = c->buf[l & 1];
+        if (l >= 2) MOLE_CUDA_TRY(cudaStreamWaitEvent(side, Bl.consumed, 0));
+        int r = launch_fetch(static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l) * lut_layer_stride_bytes,
+                             B0.uniq, B0.count, static_cast<int>(M), c->row_bytes, Bl.staging, side);
+        if (r != MOLE_OK) return r;
+        MOLE_CUDA_TRY(cudaEventRecord(Bl.ready, side));
+        return MOLE_OK;
+    };
+    const void *src = hidden_in;
+    for (int l = 0; l < L; ++l) {
+        if (l == 0 && (rc = fetch(0)) != MOLE_OK) return rc;
+        if (l + 1 < L && (rc = fetch(l + 1)) != MOLE_OK) return rc;  // queued before layer l's combine: they overlap
+        mole_offload_ctx::Buffer &Bl = c->buf[l & 1];
+        void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
+        MOLE_CUDA_TRY(cudaStreamWaitEvent(st, Bl.ready, 0));
+        StepLaunch a;
+        a.hidden = src;
+        a.residual = nullptr;
+        a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
+        a.lut = Bl.staging;
+        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
+        a.out = dst;
+        a.gates_out = nullptr;
+        a.status = status;
+        a.lut_stride = 0;
+        a.wr_stride = 0;
+        a.M = M;
+        a.L = 1;
+        a.N = c->N;
+        a.d = c->d;
+        a.rows = c->max_tokens;
+        a.dtype = c->dtype;
+        a.flags = 0;
+        a.d_split = 0;
+        a.stream = st;
+        rc = launch_step(a);
+        if (rc != MOLE_OK) return rc;
+        MOLE_CUDA_TRY(cudaEventRecord(Bl.consumed, st));
+        src = dst;
+    }
     return MOLE_OK;
 }
 

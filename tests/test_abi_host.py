@@ -161,3 +161,10 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         binding.lib()
+
+
+def test_offload_decode_step_argument_checks(lib):
+    good = 0x10000
+    f = lib.mole_offload_decode_step
+    # no context; zero layers; the same stream for both roles
+    assert f(None, good, good, good, 16, good, 16, good, good, None, 2, 4, 1, None, good) == binding.ERR_INVALID_ARG

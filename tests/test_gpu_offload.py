@@ -193,3 +193,38 @@ def test_offload_bad_ids_and_size_checks():
     finally:
         ctx.destroy()
         host.free()
+
+
+@pytest.mark.parametrize("M,L", [(1, 3), (8, 5), (64, 4), (300, 2), (5, 1)])
+def test_offload_decode_step_equals_resident_layers(M, L):
+    """The whole offload step in one call (one dedup, fetch of layer l+1 under layer l's combine)
+    gives the bytes of L resident single-layer calls; repeated steps on one context stay correct."""
+    N, d, V = 16, 1024, 700
+    g = torch.Generator().manual_seed(100 + M)
+    host = mole.HostTable((L, V, N, d), torch.bfloat16)
+    ctx = mole.OffloadContext(max_tokens=M, N=N, d=d, V=V, n_buffers=2)
+    side = torch.cuda.Stream()
+    try:
+        host.tensor.copy_(torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16))
+        wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
+        hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
+        luts_dev = host.tensor.to(DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        for step in range(3):  # back-to-back steps reuse the slot map and both staging areas
+            ids_np = inputs.zipf_ids(M, V, seed=step)
+            if step == 2 and M > 2:
+                ids_np[1] = V + 5  # an id outside the table: no routed term in any layer
+            ids = torch.from_numpy(ids_np).to(DEV)
+            out, tmp = torch.empty_like(hidden), torch.empty_like(hidden)
+            ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, status=status, side_stream=side)
+            h = hidden
+            for l in range(L):
+                h = mole.layer_forward(h, ids, luts_dev[l], wrs[l])
+            torch.cuda.synchronize()
+            assert torch.equal(out, h)
+            if step == 2 and M > 2:
+                assert torch.equal(out[1], hidden[1])
+        assert int(status.item()) == (mole.STATUS_BAD_ID if M > 2 else 0)
+    finally:
+        ctx.destroy()
+        host.free()
