@@ -248,6 +248,24 @@ struct Elem<__nv_bfloat16> {
     }
     // element i of an array in shared memory (32-bit shared address)
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds16(base + 2 * i) << 16); }
+    // the same element as a raw 16-bit operand of the mixed-precision fma below
+    typedef unsigned short H;
+    static __device__ __forceinline__ H lds_h(uint32_t base, int i)
+    {
+        unsigned short v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(base + 2u * i));
+        return v;
+    }
+    // acc[e] += v[e] * h for the 8 values of a vector, through sm_100's mixed-precision fma
+    // (fma.rn.f32.bf16: bf16 x bf16 products are exact in fp32, one rounding at the add -- the
+    // same result as widening both operands and calling fmaf, without the widening instructions)
+    static __device__ __forceinline__ void fma_elem(float &acc, const uint4 &v, int e, H h)
+    {
+        const uint32_t w = e < 2 ? v.x : (e < 4 ? v.y : (e < 6 ? v.z : v.w));
+        unsigned short lo, hi;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+        asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(acc) : "h"((e & 1) ? hi : lo), "h"(h));
+    }
 };
 template <>
 struct Elem<float> {
@@ -278,6 +296,13 @@ struct Elem<float> {
         return reinterpret_cast<const float *>(p)[i];
     }
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds32(base + 4 * i)); }
+    typedef float H;
+    static __device__ __forceinline__ H lds_h(uint32_t base, int i) { return __uint_as_float(lds32(base + 4 * i)); }
+    static __device__ __forceinline__ void fma_elem(float &acc, const uint4 &v, int e, H h)
+    {
+        const uint32_t w = e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w));
+        acc = fmaf(h, __uint_as_float(w), acc);
+    }
 };
 #endif  // __CUDACC__
 

@@ -152,39 +152,33 @@ __device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, vol
 // reads 512 consecutive bytes per step (no bank conflicts for any N).  A 16-byte vector holds
 // either VEC consecutive experts of one column (N >= VEC) or VEC / N whole columns (N < VEC);
 // since the sweep stride is a multiple of 32 vectors, a lane always meets the same experts and
-// keeps only min(VEC, N) accumulators, as fp32 pairs, across all chunks of an item.
+// keeps only min(VEC, N) fp32 accumulators across all chunks of an item.
 template <typename T, int NFAST>
 struct Sweep {
     using E = Elem<T>;
+    using H = typename E::H;
     static constexpr int VEC = E::VEC;
     static constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
     static constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
     static constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
-    static constexpr int PPC = NV / 2;                          // fp32 pairs per column of a vector
-    static constexpr int UNR = 4;                               // vectors in flight per lane
-    f32x2 acc[NV / 2];
+    static constexpr int UNR = 16;  // vectors in flight per lane: all of a chunk for the shapes of Table 2
+    float acc[NV];
 
     __device__ __forceinline__ void clear()
     {
 #pragma unroll
-        for (int i = 0; i < NV / 2; ++i) acc[i] = 0ull;
+        for (int i = 0; i < NV; ++i) acc[i] = 0.f;
     }
-    // one vector: its VEC values, as fp32 pairs, times the hidden value(s) of its column(s)
-    __device__ __forceinline__ void mac(const uint4 &w, const float (&h)[CPV])
-    {
-        f32x2 wp[VEC / 2];
-        E::unpack_pairs(w, wp);
-#pragma unroll
-        for (int cc = 0; cc < CPV; ++cc) {
-            const f32x2 hh = pack2(h[cc], h[cc]);
-#pragma unroll
-            for (int i = 0; i < PPC; ++i) acc[i] = fma2(hh, wp[cc * PPC + i], acc[i]);
-        }
-    }
-    static __device__ __forceinline__ void hidden_of(uint32_t haddr, int u, float (&h)[CPV])
+    // one vector: its VEC values times the hidden value(s) of its column(s)
+    __device__ __forceinline__ void mac(const uint4 &w, const H (&h)[CPV])
     {
 #pragma unroll
-        for (int cc = 0; cc < CPV; ++cc) h[cc] = E::lds_scalar(haddr, NFAST >= VEC ? u / QL : u * CPV + cc);
+        for (int e = 0; e < VEC; ++e) E::fma_elem(acc[e % NV], w, e, h[e / NV]);
+    }
+    static __device__ __forceinline__ void hidden_of(uint32_t haddr, int u, H (&h)[CPV])
+    {
+#pragma unroll
+        for (int cc = 0; cc < CPV; ++cc) h[cc] = E::lds_h(haddr, NFAST >= VEC ? u / QL : u * CPV + cc);
     }
     // waddr: the chunk in shared memory; haddr: the hidden values of the chunk's first column on
     __device__ __forceinline__ void chunk(uint32_t waddr, uint32_t haddr, int ncols, int tid, int nc)
@@ -194,7 +188,7 @@ struct Sweep {
 #pragma unroll 1
         for (; u0 + (UNR - 1) * nc < nvec; u0 += UNR * nc) {  // full batches: all loads first
             uint4 wv[UNR];
-            float hv[UNR][CPV];
+            H hv[UNR][CPV];
 #pragma unroll
             for (int r = 0; r < UNR; ++r) {
                 wv[r] = lds128(waddr + 16u * (u0 + r * nc));
@@ -205,7 +199,7 @@ struct Sweep {
         }
 #pragma unroll 1
         for (; u0 < nvec; u0 += nc) {  // tail
-            float h[CPV];
+            H h[CPV];
             const uint4 w = lds128(waddr + 16u * u0);
             hidden_of(haddr, u0, h);
             mac(w, h);
@@ -214,15 +208,12 @@ struct Sweep {
     // sum over the lanes of the warp; partial_warp[j] = this warp's share of logit j
     __device__ __forceinline__ void finish(int lane, float *partial_warp)
     {
-        float a[NV];
-#pragma unroll
-        for (int i = 0; i < NV / 2; ++i) unpack2(acc[i], a[2 * i], a[2 * i + 1]);
         int base = 0;
-        lane_reduce_scatter<NV, NV, 16, QL>(a, lane, base);
+        lane_reduce_scatter<NV, NV, 16, QL>(acc, lane, base);
         constexpr int left = ReduceScatterLeft<NV, 16, QL>::value;
         const int first = (NFAST >= VEC ? (lane % QL) * VEC : 0) + base;
 #pragma unroll
-        for (int i = 0; i < left; ++i) partial_warp[first + i] = a[i];
+        for (int i = 0; i < left; ++i) partial_warp[first + i] = acc[i];
     }
 };
 // any N <= 64: one warp per expert, lanes stride over the columns; partial[j] accumulates over chunks
@@ -262,7 +253,7 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     constexpr int GPW = 32 / P;   // column groups per warp
     constexpr int W = 4 / P;      // 32-bit words a lane finishes
     constexpr int VPW = VEC / 4;  // values per word: 2 (bf16) or 1 (fp32)
-    constexpr int UNR = 4;        // rows in flight per lane
+    constexpr int UNR = (16 / P) < 4 ? 4 : 16 / P;  // rows in flight per lane: all of a lane's experts when N <= 16
     const int part = lane / GPW, gl = lane % GPW;
     const int chunk = (N + P - 1) / P;
     const int jb = part * chunk, je = (jb + chunk < N) ? jb + chunk : N;
@@ -271,10 +262,10 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
         const int grp = g0 + gl;
         const bool in = grp < ngrp;
         const int gg = in ? grp : ngrp - 1;
-        f32x2 accp[VEC / 2];
+        float acc[VEC];
         float esum = 0.f;
 #pragma unroll
-        for (int i = 0; i < VEC / 2; ++i) accp[i] = 0ull;
+        for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
         if (valid) {
             int j0 = jb;
 #pragma unroll 1
@@ -288,29 +279,24 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
                 }
 #pragma unroll
                 for (int r = 0; r < UNR; ++r) {
-                    f32x2 vp[VEC / 2];
-                    E::unpack_pairs(rv[r], vp);
-                    const f32x2 g2 = pack2(gv[r], gv[r]);
+                    float vf[VEC];
+                    E::unpack(rv[r], vf);
                     esum += gv[r];
 #pragma unroll
-                    for (int i = 0; i < VEC / 2; ++i) accp[i] = fma2(g2, vp[i], accp[i]);
+                    for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
                 }
             }
 #pragma unroll 1
             for (; j0 < je; ++j0) {  // tail
                 const uint4 rv = lds128(rows + 16u * (j0 * ngrp + gg));
                 const float g = __uint_as_float(lds32(gates + 4u * j0));
-                f32x2 vp[VEC / 2];
-                E::unpack_pairs(rv, vp);
-                const f32x2 g2 = pack2(g, g);
+                float vf[VEC];
+                E::unpack(rv, vf);
                 esum += g;
 #pragma unroll
-                for (int i = 0; i < VEC / 2; ++i) accp[i] = fma2(g2, vp[i], accp[i]);
+                for (int i = 0; i < VEC; ++i) acc[i] = fmaf(g, vf[i], acc[i]);
             }
         }
-        float acc[VEC];
-#pragma unroll
-        for (int i = 0; i < VEC / 2; ++i) unpack2(accp[i], acc[2 * i], acc[2 * i + 1]);
         int base = 0;
         if constexpr (P > 1) {
             lane_reduce_scatter<VEC, VEC, 16, GPW>(acc, lane, base);
