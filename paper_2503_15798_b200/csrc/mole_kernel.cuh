@@ -161,7 +161,7 @@ struct Sweep {
     static constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
     static constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
     static constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
-    static constexpr int UNR = 16;  // vectors in flight per lane: all of a chunk for the shapes of Table 2
+    static constexpr int UNR = 4;  // vectors in flight per lane (deeper batches grow the loop body; measured slower)
     float acc[NV];
 
     __device__ __forceinline__ void clear()
@@ -253,7 +253,7 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     constexpr int GPW = 32 / P;   // column groups per warp
     constexpr int W = 4 / P;      // 32-bit words a lane finishes
     constexpr int VPW = VEC / 4;  // values per word: 2 (bf16) or 1 (fp32)
-    constexpr int UNR = (16 / P) < 4 ? 4 : 16 / P;  // rows in flight per lane: all of a lane's experts when N <= 16
+    constexpr int UNR = 4;        // rows in flight per lane
     const int part = lane / GPW, gl = lane % GPW;
     const int chunk = (N + P - 1) / P;
     const int jb = part * chunk, je = (jb + chunk < N) ? jb + chunk : N;
@@ -356,6 +356,23 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
             }
         }
     }
+}
+
+// Cold paths, kept out of the consumers' loop body (its size shows in instruction-fetch stalls).
+__device__ __noinline__ void report_timeout(volatile int *dead, uint32_t *status)
+{
+    if (!*dead && status) atomicOr(status, MOLE_STATUS_TIMEOUT);
+    *dead = 1;
+}
+__device__ __noinline__ void write_gates(float *gates_out, long long t, int N, int lane, float e0, float e1)
+{
+    const float esum = warp_sum(e0 + e1);
+    if (lane < N) gates_out[t * N + lane] = e0 / esum;
+    if (lane + 32 < N) gates_out[t * N + lane + 32] = e1 / esum;
+}
+__device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
+{
+    return warp_max(fmaxf(lane < N ? z0 : -INFINITY, lane + 32 < N ? z1 : -INFINITY));
 }
 
 // Wait for a phase of a ring barrier: one inline poll, then the bounded slow path.
@@ -499,10 +516,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             int ok = 1;
             if (lane == 0) {
                 ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, true);
-                if (!ok) {
-                    if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
-                    *dead = 1;
-                }
+                if (!ok) report_timeout(dead, p.status);
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
@@ -521,10 +535,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         bool alive = true;
 
         auto give_up = [&]() {
-            if (lane == 0) {
-                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
-                *dead = 1;
-            }
+            if (lane == 0) report_timeout(dead, p.status);
             alive = false;
         };
         // Make the ring slot `st` usable (its copies have landed) -- or, after a failure, give
@@ -616,16 +627,12 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                         // enough for exp to leave the comfortable range.
                         const bool big = (j0 < N && !(fabsf(z0) < 80.f)) || (j1 < N && !(fabsf(z1) < 80.f));
                         float zmax = 0.f;
-                        if (__any_sync(0xffffffffu, big)) zmax = warp_max(fmaxf(j0 < N ? z0 : -INFINITY, j1 < N ? z1 : -INFINITY));
+                        if (__any_sync(0xffffffffu, big)) zmax = logit_max(z0, z1, N, lane);
                         const float e0 = j0 < N ? expf(z0 - zmax) : 0.f;
                         const float e1 = j1 < N ? expf(z1 - zmax) : 0.f;
                         if (j0 < N) gates[j0] = e0;
                         if (j1 < N) gates[j1] = e1;
-                        if (p.gates_out) {
-                            const float esum = warp_sum(e0 + e1);
-                            if (j0 < N) p.gates_out[t * N + j0] = e0 / esum;
-                            if (j1 < N) p.gates_out[t * N + j1] = e1 / esum;
-                        }
+                        if (p.gates_out) write_gates(p.gates_out, t, N, lane, e0, e1);
                     }
                 }
                 named_bar_sync(kBarGates, nc);
