@@ -125,28 +125,37 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
 
 typedef void (*StepKernel)(const StepParams);
 
-template <typename T, int P>
+template <typename T, int P, int MODE>
 static StepKernel pick_n(int n_fast)
 {
     switch (n_fast) {
-        case 4: return mole_step_kernel<T, 4, P>;
-        case 8: return mole_step_kernel<T, 8, P>;
-        case 16: return mole_step_kernel<T, 16, P>;
-        case 32: return mole_step_kernel<T, 32, P>;
-        case 64: return mole_step_kernel<T, 64, P>;
-        default: return mole_step_kernel<T, 0, P>;
+        case 4: return mole_step_kernel<T, 4, P, MODE>;
+        case 8: return mole_step_kernel<T, 8, P, MODE>;
+        case 16: return mole_step_kernel<T, 16, P, MODE>;
+        case 32: return mole_step_kernel<T, 32, P, MODE>;
+        case 64: return mole_step_kernel<T, 64, P, MODE>;
+        default: return nullptr;
     }
 }
 
-template <typename T>
+template <typename T, int MODE>
 static StepKernel pick_p(int n_fast, int lanes)
 {
-    return lanes == 4 ? pick_n<T, 4>(n_fast) : (lanes == 2 ? pick_n<T, 2>(n_fast) : pick_n<T, 1>(n_fast));
+    return lanes == 4 ? pick_n<T, 4, MODE>(n_fast) : (lanes == 2 ? pick_n<T, 2, MODE>(n_fast) : pick_n<T, 1, MODE>(n_fast));
 }
 
-static StepKernel pick_kernel(int dtype, int n_fast, int lanes)
+// The generic-N router and the fp32 storage type exist only with run-time flags (MODE 0); bf16 with
+// a compiled-in N also in the three specialised shapes.
+static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring)
 {
-    return dtype == MOLE_DTYPE_BF16 ? pick_p<__nv_bfloat16>(n_fast, lanes) : pick_p<float>(n_fast, lanes);
+    if (n_fast == 0) {
+        if (dtype == MOLE_DTYPE_BF16)
+            return lanes == 4 ? mole_step_kernel<__nv_bfloat16, 0, 4, 0> : (lanes == 2 ? mole_step_kernel<__nv_bfloat16, 0, 2, 0> : mole_step_kernel<__nv_bfloat16, 0, 1, 0>);
+        return lanes == 4 ? mole_step_kernel<float, 0, 4, 0> : (lanes == 2 ? mole_step_kernel<float, 0, 2, 0> : mole_step_kernel<float, 0, 1, 0>);
+    }
+    if (dtype != MOLE_DTYPE_BF16) return pick_p<float, 0>(n_fast, lanes);
+    if (chunks == 1) return in_ring ? pick_p<__nv_bfloat16, 1>(n_fast, lanes) : pick_p<__nv_bfloat16, 2>(n_fast, lanes);
+    return in_ring ? pick_p<__nv_bfloat16, 3>(n_fast, lanes) : pick_p<__nv_bfloat16, 0>(n_fast, lanes);
 }
 
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
@@ -209,7 +218,8 @@ int launch_step(const StepLaunch &a)
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)));
+    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)), plan.d_split, plan.wr_in_ring);
+    if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
     // a persistent grid: as many blocks as fit at once never more than the tokens
