@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
 
     const int N = NFAST > 0 ? NFAST : p.N;
     const int K = (MODE == 1 || MODE == 2) ? 1 : p.K, dcc = p.dcc, d = p.d, L = p.L, stages = p.stages, nc = p.consumers, HR = p.hring;
-    const bool ring = MODE == 0 ? (ring != 0) : (MODE != 2);  // router chunks travel through the ring
+    const bool ring = MODE == 0 ? (p.wr_in_ring != 0) : (MODE != 2);  // router chunks travel through the ring
     const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, ring, nc);
     const uint32_t slot_bytes = up128(m.chunk_bytes), hid_stride = up128(m.hid_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
