@@ -387,7 +387,15 @@ __device__ __forceinline__ bool wait_ring(uint64_t *bar, uint32_t parity, volati
 // MODE: the common launch shapes with their flags fixed at compile time (a smaller loop body:
 // measured 10 % faster), 0 = any: 1 = router chunks in the ring, one chunk per item; 2 = router
 // resident, one chunk per item; 3 = router chunks in the ring, several chunks per item.
-template <typename T, int NFAST, int P, int MODE>
+// SHAPE: the layer widths of the paper's Table 2 with d, the chunk width and the number of compute
+// threads as constants (0 = any): 1: d = 768; 2: d = 1024; 3: d = 2048 in chunks of 512.
+template <int SHAPE>
+struct ShapeOf {
+    static constexpr int d = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 2048);
+    static constexpr int dcc = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 512);
+    static constexpr int consumers = SHAPE == 1 ? 96 : 128;
+};
+template <typename T, int NFAST, int P, int MODE, int SHAPE>
 __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const StepParams p)
 {
     using E = Elem<T>;
@@ -398,7 +406,9 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
     pdl_launch_dependents();
 
     const int N = NFAST > 0 ? NFAST : p.N;
-    const int K = (MODE == 1 || MODE == 2) ? 1 : p.K, dcc = p.dcc, d = p.d, L = p.L, stages = p.stages, nc = p.consumers, HR = p.hring;
+    const int K = (MODE == 1 || MODE == 2) ? 1 : p.K, L = p.L, stages = p.stages, HR = p.hring;
+    const int dcc = SHAPE ? ShapeOf<SHAPE>::dcc : p.dcc, d = SHAPE ? ShapeOf<SHAPE>::d : p.d;
+    const int nc = SHAPE ? ShapeOf<SHAPE>::consumers : p.consumers;
     const bool ring = MODE == 0 ? (p.wr_in_ring != 0) : (MODE != 2);  // router chunks travel through the ring
     const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, ring, nc);
     const uint32_t slot_bytes = up128(m.chunk_bytes), hid_stride = up128(m.hid_bytes);

@@ -129,11 +129,11 @@ template <typename T, int P, int MODE>
 static StepKernel pick_n(int n_fast)
 {
     switch (n_fast) {
-        case 4: return mole_step_kernel<T, 4, P, MODE>;
-        case 8: return mole_step_kernel<T, 8, P, MODE>;
-        case 16: return mole_step_kernel<T, 16, P, MODE>;
-        case 32: return mole_step_kernel<T, 32, P, MODE>;
-        case 64: return mole_step_kernel<T, 64, P, MODE>;
+        case 4: return mole_step_kernel<T, 4, P, MODE, 0>;
+        case 8: return mole_step_kernel<T, 8, P, MODE, 0>;
+        case 16: return mole_step_kernel<T, 16, P, MODE, 0>;
+        case 32: return mole_step_kernel<T, 32, P, MODE, 0>;
+        case 64: return mole_step_kernel<T, 64, P, MODE, 0>;
         default: return nullptr;
     }
 }
@@ -146,12 +146,21 @@ static StepKernel pick_p(int n_fast, int lanes)
 
 // The generic-N router and the fp32 storage type exist only with run-time flags (MODE 0); bf16 with
 // a compiled-in N also in the three specialised shapes.
-static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring)
+static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers)
 {
+    // the layer widths of the paper's Table 2 (160M, 410M and 1B models) with their sizes compiled in
+    if (dtype == MOLE_DTYPE_BF16) {
+        if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 768 && consumers == 96)
+            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1>;
+        if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 1024 && consumers == 128)
+            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 2> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2>;
+        if (n_fast == 32 && lanes == 2 && chunks == 4 && d == 2048 && dcc == 512 && consumers == 128 && in_ring)
+            return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 3>;
+    }
     if (n_fast == 0) {
         if (dtype == MOLE_DTYPE_BF16)
-            return lanes == 4 ? mole_step_kernel<__nv_bfloat16, 0, 4, 0> : (lanes == 2 ? mole_step_kernel<__nv_bfloat16, 0, 2, 0> : mole_step_kernel<__nv_bfloat16, 0, 1, 0>);
-        return lanes == 4 ? mole_step_kernel<float, 0, 4, 0> : (lanes == 2 ? mole_step_kernel<float, 0, 2, 0> : mole_step_kernel<float, 0, 1, 0>);
+            return lanes == 4 ? mole_step_kernel<__nv_bfloat16, 0, 4, 0, 0> : (lanes == 2 ? mole_step_kernel<__nv_bfloat16, 0, 2, 0, 0> : mole_step_kernel<__nv_bfloat16, 0, 1, 0, 0>);
+        return lanes == 4 ? mole_step_kernel<float, 0, 4, 0, 0> : (lanes == 2 ? mole_step_kernel<float, 0, 2, 0, 0> : mole_step_kernel<float, 0, 1, 0, 0>);
     }
     if (dtype != MOLE_DTYPE_BF16) return pick_p<float, 0>(n_fast, lanes);
     if (chunks == 1) return in_ring ? pick_p<__nv_bfloat16, 1>(n_fast, lanes) : pick_p<__nv_bfloat16, 2>(n_fast, lanes);
@@ -218,7 +227,8 @@ int launch_step(const StepLaunch &a)
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)), plan.d_split, plan.wr_in_ring);
+    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)), plan.d_split, plan.wr_in_ring,
+                               a.d, plan.dc, plan.consumers);
     if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
