@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
 TRAFFIC = {
-    # profiles/mole_step_kernel_160m_batch256.md: 7.60 MB per 2-layer launch, x6 for the 12 layers of a full launch
-    ("160m", 256, 12): 45.6e6,
+    # profiles/mole_step_kernel_160m_batch256.md: 7.59 MB per 2-layer launch, x6 for the 12 layers of a full launch
+    ("160m", 256, 12): 45.5e6,
 }
 
 
