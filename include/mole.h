@@ -65,7 +65,7 @@ extern "C" {
 
 /* bits OR-ed by kernels into an optional device status word (uint32_t, caller zeroes it) */
 #define MOLE_STATUS_BAD_ID 1u  /* some id was outside [0, V) */
-#define MOLE_STATUS_TIMEOUT 2u /* a bounded wait inside a kernel gave up; output of that token not written */
+#define MOLE_STATUS_TIMEOUT 2u /* a bounded wait inside a kernel gave up; the launch's outputs are undefined */
 
 /* element type of hidden / residual / lut / w_router / out */
 #define MOLE_DTYPE_BF16 0

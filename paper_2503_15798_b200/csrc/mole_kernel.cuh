@@ -375,11 +375,20 @@ __device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
     return warp_max(fmaxf(lane < N ? z0 : -INFINITY, lane + 32 < N ? z1 : -INFINITY));
 }
 
-// Wait for a phase of a ring barrier: one inline poll, then the bounded slow path.
-__device__ __forceinline__ bool wait_ring(uint64_t *bar, uint32_t parity, volatile int *dead)
+// Everything about a ring slot that is not the first, successful poll: the bounded wait of a warp
+// that is still computing (returns whether the data arrived; reports the timeout otherwise), or --
+// for a warp that has given up -- a short wait that lets copies already issued land, so that none
+// is in flight when the block exits.
+__device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volatile int *dead, bool alive, bool issued,
+                                          uint32_t *status, int lane)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_or_give_up(bar, parity, dead, kWaitPolls);
+    if (alive) {
+        if (wait_or_give_up(bar, parity, dead, kWaitPolls)) return true;
+        if (lane == 0) report_timeout(dead, status);
+        return false;
+    }
+    if (issued) (void)wait_or_give_up(bar, parity, dead + 2, kDrainPolls);
+    return false;
 }
 
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
@@ -546,6 +555,10 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         const uint32_t smem_base = smem_u32(smem);
         const uint32_t hid_s = smem_base + m.off_hid, gates_s = smem_u32(gates);
         const uint32_t chunk_cols_bytes = static_cast<uint32_t>(dcc) * EB;
+        // After a wait has timed out (`alive` false) the warp stops waiting but keeps going through the
+        // arithmetic and the barriers on whatever the slots hold -- every address stays inside shared
+        // memory and the block's own rows of `out` -- so that no other warp is left at a barrier; the
+        // status word says that the outputs are meaningless.
         bool alive = true;
 
         auto give_up = [&]() {
@@ -556,11 +569,8 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         // copies that were issued a short time to land so that none is in flight at exit.
         long long ci = 0;  // chunks consumed so far
         auto acquire = [&](int st, uint32_t ph) {
-            if (alive) {
-                if (!wait_ring(full + st, ph, dead)) give_up();
-            } else if (ci < *issued) {
-                (void)wait_or_give_up(full + st, ph, dead + 2, kDrainPolls);
-            }
+            if (alive && mbar_try_wait(full + st, ph)) return;  // the usual case: the copies have landed
+            alive = acquire_slow(full + st, ph, dead, alive, ci < *issued, p.status, lane);
         };
         if (!ring && ntok > 0) {
             if (!wait_or_give_up(wrbar, 0, dead, kWaitPolls)) give_up();
@@ -593,7 +603,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
 #pragma unroll 1
                     for (int q = 0; q < K; ++q) {
                         acquire(st, ph);
-                        if (alive) {
+                        {
                             const uint32_t waddr = smem_base + static_cast<uint32_t>(st) * slot_bytes;
                             if constexpr (NFAST > 0) sweep.chunk(waddr, haddr + q * chunk_cols_bytes, dcc, tid, nc);
                             else sweep.chunk_any(waddr, haddr + q * chunk_cols_bytes, dcc, N, warp, lane, nwarps, q == 0, partial);
@@ -602,13 +612,13 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                     }
                 } else {
                     acquire(st, ph);  // the first rows chunk brings the hidden state with it
-                    if (alive) {
+                    {
                         if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, haddr, d, tid, nc);
                         else sweep.chunk_any(smem_base + m.off_wr, haddr, d, N, warp, lane, nwarps, true, partial);
                     }
                 }
                 if constexpr (NFAST > 0) {
-                    if (alive) sweep.finish(lane, partial + warp * N);
+                    sweep.finish(lane, partial + warp * N);
                 }
 
                 // ---- warp 0 turns the partial logits into softmax numerators for everybody ----
@@ -616,7 +626,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                     named_bar_arrive(kBarLogits, nc);
                 } else {
                     named_bar_sync(kBarLogits, nc);
-                    if (alive) {
+                    {
                         const int j0 = lane, j1 = lane + 32;
                         float z0 = 0.f, z1 = 0.f;
                         if constexpr (NFAST > 0) {
@@ -655,7 +665,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
 #pragma unroll 1
                 for (int kk = 0; kk < K; ++kk) {
                     if (ring || kk > 0) acquire(st, ph);
-                    if (alive) {
+                    {
                         const bool valid = meta[st] != 0;
                         const uint32_t off = kk * chunk_cols_bytes;
                         const unsigned char *res_g =
