@@ -175,35 +175,6 @@ __device__ __forceinline__ void sts32(uint32_t a, uint32_t v)
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
 }
 
-// Two fp32 values in one 64-bit register and the packed fused multiply-add of sm_100
-// (two independent IEEE fmas per instruction: same results as two scalar fmaf).
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
-    return r;
-}
-__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi)
-{
-    uint32_t a, b;
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
-    lo = __uint_as_float(a);
-    hi = __uint_as_float(b);
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
-{
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-
 // 16-byte vectors of the two storage types
 template <typename T>
 struct Elem;
@@ -220,31 +191,6 @@ struct Elem<__nv_bfloat16> {
         f[5] = __uint_as_float(v.z & 0xffff0000u);
         f[6] = __uint_as_float(v.w << 16);
         f[7] = __uint_as_float(v.w & 0xffff0000u);
-    }
-    // the 8 values as 4 fp32 pairs (columns 0-1, 2-3, 4-5, 6-7)
-    static __device__ __forceinline__ void unpack_pairs(const uint4 &v, f32x2 (&p)[4])
-    {
-        p[0] = pack2u(v.x << 16, v.x & 0xffff0000u);
-        p[1] = pack2u(v.y << 16, v.y & 0xffff0000u);
-        p[2] = pack2u(v.z << 16, v.z & 0xffff0000u);
-        p[3] = pack2u(v.w << 16, v.w & 0xffff0000u);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[8])
-    {
-        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]);
-        __nv_bfloat162 b = __floats2bfloat162_rn(f[2], f[3]);
-        __nv_bfloat162 c = __floats2bfloat162_rn(f[4], f[5]);
-        __nv_bfloat162 e = __floats2bfloat162_rn(f[6], f[7]);
-        uint4 v;
-        v.x = *reinterpret_cast<uint32_t *>(&a);
-        v.y = *reinterpret_cast<uint32_t *>(&b);
-        v.z = *reinterpret_cast<uint32_t *>(&c);
-        v.w = *reinterpret_cast<uint32_t *>(&e);
-        return v;
-    }
-    static __device__ __forceinline__ float scalar(const void *p, long long i)
-    {
-        return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p)[i]);
     }
     // element i of an array in shared memory (32-bit shared address)
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds16(base + 2 * i) << 16); }
@@ -276,24 +222,6 @@ struct Elem<float> {
         f[1] = __uint_as_float(v.y);
         f[2] = __uint_as_float(v.z);
         f[3] = __uint_as_float(v.w);
-    }
-    static __device__ __forceinline__ void unpack_pairs(const uint4 &v, f32x2 (&p)[2])
-    {
-        p[0] = pack2u(v.x, v.y);
-        p[1] = pack2u(v.z, v.w);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[4])
-    {
-        uint4 v;
-        v.x = __float_as_uint(f[0]);
-        v.y = __float_as_uint(f[1]);
-        v.z = __float_as_uint(f[2]);
-        v.w = __float_as_uint(f[3]);
-        return v;
-    }
-    static __device__ __forceinline__ float scalar(const void *p, long long i)
-    {
-        return reinterpret_cast<const float *>(p)[i];
     }
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds32(base + 4 * i)); }
     typedef float H;
