@@ -161,7 +161,7 @@ struct Sweep {
     static constexpr int NV = NFAST < VEC ? NFAST : VEC;        // accumulators per lane
     static constexpr int QL = NFAST >= VEC ? NFAST / VEC : 1;   // vectors per column
     static constexpr int CPV = NFAST >= VEC ? 1 : VEC / NFAST;  // columns per vector
-    static constexpr int UNR = 4;  // vectors in flight per lane (deeper batches grow the loop body; measured slower)
+    static constexpr int UNR = 16;  // vectors in flight per lane: a whole chunk for the widths of Table 2 (measured best)
     float acc[NV];
 
     __device__ __forceinline__ void clear()
@@ -253,7 +253,7 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     constexpr int GPW = 32 / P;   // column groups per warp
     constexpr int W = 4 / P;      // 32-bit words a lane finishes
     constexpr int VPW = VEC / 4;  // values per word: 2 (bf16) or 1 (fp32)
-    constexpr int UNR = 4;        // rows in flight per lane
+    constexpr int UNR = 16;       // rows in flight per lane: all N = 16 experts of a column group (measured best)
     const int part = lane / GPW, gl = lane % GPW;
     const int chunk = (N + P - 1) / P;
     const int jb = part * chunk, je = (jb + chunk < N) ? jb + chunk : N;
