@@ -273,18 +273,28 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
                 uint4 rv[UNR];
                 float gv[UNR];
 #pragma unroll
-                for (int r = 0; r < UNR; ++r) {
-                    rv[r] = lds128(rows + 16u * ((j0 + r) * ngrp + gg));
-                    gv[r] = __uint_as_float(lds32(gates + 4u * (j0 + r)));
+                for (int r = 0; r < UNR; ++r) rv[r] = lds128(rows + 16u * ((j0 + r) * ngrp + gg));
+                if ((j0 & 3) == 0) {  // the batch's softmax numerators: four per (broadcast) load when aligned
+#pragma unroll
+                    for (int r = 0; r < UNR; r += 4) {
+                        const uint4 g4 = lds128(gates + 4u * (j0 + r));
+                        gv[r] = __uint_as_float(g4.x), gv[r + 1] = __uint_as_float(g4.y);
+                        gv[r + 2] = __uint_as_float(g4.z), gv[r + 3] = __uint_as_float(g4.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < UNR; ++r) gv[r] = __uint_as_float(lds32(gates + 4u * (j0 + r)));
                 }
+                float es[4] = {0.f, 0.f, 0.f, 0.f};  // their sum, four short chains instead of one long one
 #pragma unroll
                 for (int r = 0; r < UNR; ++r) {
                     float vf[VEC];
                     E::unpack(rv[r], vf);
-                    esum += gv[r];
+                    es[r & 3] += gv[r];
 #pragma unroll
                     for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
                 }
+                esum += (es[0] + es[1]) + (es[2] + es[3]);
             }
 #pragma unroll 1
             for (; j0 < je; ++j0) {  // tail
