@@ -40,6 +40,8 @@ struct StepPlan {
     int smem;           // dynamic shared memory, bytes
     int blocks_per_sm;  // resident blocks per SM the shared memory allows
     int n_fast;         // N if the unrolled router path exists for it, else 0
+    int rows_by_expert; // several chunks per item: 1 = the rows are cut by experts, 0 = by columns
+    int lanes;          // combine: lanes per 16-byte column group (by columns) or column groups per lane (by experts)
 };
 int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan);
 

@@ -368,6 +368,113 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
     }
 }
 
+// The same weighted sum when an item's rows arrive cut by EXPERTS instead of by columns: chunk kk
+// holds the whole rows of experts kk*ne .. kk*ne + ne - 1, contiguous in the table, so that one bulk
+// copy brings it (a column chunk of several rows is N short pieces, which the copy engine moves at a
+// third of the rate).  A lane owns up to GPL column groups of 16 bytes (group = tid + i * nc) over
+// ALL d columns and carries their fp32 sums from chunk to chunk; after the last chunk it divides by
+// the sum of the numerators, adds the residual, rounds once and stores.
+template <typename T, int GPL>
+struct RowSums {
+    using E = Elem<T>;
+    static constexpr int VEC = E::VEC;
+    static constexpr int UNR = 8;  // experts in flight per column group
+    float acc[GPL][VEC];
+    float esum;
+
+    __device__ __forceinline__ void clear()
+    {
+#pragma unroll
+        for (int i = 0; i < GPL; ++i)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[i][e] = 0.f;
+        esum = 0.f;
+    }
+    // rows: the chunk [ne][d] in shared memory; gates: numerators of its first expert on
+    __device__ __forceinline__ void chunk(uint32_t rows, uint32_t gates, int ne, int ngrp, int tid, int nc)
+    {
+        int j0 = 0;
+#pragma unroll 1
+        for (; j0 + UNR <= ne; j0 += UNR) {  // full batches: all loads first
+            uint4 rv[GPL][UNR];
+            float gv[UNR];
+#pragma unroll
+            for (int i = 0; i < GPL; ++i) {
+                const int g = tid + i * nc;
+                const int gg = g < ngrp ? g : ngrp - 1;
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) rv[i][r] = lds128(rows + 16u * ((j0 + r) * ngrp + gg));
+            }
+#pragma unroll
+            for (int r = 0; r < UNR; r += 4) {  // UNR and every chunk's first expert are multiples of four here
+                const uint4 g4 = lds128(gates + 4u * (j0 + r));
+                gv[r] = __uint_as_float(g4.x), gv[r + 1] = __uint_as_float(g4.y);
+                gv[r + 2] = __uint_as_float(g4.z), gv[r + 3] = __uint_as_float(g4.w);
+            }
+            float es[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < UNR; ++r) es[r & 3] += gv[r];
+            esum += (es[0] + es[1]) + (es[2] + es[3]);
+#pragma unroll
+            for (int i = 0; i < GPL; ++i)
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) {
+                    float vf[VEC];
+                    E::unpack(rv[i][r], vf);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[i][e] = fmaf(gv[r], vf[e], acc[i][e]);
+                }
+        }
+#pragma unroll 1
+        for (; j0 < ne; ++j0) {  // tail (and every chunk of fewer than UNR experts)
+            const float g = __uint_as_float(lds32(gates + 4u * j0));
+            esum += g;
+#pragma unroll
+            for (int i = 0; i < GPL; ++i) {
+                const int grp = tid + i * nc;
+                const int gg = grp < ngrp ? grp : ngrp - 1;
+                const uint4 rv = lds128(rows + 16u * (j0 * ngrp + gg));
+                float vf[VEC];
+                E::unpack(rv, vf);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[i][e] = fmaf(g, vf[e], acc[i][e]);
+            }
+        }
+    }
+    // residual from global memory (residual_g) or from the hidden state in shared memory (haddr);
+    // result to global memory (dst_g) or to the running hidden state in shared memory (dst_s)
+    __device__ __forceinline__ void finish(uint32_t haddr, const unsigned char *residual_g, unsigned char *dst_g, uint32_t dst_s,
+                                           int ngrp, bool valid, int tid, int nc)
+    {
+        constexpr int VPW = VEC / 4;
+        const float inv = __frcp_rn(esum);
+#pragma unroll
+        for (int i = 0; i < GPL; ++i) {
+            const int grp = tid + i * nc;
+            if (grp < ngrp) {
+                uint4 v = residual_g ? __ldcg(reinterpret_cast<const uint4 *>(residual_g) + grp) : lds128(haddr + 16u * grp);
+                if (valid) {
+                    uint32_t rw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        if constexpr (VPW == 2) {
+                            const float lo = fmaf(acc[i][2 * w], inv, __uint_as_float(rw[w] << 16));
+                            const float hi = fmaf(acc[i][2 * w + 1], inv, __uint_as_float(rw[w] & 0xffff0000u));
+                            const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+                            rw[w] = *reinterpret_cast<const uint32_t *>(&b);
+                        } else {
+                            rw[w] = __float_as_uint(fmaf(acc[i][w], inv, __uint_as_float(rw[w])));
+                        }
+                    }
+                    v = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+                }
+                if (dst_g) *(reinterpret_cast<uint4 *>(dst_g) + grp) = v;
+                else sts128(dst_s + 16u * grp, v);
+            }
+        }
+    }
+};
+
 // Cold paths, kept out of the consumers' loop body (its size shows in instruction-fetch stalls).
 __device__ __noinline__ void report_timeout(volatile int *dead, uint32_t *status)
 {
@@ -402,10 +509,11 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 }
 
 // T: storage type.  NFAST: compile-time N of the unrolled router (0 = any N <= 64, slower).
-// P: lanes that share one 16-byte column group in the combine.
+// P: lanes that share one 16-byte column group in the combine (MODE 3: column groups per lane).
 // MODE: the common launch shapes with their flags fixed at compile time (a smaller loop body:
 // measured 10 % faster), 0 = any: 1 = router chunks in the ring, one chunk per item; 2 = router
-// resident, one chunk per item; 3 = router chunks in the ring, several chunks per item.
+// resident, one chunk per item; 3 = router chunks in the ring, several chunks per item, the rows
+// cut by experts (K divides N) instead of by columns.
 // SHAPE: the layer widths of the paper's Table 2 with d, the chunk width and the number of compute
 // threads as constants (0 = any): 1: d = 768; 2: d = 1024; 3: d = 2048 in chunks of 512.
 template <int SHAPE>
@@ -429,6 +537,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
     const int dcc = SHAPE ? ShapeOf<SHAPE>::dcc : p.dcc, d = SHAPE ? ShapeOf<SHAPE>::d : p.d;
     const int nc = SHAPE ? ShapeOf<SHAPE>::consumers : p.consumers;
     const bool ring = MODE == 0 ? (p.wr_in_ring != 0) : (MODE != 2);  // router chunks travel through the ring
+    constexpr bool kRowsByExpert = MODE == 3;  // rows chunk kk = the whole rows of experts kk*N/K ..
     const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, ring, nc);
     const uint32_t slot_bytes = up128(m.chunk_bytes), hid_stride = up128(m.hid_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -511,7 +620,12 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 const int kk = ring ? q - K : q;
                 const unsigned char *src = static_cast<const unsigned char *>(p.lut) + static_cast<size_t>(l) * p.lut_stride +
                                            (static_cast<size_t>(valid ? row : 0) * N * d + static_cast<size_t>(kk) * dcc) * EB;
-                if (K == 1) {
+                if (kRowsByExpert) {
+                    // N / K whole rows, contiguous: the same number of bytes as a column chunk
+                    if (lane == 0)
+                        bulk_g2s(slot, src + (static_cast<size_t>(kk) * (N / K) * d - static_cast<size_t>(kk) * dcc) * EB,
+                                 m.chunk_bytes, full + st);
+                } else if (K == 1) {
                     if (lane == 0) bulk_g2s(slot, src, m.chunk_bytes, full + st);  // the N rows of an id are contiguous
                 } else {
                     const uint32_t piece = static_cast<uint32_t>(dcc) * EB;
@@ -672,19 +786,36 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 named_bar_sync(kBarGates, nc);
 
                 // ---- weighted sum of the rows, chunk by chunk (Eq. 8) ----
+                if constexpr (kRowsByExpert) {
+                    RowSums<T, P> sums;
+                    sums.clear();
+                    const int ne = N / K, ngrp_all = d / VEC;
+                    bool valid = true;
 #pragma unroll 1
-                for (int kk = 0; kk < K; ++kk) {
-                    if (ring || kk > 0) acquire(st, ph);
-                    {
-                        const bool valid = meta[st] != 0;
-                        const uint32_t off = kk * chunk_cols_bytes;
-                        const unsigned char *res_g =
-                            p.residual ? static_cast<const unsigned char *>(p.residual) + tbyte + off : nullptr;
-                        unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + tbyte + off : nullptr;
-                        combine_item<T, P>(smem_base + static_cast<uint32_t>(st) * slot_bytes, haddr + off, gates_s, res_g, dst,
-                                           hid_s + off, N, ngrp, valid, warp, lane, nwarps);
+                    for (int kk = 0; kk < K; ++kk) {
+                        acquire(st, ph);
+                        valid = meta[st] != 0;
+                        sums.chunk(smem_base + static_cast<uint32_t>(st) * slot_bytes, gates_s + 4u * (kk * ne), ne, ngrp_all, tid, nc);
+                        release();
                     }
-                    release();
+                    const unsigned char *res_g = p.residual ? static_cast<const unsigned char *>(p.residual) + tbyte : nullptr;
+                    unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + tbyte : nullptr;
+                    sums.finish(haddr, res_g, dst, hid_s, ngrp_all, valid, tid, nc);
+                } else {
+#pragma unroll 1
+                    for (int kk = 0; kk < K; ++kk) {
+                        if (ring || kk > 0) acquire(st, ph);
+                        {
+                            const bool valid = meta[st] != 0;
+                            const uint32_t off = kk * chunk_cols_bytes;
+                            const unsigned char *res_g =
+                                p.residual ? static_cast<const unsigned char *>(p.residual) + tbyte + off : nullptr;
+                            unsigned char *dst = (l == L - 1) ? static_cast<unsigned char *>(p.out) + tbyte + off : nullptr;
+                            combine_item<T, P>(smem_base + static_cast<uint32_t>(st) * slot_bytes, haddr + off, gates_s, res_g,
+                                               dst, hid_s + off, N, ngrp, valid, warp, lane, nwarps);
+                        }
+                        release();
+                    }
                 }
                 // the next layer's router reads the hidden state that all warps have just written
                 if (l + 1 < L) named_bar_sync(kBarHidden, nc);

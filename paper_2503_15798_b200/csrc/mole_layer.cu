@@ -42,6 +42,26 @@ static int consumers_for(int dcc, int vec)
     const int lanes = (dcc / vec) * lanes_per_group(dcc, vec);
     return round_up(lanes < kMaxConsumers ? lanes : kMaxConsumers, 32);
 }
+// Several chunks per item: the rows are cut by experts -- whole rows, one bulk copy per chunk --
+// where the kernel exists for it (bf16, a compiled-in N that the chunk count divides, router
+// chunks in the ring) and a lane can carry the sums of its column groups (at most four, over
+// about four warps) from chunk to chunk; otherwise by columns.
+static int groups_per_lane(int d, int vec)
+{
+    const int groups = d / vec;
+    return groups <= 128 ? 1 : (groups <= 256 ? 2 : 4);
+}
+static bool rows_by_expert(int dtype, int N, int d, int K, int in_ring)
+{
+    const bool n_fast = N == 4 || N == 8 || N == 16 || N == 32 || N == 64;
+    if (env_int("MOLE_FORCE_COLUMN_CHUNKS") > 0) return false;  // debugging aid
+    return dtype == MOLE_DTYPE_BF16 && n_fast && K > 1 && N % K == 0 && in_ring && d / 8 <= 4 * 128;
+}
+static int consumers_by_expert(int d, int vec)
+{
+    const int gpl = groups_per_lane(d, vec);
+    return round_up((d / vec + gpl - 1) / gpl, 32);
+}
 static int env_int(const char *name)  // debugging aids: MOLE_FORCE_* override parts of the plan
 {
     const char *f = getenv(name);
@@ -60,7 +80,8 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     auto total_smem = [&](int K, int stages) {
         const int dcc = d / K;
         const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
-        return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers_for(dcc, vec)).total;
+        const int consumers = rows_by_expert(dtype, N, d, K, in_ring) ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
+        return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers).total;
     };
     int K;
     if (d_split != 0) {
@@ -80,7 +101,8 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
         }
     }
     const int dcc = d / K;
-    const int consumers = consumers_for(dcc, vec);
+    const bool by_expert = rows_by_expert(dtype, N, d, K, in_ring);
+    const int consumers = by_expert ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
     // Resident blocks per SM aimed at: one per token while tokens are few (each with the deepest ring
     // that fits), up to four token chains per SM when there are many (shallower rings, more overlap).
     int want = static_cast<int>((M + kNumSMs - 1) / kNumSMs);
@@ -119,6 +141,8 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     if (per_sm > 32) per_sm = 32;
     if (per_sm < 1) per_sm = 1;
     plan->blocks_per_sm = per_sm;
+    plan->rows_by_expert = by_expert ? 1 : 0;
+    plan->lanes = by_expert ? groups_per_lane(d, vec) : lanes_per_group(dcc, vec);
     plan->n_fast = (N == 4 || N == 8 || N == 16 || N == 32 || N == 64) ? N : 0;
     return MOLE_OK;
 }
@@ -146,7 +170,8 @@ static StepKernel pick_p(int n_fast, int lanes)
 
 // The generic-N router and the fp32 storage type exist only with run-time flags (MODE 0); bf16 with
 // a compiled-in N also in the three specialised shapes.
-static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers)
+static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers,
+                              int by_expert)
 {
     // the layer widths of the paper's Table 2 (160M, 410M and 1B models) with their sizes compiled in
     if (dtype == MOLE_DTYPE_BF16) {
@@ -154,8 +179,9 @@ static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int 
             return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1>;
         if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 1024 && consumers == 128)
             return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 2> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2>;
-        if (n_fast == 32 && lanes == 2 && chunks == 4 && d == 2048 && dcc == 512 && consumers == 128 && in_ring)
+        if (n_fast == 32 && lanes == 2 && chunks == 4 && d == 2048 && dcc == 512 && consumers == 128 && by_expert)
             return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 3>;
+        if (by_expert) return pick_p<__nv_bfloat16, 3>(n_fast, lanes);
     }
     if (n_fast == 0) {
         if (dtype == MOLE_DTYPE_BF16)
@@ -164,7 +190,7 @@ static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int 
     }
     if (dtype != MOLE_DTYPE_BF16) return pick_p<float, 0>(n_fast, lanes);
     if (chunks == 1) return in_ring ? pick_p<__nv_bfloat16, 1>(n_fast, lanes) : pick_p<__nv_bfloat16, 2>(n_fast, lanes);
-    return in_ring ? pick_p<__nv_bfloat16, 3>(n_fast, lanes) : pick_p<__nv_bfloat16, 0>(n_fast, lanes);
+    return pick_p<__nv_bfloat16, 0>(n_fast, lanes);
 }
 
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
@@ -227,8 +253,8 @@ int launch_step(const StepLaunch &a)
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast, lanes_per_group(plan.dc, 16 / elem_bytes(a.dtype)), plan.d_split, plan.wr_in_ring,
-                               a.d, plan.dc, plan.consumers);
+    StepKernel k = pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
+                               plan.rows_by_expert);
     if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;

@@ -1,5 +1,7 @@
 """GPU parity: the fused sm_100a layer, through the C ABI, against the fp64 CPU oracle on the
 same seeded inputs, element by element."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -288,6 +290,28 @@ def test_maximum_sizes_N64_and_wide_d():
     check_gates(gates, gref)
 
 
+@pytest.mark.parametrize("M,N,d,split", [(37, 64, 1024, 4), (37, 64, 1024, 16), (21, 64, 4096, 8), (21, 64, 4096, 16),
+                                         (70, 32, 2048, 2), (301, 32, 2048, 4)])
+def test_rows_cut_by_experts_single_layer(M, N, d, split):
+    """Router matrices too large to stay resident travel through the ring; with several chunks per
+    item the rows then arrive as whole rows of N / split experts: one, two and four column groups
+    per lane, chunks of more and of fewer experts than one load batch."""
+    hidden, ids, lut, wr = rand_case(M, N, d, 50, seed=M + N + split)
+    ref, gref, _ = oracle_layer(hidden, ids, lut, wr)
+    out, gates, status = run_gpu(hidden, ids, lut, wr, d_split=split)
+    assert status == 0
+    check_out(out, ref)
+    check_gates(gates, gref)
+    os.environ["MOLE_FORCE_COLUMN_CHUNKS"] = "1"  # the same launch with the rows cut by columns
+    try:
+        out2, gates2, status2 = run_gpu(hidden, ids, lut, wr, d_split=split)
+    finally:
+        del os.environ["MOLE_FORCE_COLUMN_CHUNKS"]
+    assert status2 == 0
+    check_out(out2, ref)
+    check_gates(gates2, gref)
+
+
 # ---- chained layers ------------------------------------------------------------------------------
 
 def _step_case(M, N, d, L, V=400):
@@ -317,7 +341,24 @@ def test_decode_step_fused_and_chained_equal_layer_after_layer(M, N, d, L, split
         check_out(h, ref)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    assert torch.equal(fused, h) and torch.equal(chained, h)  # same split => same bits
+    assert torch.equal(chained, h)  # one launch per layer, chained or not: the same bits
+    # The fused launch sums an item's experts in the same order as the single layers when the rows
+    # arrive cut by columns (always with one chunk); cut by experts (several chunks, bf16, K | N) the
+    # order of the fp32 sum differs, and with it now and then a rounding decision.
+    os.environ["MOLE_FORCE_COLUMN_CHUNKS"] = "1"
+    try:
+        by_columns = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), None, status=status,
+                                      mode=mole.STEP_FUSED, d_split=split)
+        torch.cuda.synchronize()
+    finally:
+        del os.environ["MOLE_FORCE_COLUMN_CHUNKS"]
+    assert torch.equal(by_columns, h)
+    if split == 1:
+        assert torch.equal(fused, h)
+    else:
+        err = np.abs(as_f64(fused) - as_f64(h))
+        assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(as_f64(h)))).all(), float(err.max())
+    assert int(status.item()) == 0
     assert torch.equal(hidden, keep)  # the input is never written
 
 
