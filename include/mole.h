@@ -118,9 +118,13 @@ typedef struct mole_args {
     int32_t B, T, N, d, V;
     int32_t dtype;         /* MOLE_DTYPE_* */
     int32_t reserved;      /* must be 0 */
-    int32_t d_split;       /* column chunks a token's rows are streamed in (1, 2, 4, 8 or 16; d/d_split must stay a
-                              multiple of the vector width); 0 = auto: the fewest chunks of at most 32 KB.  The
-                              chunking fixes the order of the fp32 sums: equal d_split, bit-identical results. */
+    int32_t d_split;       /* chunks a token's router matrix and rows are streamed in (1, 2, 4, 8 or 16; d/d_split must
+                              stay a multiple of the vector width); 0 = auto: the fewest chunks of at most 32 KB.
+                              The router matrix is cut by columns.  The rows are cut by experts (whole rows of
+                              N/d_split experts, one contiguous copy) when d_split > 1 divides N, N is 4, 8, 16, 32
+                              or 64, dtype is bf16, d <= 4096 and the router matrix streams with them (several
+                              layers in one launch, or a matrix above 96 KB); otherwise by columns.  Chunking and
+                              cut fix the order of the fp32 sums: the same launch shape gives the same bits. */
     void *stream;          /* cudaStream_t */
 } mole_args;
 
@@ -137,7 +141,9 @@ MOLE_API int mole_layer_forward_ex(const mole_args *args);
  *             or when the mode is MOLE_STEP_FUSED)
  * dtype as MOLE_DTYPE_*.  status (device, may be NULL) as in mole_args.
  *
- * Two ways to run it, with bit-identical results for equal d_split:
+ * Two ways to run it (bit-identical when the rows travel in one chunk; with several chunks the two
+ * may cut the rows differently -- see d_split -- and differ in the order of the fp32 sums, i.e. now
+ * and then in a rounding decision):
  *  - FUSED: tokens are independent and a token's chain h_0 -> h_1 -> ... -> h_L needs nothing
  *    but its own rows, so one launch lets each block keep a token's running hidden slice in
  *    shared memory across all L layers while the rows of later layers (which depend only on

@@ -13,7 +13,9 @@
 // needs is pulled through a ring of shared-memory slots, one chunk per slot, by bulk
 // asynchronous copies (TMA engine, untiled, no multicast) that one extra "producer" warp issues
 // `stages` chunks ahead: first (when L > 1) the K chunks [dcc][N] of the layer's router matrix,
-// then the K chunks [N][dcc] of the token's table rows.  The rows depend only on the id, so they
+// then the K chunks of the token's table rows -- [N][dcc], N short pieces per chunk, or, where K
+// divides N (MODE 3), the whole rows [N/K][d] of N/K experts in one contiguous copy, which the
+// copy engine moves three times as fast.  The rows depend only on the id, so they
 // run ahead of the arithmetic and, in a chained launch, ahead of the previous kernel.  The
 // token's hidden state arrives with its first chunk in a small ring of its own.  Completion is
 // counted on one mbarrier per slot ("full"); the consumer warps hand a slot back through a
