@@ -20,6 +20,7 @@ With N > 1 (torchrun) every rank holds its own replica of the tables and its own
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -54,6 +55,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-batch sweep and the isolated-launch rows")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--layers", type=int, default=0, help="override L (debugging; the line then says so)")
+    ap.add_argument("--vocab", type=int, default=0,
+                    help="override V, the number of table rows (small profiler captures; the line then says so)")
     ap.add_argument("--offload", action="store_true",
                     help="offload mode instead: table in pinned host memory, per-step dedup + row fetch overlapped with "
                          "the previous layer's combine; roofline = measured host-link GB/s")
@@ -306,6 +309,8 @@ def run_mole(args):
     mole.lib()  # fails loudly if the library is missing
     dev = torch.device("cuda", local_rank)
     sh = inputs.SHAPES[args.config]
+    if args.vocab > 0:
+        sh = dataclasses.replace(sh, V=args.vocab)
     L = args.layers or sh.L
     M = args.batch
     peak, peak_src = measured_peak()
