@@ -10,7 +10,8 @@ residual), chained with programmatic dependent launch and replayed from a CUDA g
 metric is tokens/s for the L-layer step; the roofline block reports the layer kernel's
 algorithmic GB/s (gathered rows + hidden in/out + router weights) against the measured HBM
 copy bandwidth.  Every step uses a different pre-generated Zipf(1.1) id batch, and the table
-(GBs) is far larger than L2.
+(GBs) is far larger than L2.  Beside it, as an extra ("fused_step"), the same step as a single
+launch that walks every token through all L layers on chip.
 
 With N > 1 (torchrun) every rank holds its own replica of the tables and its own batches
 (tokens are independent, so there is no collective on the data path): weak scaling.
@@ -39,6 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
 TRAFFIC = {
+}
+# the same for the fused all-layers launch reported as an extra
+FUSED_TRAFFIC = {
     # profiles/mole_step_kernel_160m_batch256.md: 7.59 MB per 2-layer launch, x6 for the 12 layers of a full launch
     ("160m", 256, 12): 45.5e6,
 }
@@ -331,10 +335,12 @@ def run_mole(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- headline: K steps of the L-layer decode step, as mole_decode_step runs it ------------------------
+    # ---- headline: K steps of the L-layer decode step as a model that runs other work between the layers
+    # gets it: one launch per layer, chained with programmatic dependent launch, the layer's output the next
+    # layer's hidden state, the L launches of a step replayed from a CUDA graph -----------------------------
     hidden = hidden_all[:M].contiguous()
-    fused = not (L > 1 and M > 4096)  # mole_decode_step's own choice: one fused launch up to 4096 tokens
-    graphs = StepGraphs(mole, luts, wrs, hidden, batches_for(M))
+    fused = False
+    graphs = StepGraphs(mole, luts, wrs, hidden, batches_for(M), mode=mole.STEP_CHAINED)
     graphs.run(0, max(args.warmup, 3))
     barrier()
     with ClockSampler(physical_gpu_index(local_rank)) as clocks:
@@ -356,10 +362,28 @@ def run_mole(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": TRAFFIC.get((sh.name, M, L)), "kernel": "mole_step_kernel", "peak_source": peak_src,
-                     "launch": ("one fused launch per step (all %d layers)" % L) if fused else "one launch per layer, chained",
+                     "launch": "one launch per layer (%d per step), chained with programmatic dependent launch" % L,
                      "algorithmic_bytes_per_launch": launch_bytes, "us_per_launch": ms * 1e3 / launches},
         "clocks": clocks.summary(),
     }
+
+    # ---- extra, never the headline: the same step as ONE launch that keeps a token's chain through all L
+    # layers on chip (what mole_decode_step picks by itself up to 4096 tokens) ------------------------------
+    del graphs
+    if L > 1 and M <= 4096:
+        g = StepGraphs(mole, luts, wrs, hidden, batches_for(M), mode=mole.STEP_FUSED)
+        g.run(0, max(args.warmup, 3))
+        barrier()
+        ms_f = max_over_ranks(timed_ms(torch, lambda: g.run(0, args.steps)), dist, dev)
+        barrier()
+        assert int(g.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
+        fb = sh.step_bytes(M, L)
+        gbs = fb / (ms_f * 1e-3 / args.steps) / 1e9
+        line["fused_step"] = {"what": "all %d layers of a step in one launch (layer-batched), an extra beside the headline" % L,
+                              "value": whole_job_tokens_per_s(world, M, args.steps, ms_f), "unit": UNIT,
+                              "us_per_step": ms_f * 1e3 / args.steps, "algorithmic_bytes_per_launch": fb,
+                              "achieved": gbs, "frac": gbs / peak, "traffic": FUSED_TRAFFIC.get((sh.name, M, L))}
+        del g
 
     # ---- end to end: host buffers in, host buffer out, through the C ABI, every step ---------------------
     h_host = hidden.cpu().pin_memory()
