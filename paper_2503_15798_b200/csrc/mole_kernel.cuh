@@ -16,8 +16,9 @@
 // then the K chunks of the token's table rows -- [N][dcc], N short pieces per chunk, or, where K
 // divides N (MODE 3), the whole rows [N/K][d] of N/K experts in one contiguous copy, which the
 // copy engine moves three times as fast.  The rows depend only on the id, so they
-// run ahead of the arithmetic and, in a chained launch, ahead of the previous kernel.  The
-// token's hidden state arrives with its first chunk in a small ring of its own.  Completion is
+// run ahead of the arithmetic and, in a chained launch, ahead of the previous kernel.  A
+// token's hidden state arrives with its first chunk in a small ring of its own (the block's first
+// token excepted: the compute warps load it themselves).  Completion is
 // counted on one mbarrier per slot ("full"); the consumer warps hand a slot back through a
 // second one ("empty").  With L == 1 the router matrix is loaded once per block instead.
 //
@@ -518,13 +519,16 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 // cut by experts (K divides N) instead of by columns.
 // SHAPE: the layer widths of the paper's Table 2 with d, the chunk width and the number of compute
 // threads as constants (0 = any): 1: d = 768; 2: d = 1024; 3: d = 2048 in chunks of 512.
+// DIRECT: the compute warps load the hidden state of the block's first token themselves, with plain
+// 16-byte loads, instead of waiting for the producer's bulk copy (a variant of its own because any
+// growth of the loop body costs the other launches 2 - 6 %).
 template <int SHAPE>
 struct ShapeOf {
     static constexpr int d = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 2048);
     static constexpr int dcc = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 512);
     static constexpr int consumers = SHAPE == 1 ? 96 : 128;
 };
-template <typename T, int NFAST, int P, int MODE, int SHAPE>
+template <typename T, int NFAST, int P, int MODE, int SHAPE, int DIRECT = 0>
 __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const StepParams p)
 {
     using E = Elem<T>;
@@ -584,7 +588,10 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             bulk_g2s(smem + m.off_hring + static_cast<size_t>(entry) * hid_stride,
                      static_cast<const unsigned char *>(p.hidden) + static_cast<size_t>(t) * d * EB, m.hid_bytes, full + st);
         };
-        // Issue the next chunk; the hidden state (first chunk of a token) only if with_hidden.
+        // Issue the next chunk; the hidden state (first chunk of a token) only if with_hidden.  With
+        // DIRECT the block's first token is the exception: the compute warps fetch its hidden state
+        // themselves.
+        constexpr int k_first_copied = DIRECT ? 1 : 0;
         auto issue = [&](long long ci, bool with_hidden) {
             if (l == 0 && q == 0) {
                 if ((k & 31) == 0) {  // ids of the next 32 tokens of this block, one per lane
@@ -605,7 +612,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
             if (lane == 0) {
                 meta[st] = valid ? 1 : 0;
                 if (!valid && first && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
-                mbar_expect_tx(full + st, m.chunk_bytes + (first ? m.hid_bytes : 0u));
+                mbar_expect_tx(full + st, m.chunk_bytes + (first && k >= k_first_copied ? m.hid_bytes : 0u));
                 *issued = static_cast<int>(ci + 1 < 0x7fffffff ? ci + 1 : 0x7fffffff);
             }
             __syncwarp();
@@ -635,7 +642,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                         bulk_g2s(slot + static_cast<size_t>(j) * piece, src + static_cast<size_t>(j) * d * EB, piece, full + st);
                 }
             }
-            if (with_hidden && first && lane == 31) hidden_copy(k, he, st);
+            if (with_hidden && first && k >= k_first_copied && lane == 31) hidden_copy(k, he, st);
             if (++q == cpi) {
                 q = 0;
                 if (++l == L) {
@@ -658,7 +665,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         fence_proxy_async_global();
         if (lane == 31) {
             const int per_tok = L * cpi;  // chunk tok*per_tok is the first chunk of token tok
-            for (int tok = 0; static_cast<long long>(tok) * per_tok < pre; ++tok)
+            for (int tok = k_first_copied; static_cast<long long>(tok) * per_tok < pre; ++tok)
                 hidden_copy(tok, tok % HR, static_cast<int>((static_cast<long long>(tok) * per_tok) % stages));
         }
         for (long long ci = pre; ci < total; ++ci) {
@@ -686,6 +693,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         // memory and the block's own rows of `out` -- so that no other warp is left at a barrier; the
         // status word says that the outputs are meaningless.
         bool alive = true;
+        constexpr bool direct = DIRECT != 0;
 
         auto give_up = [&]() {
             if (lane == 0) report_timeout(dead, p.status);
@@ -723,6 +731,15 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 // the item's hidden state: as loaded (first layer) or as left by the previous layer
                 const uint32_t haddr = (l == 0) ? smem_base + m.off_hring + static_cast<uint32_t>(he) * hid_stride : hid_s;
 
+                if (k == 0 && l == 0 && direct) {
+                    // first token of the block: plain 16-byte loads straight after the grid dependency
+                    // (measured faster than the bulk copy for chained one-token blocks once a launch has
+                    // more than about a hundred of them, slower below)
+                    const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const unsigned char *>(p.hidden) + tbyte);
+                    for (int g = tid; g < d / VEC; g += nc) sts128(haddr + 16u * g, __ldcg(src + g));
+                    named_bar_sync(kBarHidden, nc);
+                }
+
                 // ---- router: partial logits over all d columns ----
                 sweep.clear();
                 if (ring) {
@@ -737,7 +754,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                         release();
                     }
                 } else {
-                    acquire(st, ph);  // the first rows chunk brings the hidden state with it
+                    if (k > 0 || !direct) acquire(st, ph);  // the first rows chunk brings the hidden state with it
                     {
                         if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, haddr, d, tid, nc);
                         else sweep.chunk_any(smem_base + m.off_wr, haddr, d, N, warp, lane, nwarps, true, partial);
@@ -806,7 +823,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 } else {
 #pragma unroll 1
                     for (int kk = 0; kk < K; ++kk) {
-                        if (ring || kk > 0) acquire(st, ph);
+                        if (ring || kk > 0 || direct) acquire(st, ph);
                         {
                             const bool valid = meta[st] != 0;
                             const uint32_t off = kk * chunk_cols_bytes;

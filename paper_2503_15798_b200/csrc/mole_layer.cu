@@ -171,14 +171,18 @@ static StepKernel pick_p(int n_fast, int lanes)
 // The generic-N router and the fp32 storage type exist only with run-time flags (MODE 0); bf16 with
 // a compiled-in N also in the three specialised shapes.
 static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers,
-                              int by_expert)
+                              int by_expert, bool direct)
 {
-    // the layer widths of the paper's Table 2 (160M, 410M and 1B models) with their sizes compiled in
+    // the layer widths of the paper's Table 2 (160M, 410M and 1B models) with their sizes compiled in;
+    // `direct`: single-layer launches of 128 tokens up to one token per resident block, where the compute
+    // warps loading the hidden state themselves measured 6 % faster per chained layer (slower below)
     if (dtype == MOLE_DTYPE_BF16) {
         if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 768 && consumers == 96)
-            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1>;
+            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 1>
+                           : (direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1>);
         if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 1024 && consumers == 128)
-            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 2> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2>;
+            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 2>
+                           : (direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2>);
         if (n_fast == 32 && lanes == 2 && chunks == 4 && d == 2048 && dcc == 512 && consumers == 128 && by_expert)
             return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 3>;
         if (by_expert) return pick_p<__nv_bfloat16, 3>(n_fast, lanes);
@@ -254,7 +258,7 @@ int launch_step(const StepLaunch &a)
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
     StepKernel k = pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
-                               plan.rows_by_expert);
+                               plan.rows_by_expert, a.M >= 128 && a.M <= 4LL * sms);
     if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
