@@ -40,10 +40,12 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
 TRAFFIC = {
+    # profiles/mole_step_kernel_single_layer_160m_batch256.md: mean of three captured launches (one layer each)
+    ("160m", 256, 12): 4.43e6,
 }
 # the same for the fused all-layers launch reported as an extra
 FUSED_TRAFFIC = {
-    # profiles/mole_step_kernel_160m_batch256.md: 7.59 MB per 2-layer launch, x6 for the 12 layers of a full launch
+    # profiles/mole_step_kernel_fused_160m_batch256.md: 7.59 MB per 2-layer launch, x6 for the 12 layers of a full launch
     ("160m", 256, 12): 45.5e6,
 }
 
