@@ -559,12 +559,28 @@ def run_offload(args):
         ms = timed_ms(torch, lambda: [step(k) for k in range(steps)])
         torch.cuda.synchronize()
         assert int(status.item()) == 0
+        us_calls = ms * 1e3 / steps
+        # the same steps replayed from CUDA graphs (one per id batch; the side stream joins the capture):
+        # at small batches the 2L+1 launches of a step are otherwise bound by the host's launch rate
+        graphs = []
+        for k in range(N_BATCHES):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step(k)
+            graphs.append(g)
+        for k in range(max(args.warmup, 3)):
+            graphs[k % N_BATCHES].replay()
+        torch.cuda.synchronize()
+        ms = timed_ms(torch, lambda: [graphs[k % N_BATCHES].replay() for k in range(steps)])
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        del graphs
         us_step = ms * 1e3 / steps
         link_bytes = uniq_rows * row_bytes * L  # distinct rows only cross the link
         rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                      "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                      "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 1 + 2 * L})
+                     "launches_per_step": 1 + 2 * L, "us_per_step_without_graph": us_calls})
         ctx.destroy()
     top = rows[-1]
     line = {
@@ -575,7 +591,7 @@ def run_offload(args):
         "config": {"workload": f"{sh.name}-shaped offload decode: table {sh.layer_table_bytes * L / 1e9:.2f} GB in pinned host "
                                f"memory, L={L}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
                    "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": 64,
-                   "l2": "rows come from host memory; 32 rotating id batches"},
+                   "l2": "rows come from host memory; 32 rotating id batches, one CUDA graph per batch"},
         "gpu_launches": (1 + 2 * L) * max(20, min(args.steps, 400)),
         "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": link_fetch, "unit": "GB/s",
                      "frac": top["frac_of_link"], "traffic": None, "kernel": "mole_fetch_kernel",

@@ -279,6 +279,11 @@ MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const vo
  *   table, layer l at + l*lut_layer_stride_bytes;  w_router_base device, layer l at
  *   + l*wr_layer_stride_bytes.
  * Output is bit-identical to L calls of mole_layer_forward.  stream and side_stream must differ.
+ * The call may be captured into a CUDA graph (stream capturing, side_stream an ordinary stream: it
+ * joins the capture and is joined back before the call returns).  While capturing, the call does not
+ * wait for the events of the previous call on the same context -- a captured stream may not depend on
+ * work outside the capture -- so the graphs of one context must be launched into one stream (or
+ * otherwise ordered), and the context should not go back to uncaptured calls afterwards.
  */
 MOLE_API int mole_offload_decode_step(mole_offload_ctx *ctx, const void *hidden_in, const int32_t *ids,
                              const void *lut_host_base, int64_t lut_layer_stride_bytes, const void *w_router_base,

@@ -348,8 +348,15 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
     // after the previous step's layers have stopped reading the slot map and both staging areas
     MOLE_CUDA_TRY(cudaEventRecord(c->step_begin, st));
     MOLE_CUDA_TRY(cudaStreamWaitEvent(side, c->step_begin, 0));
-    MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B0.consumed, 0));
-    MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B1.consumed, 0));
+    // While `stream` is being captured into a CUDA graph the waits on the previous call's events are
+    // left out (a captured stream may not depend on work outside the capture): the step then relies
+    // on the stream order of whole graph launches, which step_begin already carries to the side stream.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    MOLE_CUDA_TRY(cudaStreamIsCapturing(st, &capturing));
+    if (capturing == cudaStreamCaptureStatusNone) {
+        MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B0.consumed, 0));
+        MOLE_CUDA_TRY(cudaStreamWaitEvent(side, B1.consumed, 0));
+    }
     // one dedup for the whole step: every layer looks up the same ids (slot map and distinct ids in buffer 0)
     int rc = launch_dedup(ids, static_cast<int>(M), c->V, c->table, B0.uniq, B0.slot, B0.count, status, side);
     if (rc != MOLE_OK) return rc;

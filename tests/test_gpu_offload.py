@@ -228,3 +228,43 @@ def test_offload_decode_step_equals_resident_layers(M, L):
     finally:
         ctx.destroy()
         host.free()
+
+
+def test_offload_decode_step_replayed_from_cuda_graphs():
+    """The offload step captured into CUDA graphs (the side stream joins the capture and is joined
+    back): replays, with other steps' replays in between, give the bytes of the uncaptured call."""
+    M, L, N, d, V = 24, 5, 16, 768, 500
+    g = torch.Generator().manual_seed(77)
+    host = mole.HostTable((L, V, N, d), torch.bfloat16)
+    ctx = mole.OffloadContext(max_tokens=M, N=N, d=d, V=V, n_buffers=2)
+    side = torch.cuda.Stream()
+    try:
+        host.tensor.copy_(torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16))
+        wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
+        hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        out, tmp = torch.empty_like(hidden), torch.empty_like(hidden)
+        batches = [torch.from_numpy(inputs.zipf_ids(M, V, seed=40 + b)).to(DEV) for b in range(3)]
+        want = []
+        for ids in batches:  # uncaptured calls first (they also set the kernels' attributes)
+            ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, status=status, side_stream=side)
+            torch.cuda.synchronize()
+            want.append(out.clone())
+        graphs = []
+        for ids in batches:
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, status=status, side_stream=side)
+            graphs.append(gr)
+        for k in (0, 1, 2, 1, 0, 2, 2):
+            out.zero_()
+            graphs[k].replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, want[k])
+        for k in range(30):  # back to back, no synchronisation in between
+            graphs[k % 3].replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, want[29 % 3]) and int(status.item()) == 0
+    finally:
+        ctx.destroy()
+        host.free()
