@@ -46,7 +46,7 @@
 extern "C" {
 #endif
 
-#define MOLE_VERSION 200
+#define MOLE_VERSION 210
 
 /* every entry point is exported from the shared library with default visibility */
 #if defined(__GNUC__)
@@ -101,8 +101,9 @@ MOLE_API int mole_layer_forward(const void *hidden, const int32_t *ids, const vo
 
 /*
  * mole_layer_forward_ex -- the same operation with every option.  The appendix listing of
- * the paper routes on the normalised hidden state but adds the un-normalised residual plus
- * the shared expert's output; `residual` lets a caller do exactly that.
+ * the paper (App. A.2) routes on the normalised hidden state but adds the un-normalised residual
+ * plus the shared expert's output: `norm_weight` fuses that normalisation in front of the router,
+ * `residual` takes (residual + shared expert output).
  */
 typedef struct mole_args {
     uint32_t struct_size;  /* sizeof(mole_args), checked */
@@ -126,6 +127,13 @@ typedef struct mole_args {
                               layers in one launch, or a matrix above 96 KB); otherwise by columns.  Chunking and
                               cut fix the order of the fp32 sums: the same launch shape gives the same bits. */
     void *stream;          /* cudaStream_t */
+    const void *norm_weight; /* device [d], dtype, or NULL.  Not NULL: the router reads RMSNorm(hidden) =
+                              (hidden / sqrt(mean(hidden^2) + norm_eps)) * norm_weight, rounded once to dtype, while
+                              the residual stays `residual` (or hidden itself) -- the decoder layer of the paper's
+                              App. A.2 listing, whose router input is the normalised state and whose residual is
+                              not.  The normalisation happens in shared memory inside the same kernel. */
+    float norm_eps;        /* >= 0; read only with norm_weight */
+    int32_t reserved2;     /* must be 0 */
 } mole_args;
 
 MOLE_API int mole_layer_forward_ex(const mole_args *args);

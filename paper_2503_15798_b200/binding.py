@@ -40,6 +40,7 @@ class MoleArgs(ctypes.Structure):
         ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
         ("dtype", c_int32), ("reserved", c_int32), ("d_split", c_int32),
         ("stream", c_void_p),
+        ("norm_weight", c_void_p), ("norm_eps", ctypes.c_float), ("reserved2", c_int32),
     ]
 
 
@@ -131,9 +132,11 @@ def _dev(t: torch.Tensor, name: str):
 
 
 def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_out=None, status=None,
-                  d_split: int = 0, chain: bool = False, stream=None, B=None, T=None):
+                  d_split: int = 0, chain: bool = False, stream=None, B=None, T=None, norm_weight=None,
+                  norm_eps: float = 1e-6):
     """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d],
-    w_router [d][N]; returns out (allocated like hidden if not given)."""
+    w_router [d][N]; returns out (allocated like hidden if not given).  norm_weight [d]: the router
+    reads RMSNorm(hidden) with that scale and norm_eps, the residual stays un-normalised."""
     for name, t in (("hidden", hidden), ("ids", ids), ("lut", lut), ("w_router", w_router)):
         _dev(t, name)
     V, N, d = lut.shape
@@ -163,6 +166,11 @@ def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_
     a.B, a.T, a.N, a.d, a.V = B, T, N, d, V
     a.dtype, a.reserved, a.d_split = tag, 0, d_split
     a.stream = _stream(stream)
+    if norm_weight is not None:
+        _dev(norm_weight, "norm_weight")
+        if norm_weight.dtype != hidden.dtype or norm_weight.numel() != d:
+            raise ValueError("norm_weight must be [d] of the element type of hidden")
+    a.norm_weight, a.norm_eps, a.reserved2 = _ptr(norm_weight), float(norm_eps), 0
     _check(lib().mole_layer_forward_ex(ctypes.byref(a)), "mole_layer_forward_ex")
     return out
 

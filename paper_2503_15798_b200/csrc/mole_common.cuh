@@ -43,7 +43,8 @@ struct StepPlan {
     int rows_by_expert; // several chunks per item: 1 = the rows are cut by experts, 0 = by columns
     int lanes;          // combine: lanes per 16-byte column group (by columns) or column groups per lane (by experts)
 };
-int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan);
+// `by_columns`: never cut the rows by experts (kernel variants that exist for the column cut only)
+int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns = false);
 
 // One launch of the fused kernel over L chained layers (L == 1: a single layer).
 // `row_index` is ids (resident mode) or slot (offload mode); `rows` the number of table rows
@@ -61,6 +62,8 @@ struct StepLaunch {
     uint32_t flags;
     int d_split;
     cudaStream_t stream;
+    const void *norm_weight = nullptr;  // [d], dtype: the router reads RMSNorm(hidden) (single layer only); NULL: hidden
+    float norm_eps = 0.f;
 };
 int launch_step(const StepLaunch &a);
 

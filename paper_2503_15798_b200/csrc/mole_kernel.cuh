@@ -47,6 +47,8 @@ constexpr uint32_t kDrainPolls = 1u << 14;  // after a failure: short waits for 
 
 struct StepParams {
     const void *hidden, *residual, *row_index, *lut, *w_router;
+    const void *norm_weight;  // [d] scale of the RMSNorm in front of the router (NORM kernels), else unused
+    float norm_eps;
     void *out;
     float *gates_out;
     uint32_t *status;
@@ -478,6 +480,52 @@ struct RowSums {
     }
 };
 
+// The normalisation in front of the router of the paper's decoder layer (App. A.2 listing: the router
+// reads the normalised hidden state, the residual stays as it was): y = (x / sqrt(mean(x^2) + eps)) * w,
+// rounded once to the storage type, as a model that materialises the normalised activations would
+// hold it.  src: the token's hidden state in shared memory; dst: where the router sweep will read.
+// `scratch` holds one float per warp; two block barriers (`bar`) separate the three phases.
+template <typename T>
+__device__ __forceinline__ void rmsnorm_to_shared(uint32_t src, uint32_t dst, const void *weight_g, float eps, int d,
+                                                  float *scratch, int bar, int tid, int nc, int lane, int warp, int nwarps)
+{
+    using E = Elem<T>;
+    constexpr int VEC = E::VEC;
+    const int ngrp = d / VEC;
+    float ss = 0.f;
+    for (int g = tid; g < ngrp; g += nc) {
+        float x[VEC];
+        E::unpack(lds128(src + 16u * g), x);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) ss = fmaf(x[i], x[i], ss);
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) scratch[warp] = ss;
+    named_bar_sync(bar, nc);
+    float total = 0.f;
+    for (int w = 0; w < nwarps; ++w) total += scratch[w];  // the same order in every thread
+    const float r = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
+    const uint4 *wg = static_cast<const uint4 *>(weight_g);
+    for (int g = tid; g < ngrp; g += nc) {
+        float x[VEC], w[VEC];
+        E::unpack(lds128(src + 16u * g), x);
+        E::unpack(__ldg(wg + g), w);
+        uint32_t o[4];
+        if constexpr (VEC == 8) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn((x[2 * i] * r) * w[2 * i], (x[2 * i + 1] * r) * w[2 * i + 1]);
+                o[i] = *reinterpret_cast<const uint32_t *>(&b);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[i] = __float_as_uint((x[i] * r) * w[i]);
+        }
+        sts128(dst + 16u * g, make_uint4(o[0], o[1], o[2], o[3]));
+    }
+    named_bar_sync(bar, nc);  // the normalised state is complete (and `scratch` free again)
+}
+
 // Cold paths, kept out of the consumers' loop body (its size shows in instruction-fetch stalls).
 __device__ __noinline__ void report_timeout(volatile int *dead, uint32_t *status)
 {
@@ -522,13 +570,16 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 // DIRECT: the compute warps load the hidden state of the block's first token themselves, with plain
 // 16-byte loads, instead of waiting for the producer's bulk copy (a variant of its own because any
 // growth of the loop body costs the other launches 2 - 6 %).
+// NORM (single-layer launches, MODE 0): the router reads RMSNorm(hidden) -- normalised in shared
+// memory after the hidden state has landed -- while the residual stays the hidden state itself
+// (App. A.2 listing).
 template <int SHAPE>
 struct ShapeOf {
     static constexpr int d = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 2048);
     static constexpr int dcc = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 512);
     static constexpr int consumers = SHAPE == 1 ? 96 : 128;
 };
-template <typename T, int NFAST, int P, int MODE, int SHAPE, int DIRECT = 0>
+template <typename T, int NFAST, int P, int MODE, int SHAPE, int DIRECT = 0, int NORM = 0>
 __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const StepParams p)
 {
     using E = Elem<T>;
@@ -741,23 +792,32 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 }
 
                 // ---- router: partial logits over all d columns ----
+                const uint32_t raddr = NORM ? hid_s : haddr;  // what the router reads: RMSNorm(hidden) or hidden itself
                 sweep.clear();
                 if (ring) {
 #pragma unroll 1
                     for (int q = 0; q < K; ++q) {
                         acquire(st, ph);
+                        if constexpr (NORM) {  // the hidden state came with the item's first chunk
+                            if (q == 0)
+                                rmsnorm_to_shared<T>(haddr, hid_s, p.norm_weight, p.norm_eps, d, partial, kBarHidden, tid, nc, lane,
+                                                     warp, nwarps);
+                        }
                         {
                             const uint32_t waddr = smem_base + static_cast<uint32_t>(st) * slot_bytes;
-                            if constexpr (NFAST > 0) sweep.chunk(waddr, haddr + q * chunk_cols_bytes, dcc, tid, nc);
-                            else sweep.chunk_any(waddr, haddr + q * chunk_cols_bytes, dcc, N, warp, lane, nwarps, q == 0, partial);
+                            if constexpr (NFAST > 0) sweep.chunk(waddr, raddr + q * chunk_cols_bytes, dcc, tid, nc);
+                            else sweep.chunk_any(waddr, raddr + q * chunk_cols_bytes, dcc, N, warp, lane, nwarps, q == 0, partial);
                         }
                         release();
                     }
                 } else {
                     if (k > 0 || !direct) acquire(st, ph);  // the first rows chunk brings the hidden state with it
+                    if constexpr (NORM)
+                        rmsnorm_to_shared<T>(haddr, hid_s, p.norm_weight, p.norm_eps, d, partial, kBarHidden, tid, nc, lane, warp,
+                                             nwarps);
                     {
-                        if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, haddr, d, tid, nc);
-                        else sweep.chunk_any(smem_base + m.off_wr, haddr, d, N, warp, lane, nwarps, true, partial);
+                        if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, raddr, d, tid, nc);
+                        else sweep.chunk_any(smem_base + m.off_wr, raddr, d, N, warp, lane, nwarps, true, partial);
                     }
                 }
                 if constexpr (NFAST > 0) {

@@ -51,8 +51,9 @@ static int groups_per_lane(int d, int vec)
     const int groups = d / vec;
     return groups <= 128 ? 1 : (groups <= 256 ? 2 : 4);
 }
-static bool rows_by_expert(int dtype, int N, int d, int K, int in_ring)
+static bool rows_by_expert(int dtype, int N, int d, int K, int in_ring, bool by_columns = false)
 {
+    if (by_columns) return false;
     const bool n_fast = N == 4 || N == 8 || N == 16 || N == 32 || N == 64;
     if (env_int("MOLE_FORCE_COLUMN_CHUNKS") > 0) return false;  // debugging aid
     return dtype == MOLE_DTYPE_BF16 && n_fast && K > 1 && N % K == 0 && in_ring && d / 8 <= 4 * 128;
@@ -68,7 +69,7 @@ static int env_int(const char *name)  // debugging aids: MOLE_FORCE_* override p
     return f ? atoi(f) : 0;
 }
 
-int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan)
+int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns)
 {
     if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
     if (L < 1 || M < 0) return MOLE_ERR_INVALID_ARG;
@@ -80,7 +81,7 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     auto total_smem = [&](int K, int stages) {
         const int dcc = d / K;
         const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
-        const int consumers = rows_by_expert(dtype, N, d, K, in_ring) ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
+        const int consumers = rows_by_expert(dtype, N, d, K, in_ring, by_columns) ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
         return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers).total;
     };
     int K;
@@ -101,7 +102,7 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
         }
     }
     const int dcc = d / K;
-    const bool by_expert = rows_by_expert(dtype, N, d, K, in_ring);
+    const bool by_expert = rows_by_expert(dtype, N, d, K, in_ring, by_columns);
     const int consumers = by_expert ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
     // Resident blocks per SM aimed at: one per token while tokens are few (each with the deepest ring
     // that fits), up to four token chains per SM when there are many (shallower rings, more overlap).
@@ -197,6 +198,27 @@ static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int 
     return pick_p<__nv_bfloat16, 0>(n_fast, lanes);
 }
 
+// The kernels whose router reads RMSNorm(hidden): run-time launch flags, rows cut by columns.
+template <typename T, int P>
+static StepKernel pick_norm_n(int n_fast)
+{
+    switch (n_fast) {
+        case 0: return mole_step_kernel<T, 0, P, 0, 0, 0, 1>;
+        case 4: return mole_step_kernel<T, 4, P, 0, 0, 0, 1>;
+        case 8: return mole_step_kernel<T, 8, P, 0, 0, 0, 1>;
+        case 16: return mole_step_kernel<T, 16, P, 0, 0, 0, 1>;
+        case 32: return mole_step_kernel<T, 32, P, 0, 0, 0, 1>;
+        case 64: return mole_step_kernel<T, 64, P, 0, 0, 0, 1>;
+        default: return nullptr;
+    }
+}
+static StepKernel pick_norm_kernel(int dtype, int n_fast, int lanes)
+{
+    if (dtype == MOLE_DTYPE_BF16)
+        return lanes == 4 ? pick_norm_n<__nv_bfloat16, 4>(n_fast) : (lanes == 2 ? pick_norm_n<__nv_bfloat16, 2>(n_fast) : pick_norm_n<__nv_bfloat16, 1>(n_fast));
+    return lanes == 4 ? pick_norm_n<float, 4>(n_fast) : (lanes == 2 ? pick_norm_n<float, 2>(n_fast) : pick_norm_n<float, 1>(n_fast));
+}
+
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
 static int ensure_smem(StepKernel k, int smem)
 {
@@ -251,14 +273,17 @@ int launch_step(const StepLaunch &a)
 {
     if (a.M == 0) return MOLE_OK;
     StepPlan plan;
-    int rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan);
+    const bool norm = a.norm_weight != nullptr;
+    if (norm && a.L != 1) return MOLE_ERR_INVALID_ARG;
+    int rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan, norm);
     if (rc != MOLE_OK) return rc;
     if (a.M * a.L > 0x3fffffffLL) return MOLE_ERR_TOO_LARGE;
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
-    StepKernel k = pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
-                               plan.rows_by_expert, a.M >= 128 && a.M <= 4LL * sms);
+    StepKernel k = norm ? pick_norm_kernel(a.dtype, plan.n_fast, plan.lanes)
+                        : pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
+                                      plan.rows_by_expert, a.M >= 128 && a.M <= 4LL * sms);
     if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
@@ -277,6 +302,8 @@ int launch_step(const StepLaunch &a)
     p.row_index = a.row_index;
     p.lut = a.lut;
     p.w_router = a.w_router;
+    p.norm_weight = a.norm_weight;
+    p.norm_eps = a.norm_eps;
     p.out = a.out;
     p.gates_out = a.gates_out;
     p.status = a.status;
@@ -338,7 +365,8 @@ int mole_layer_forward_ex(const mole_args *a)
 {
     if (!a || a->struct_size != sizeof(mole_args)) return MOLE_ERR_INVALID_ARG;
     if (a->flags & ~(MOLE_FLAG_IDS_INT64 | MOLE_FLAG_CHAIN)) return MOLE_ERR_INVALID_ARG;
-    if (a->reserved != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->reserved != 0 || a->reserved2 != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->norm_weight && (!aligned16(a->norm_weight) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f)) return MOLE_ERR_INVALID_ARG;
     int rc = check_common(a->hidden, a->ids, a->lut, a->w_router, a->out, a->residual, a->B, a->T, a->N, a->d, a->V,
                           a->dtype);
     if (rc != MOLE_OK) return rc;
@@ -365,6 +393,8 @@ int mole_layer_forward_ex(const mole_args *a)
     s.flags = a->flags;
     s.d_split = a->d_split;
     s.stream = static_cast<cudaStream_t>(a->stream);
+    s.norm_weight = a->norm_weight;
+    s.norm_eps = a->norm_eps;
     return launch_step(s);
 }
 

@@ -33,15 +33,15 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert lib.mole_version() == 200
+    assert lib.mole_version() == 210
     seen = {lib.mole_status_string(c).decode() for c in range(6)}
     assert len(seen) == 6 and "ok" in seen
     assert lib.mole_status_string(99).decode() == "unknown status"
 
 
 def test_args_struct_layout_matches_header(lib):
-    # 2 x u32, 8 pointers, 8 x i32, 1 pointer
-    assert ctypes.sizeof(binding.MoleArgs) == 8 + 8 * 8 + 8 * 4 + 8
+    # 2 x u32, 8 pointers, 8 x i32, 2 pointers, 1 float, 1 i32
+    assert ctypes.sizeof(binding.MoleArgs) == 8 + 8 * 8 + 8 * 4 + 2 * 8 + 4 + 4
 
 
 def test_plan_shapes():
@@ -124,6 +124,16 @@ def test_ex_rejects_bad_struct(lib):
     a.residual = None
     a.reserved = 9
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.reserved = 0
+    a.reserved2 = 1
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.reserved2 = 0
+    a.norm_weight = good + 4  # misaligned scale of the RMSNorm in front of the router
+    assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
+    a.norm_weight = good
+    for eps in (-1.0, float("nan"), float("inf")):
+        a.norm_eps = eps
+        assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
 
 
 def test_decode_step_and_offload_argument_checks(lib):
