@@ -281,6 +281,41 @@ class StepGraphs:
             self.graphs[k % n].replay()
 
 
+class NormStepGraphs(StepGraphs):
+    """The same chained step with the decoder layer of the paper's App. A.2 listing: every layer's
+    router reads RMSNorm(hidden) (fused into the kernel), the residual stays un-normalised."""
+
+    def __init__(self, mole, luts, wrs, gammas, hidden, id_batches, eps=1e-5):
+        import torch
+
+        self.torch, self.graphs = torch, []
+        self.out = torch.empty_like(hidden)
+        self.tmp = torch.empty_like(hidden)
+        self.status = torch.zeros(1, dtype=torch.int32, device=hidden.device)
+        L = luts.shape[0]
+
+        def step(ids):
+            src = hidden
+            for l in range(L):
+                dst = self.out if (L - 1 - l) % 2 == 0 else self.tmp
+                mole.layer_forward(src, ids, luts[l], wrs[l], dst, status=self.status, chain=l > 0,
+                                   norm_weight=gammas[l], norm_eps=eps)
+                src = dst
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for ids in id_batches:
+                step(ids)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        for ids in id_batches:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step(ids)
+            self.graphs.append(g)
+
+
 def timed_ms(torch, fn):
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
@@ -385,6 +420,22 @@ def run_mole(args):
                               "value": whole_job_tokens_per_s(world, M, args.steps, ms_f), "unit": UNIT,
                               "us_per_step": ms_f * 1e3 / args.steps, "algorithmic_bytes_per_launch": fb,
                               "achieved": gbs, "frac": gbs / peak, "traffic": FUSED_TRAFFIC.get((sh.name, M, L))}
+        del g
+
+    # ---- extra: the chained step with RMSNorm fused in front of every layer's router (App. A.2 listing) ----
+    if rank == 0:
+        gammas = torch.stack([inputs.make_router(sh.d, 1, seed=2500 + l, device=dev).reshape(sh.d) + 1.0 for l in range(L)])
+        g = NormStepGraphs(mole, luts, wrs, gammas, hidden, batches_for(M))
+        g.run(0, max(args.warmup, 3))
+        torch.cuda.synchronize()
+        steps_n = min(args.steps, 2000)
+        ms_n = timed_ms(torch, lambda: g.run(0, steps_n))
+        assert int(g.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
+        us_layer_n = ms_n * 1e3 / (steps_n * L)
+        line["norm_router_step"] = {"what": "chained step whose routers read RMSNorm(hidden), fused into the layer kernel",
+                                    "us_per_layer": us_layer_n, "value": M / (us_layer_n * L * 1e-6), "unit": UNIT,
+                                    "achieved": sh.layer_bytes(M) / us_layer_n / 1e3,
+                                    "frac": sh.layer_bytes(M) / us_layer_n / 1e3 / peak}
         del g
 
     # ---- end to end: host buffers in, host buffer out, through the C ABI, every step ---------------------
