@@ -308,6 +308,15 @@ MOLE_API const char *mole_status_string(int code);
 MOLE_API const char *mole_last_cuda_error(void);
 MOLE_API int mole_version(void);
 
+/*
+ * Debugging aids.  Every launch reads these environment variables (unset or 0: no effect); they override
+ * parts of the launch plan and never change what is computed beyond the order of fp32 sums:
+ *   MOLE_FORCE_STAGES (2..8: ring depth), MOLE_FORCE_TARGET_BLOCKS (resident blocks per SM aimed at),
+ *   MOLE_FORCE_BLOCKS_PER_SM (upper bound on the grid), MOLE_FORCE_LANES (1, 2, 4: lanes per column
+ *   group in the combine), MOLE_FORCE_COLUMN_CHUNKS (1: cut the rows by columns even where the expert
+ *   cut exists; the tests use it to run both cuts on the same inputs).
+ */
+
 /* launch shape the library would pick for M tokens and L layers in one launch (L = 1: a single
  * layer): column chunks per token, threads per block, dynamic shared memory, depth of the ring,
  * resident blocks per SM.  Pure host arithmetic, no CUDA call. */
