@@ -590,7 +590,9 @@ def run_offload(args):
     rows = []
     side = torch.cuda.Stream()
     for M in (1, 8, 64):
-        ctx = mole.OffloadContext(M, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
+        # one context sized for the largest batch, as a server would hold it: at the smaller batches a staging
+        # area has room for several layers' rows and the step fetches them in one launch
+        ctx = mole.OffloadContext(64, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
         hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
         bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
         id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
@@ -631,7 +633,8 @@ def run_offload(args):
         rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                      "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                      "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 1 + 2 * L, "us_per_step_without_graph": us_calls})
+                     "launches_per_step": 1 + L + -(-L // min(L, max(1, 64 // M))),  # dedup + layers + fetch groups
+                     "us_per_step_without_graph": us_calls})
         ctx.destroy()
     top = rows[-1]
     line = {

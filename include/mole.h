@@ -278,10 +278,12 @@ MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const vo
 
 /*
  * mole_offload_decode_step -- a whole L-layer decode step in offload mode, one call: the ids
- * are deduplicated ONCE (they are the same for every layer), then layer l+1's distinct rows are
- * fetched from its host table on side_stream while layer l combines on stream (the paper issues
- * the row transfer first so that it overlaps the rest of the layer, App. A.2 listing).  Needs a
- * context with n_buffers >= 2.
+ * are deduplicated ONCE (they are the same for every layer), then the distinct rows of the next
+ * layers are fetched from their host tables on side_stream while the current layers combine on
+ * stream (the paper issues the row transfer first so that it overlaps the rest of the layer, App. A.2
+ * listing).  A staging area holds max_tokens rows, so with B*T tokens one fetch launch brings the rows
+ * of max_tokens / (B*T) consecutive layers (at least one): a context created for the largest batch
+ * serves small batches with few, large fetches.  Needs a context with n_buffers >= 2.
  *   hidden_in device [M][d], read only;  out device [M][d] final result;  tmp device [M][d]
  *   scratch (may be NULL when L == 1);  lut_host_base HOST pointer (pinned + mapped) of layer 0's
  *   table, layer l at + l*lut_layer_stride_bytes;  w_router_base device, layer l at

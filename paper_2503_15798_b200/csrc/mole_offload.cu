@@ -93,20 +93,23 @@ __global__ void __launch_bounds__(kDedupThreads) mole_dedup_kernel(const int32_t
     if (bad && status) atomicOr(status, MOLE_STATUS_BAD_ID);
 }
 
-// staging[u] = table_host[uniq[u]] for u < *count.  blockIdx.y = u, blockIdx.x = 16 KB chunk of
-// the row.  All of a thread's loads are issued before its first store so that many reads are
-// in flight on the host link.
+// staging[z][u] = table_host[z][uniq[u]] for u < *count.  blockIdx.y = u, blockIdx.x = 16 KB chunk
+// of the row, blockIdx.z = z, one of several layers' tables (table_stride bytes apart on the host,
+// staging_stride bytes apart in the staging area) fetched for the same ids in one launch.  All of
+// a thread's loads are issued before its first store so that many reads are in flight on the host link.
 __global__ void __launch_bounds__(kFetchThreads) mole_fetch_kernel(const unsigned char *__restrict__ table_host,
                                                                    const int32_t *__restrict__ uniq,
                                                                    const int32_t *__restrict__ count, long long row_bytes,
-                                                                   unsigned char *__restrict__ staging)
+                                                                   unsigned char *__restrict__ staging, long long table_stride,
+                                                                   long long staging_stride)
 {
     const int u = blockIdx.y;
     if (u >= *count) return;
     const long long row = uniq[u];
     const long long chunk0 = static_cast<long long>(blockIdx.x) * kFetchChunk;
-    const uint4 *src = reinterpret_cast<const uint4 *>(table_host + row * row_bytes + chunk0);
-    uint4 *dst = reinterpret_cast<uint4 *>(staging + static_cast<long long>(u) * row_bytes + chunk0);
+    const long long z = blockIdx.z;
+    const uint4 *src = reinterpret_cast<const uint4 *>(table_host + z * table_stride + row * row_bytes + chunk0);
+    uint4 *dst = reinterpret_cast<uint4 *>(staging + z * staging_stride + static_cast<long long>(u) * row_bytes + chunk0);
     const long long nvec = min(static_cast<long long>(kFetchChunk), row_bytes - chunk0) / 16;
     uint4 v[kFetchVecPerThread];
 #pragma unroll
@@ -129,14 +132,17 @@ static int launch_dedup(const int32_t *ids, int M, int V, int32_t *scratch, int3
     return MOLE_OK;
 }
 
+// `layers` tables, table_stride bytes apart from lut_host on (one pinned allocation), into staging areas
+// staging_stride bytes apart
 static int launch_fetch(const void *lut_host, const int32_t *uniq, const int32_t *count, int max_rows, long long row_bytes,
-                        void *staging, cudaStream_t st)
+                        void *staging, cudaStream_t st, int layers = 1, long long table_stride = 0, long long staging_stride = 0)
 {
     void *dev_alias = nullptr;
     MOLE_CUDA_TRY(cudaHostGetDevicePointer(&dev_alias, const_cast<void *>(lut_host), 0));
-    dim3 grid(static_cast<unsigned>((row_bytes + kFetchChunk - 1) / kFetchChunk), static_cast<unsigned>(max_rows), 1);
+    dim3 grid(static_cast<unsigned>((row_bytes + kFetchChunk - 1) / kFetchChunk), static_cast<unsigned>(max_rows),
+              static_cast<unsigned>(layers));
     mole_fetch_kernel<<<grid, kFetchThreads, 0, st>>>(static_cast<const unsigned char *>(dev_alias), uniq, count, row_bytes,
-                                                      static_cast<unsigned char *>(staging));
+                                                      static_cast<unsigned char *>(staging), table_stride, staging_stride);
     MOLE_CUDA_TRY(cudaGetLastError());
     return MOLE_OK;
 }
@@ -362,47 +368,60 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
     if (rc != MOLE_OK) return rc;
     B0.M = B1.M = static_cast<int>(M);
 
-    // fetch layer l's distinct rows into staging area l & 1 (once layer l-2 has finished with it)
-    auto fetch = [&](int l) -> int {
-        mole_offload_ctx::Buffer &Bl = c->buf[l & 1];
-        if (l >= 2) MOLE_CUDA_TRY(cudaStreamWaitEvent(side, Bl.consumed, 0));
-        int r = launch_fetch(static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l) * lut_layer_stride_bytes,
-                             B0.uniq, B0.count, static_cast<int>(M), c->row_bytes, Bl.staging, side);
+    // A staging area holds max_tokens rows; a step of M tokens needs at most M per layer, so one area
+    // takes the rows of g = max_tokens / M consecutive layers (the ids are the same for all of them):
+    // one fetch launch per group of g layers into staging area (group & 1), issued before the previous
+    // group's layers so that it runs under them.  Fewer, larger fetches: at small batches the step is
+    // bound by the launch + PCIe round trip of every fetch, not by the link.
+    int g = static_cast<int>(c->max_tokens / M);
+    g = g < 1 ? 1 : (g > L ? L : g);
+    const int groups = (L + g - 1) / g;
+    const long long area = M * c->row_bytes;  // one layer's rows inside a staging area
+    auto fetch = [&](int k) -> int {
+        mole_offload_ctx::Buffer &Bk = c->buf[k & 1];
+        const int l0 = k * g, n = (l0 + g <= L) ? g : L - l0;
+        if (k >= 2) MOLE_CUDA_TRY(cudaStreamWaitEvent(side, Bk.consumed, 0));
+        int r = launch_fetch(static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l0) * lut_layer_stride_bytes,
+                             B0.uniq, B0.count, static_cast<int>(M), c->row_bytes, Bk.staging, side, n, lut_layer_stride_bytes,
+                             area);
         if (r != MOLE_OK) return r;
-        MOLE_CUDA_TRY(cudaEventRecord(Bl.ready, side));
+        MOLE_CUDA_TRY(cudaEventRecord(Bk.ready, side));
         return MOLE_OK;
     };
     const void *src = hidden_in;
-    for (int l = 0; l < L; ++l) {
-        if (l == 0 && (rc = fetch(0)) != MOLE_OK) return rc;
-        if (l + 1 < L && (rc = fetch(l + 1)) != MOLE_OK) return rc;  // queued before layer l's combine: they overlap
-        mole_offload_ctx::Buffer &Bl = c->buf[l & 1];
-        void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
-        MOLE_CUDA_TRY(cudaStreamWaitEvent(st, Bl.ready, 0));
-        StepLaunch a;
-        a.hidden = src;
-        a.residual = nullptr;
-        a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
-        a.lut = Bl.staging;
-        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
-        a.out = dst;
-        a.gates_out = nullptr;
-        a.status = status;
-        a.lut_stride = 0;
-        a.wr_stride = 0;
-        a.M = M;
-        a.L = 1;
-        a.N = c->N;
-        a.d = c->d;
-        a.rows = c->max_tokens;
-        a.dtype = c->dtype;
-        a.flags = 0;
-        a.d_split = 0;
-        a.stream = st;
-        rc = launch_step(a);
-        if (rc != MOLE_OK) return rc;
-        MOLE_CUDA_TRY(cudaEventRecord(Bl.consumed, st));
-        src = dst;
+    if ((rc = fetch(0)) != MOLE_OK) return rc;
+    for (int k = 0; k < groups; ++k) {
+        if (k + 1 < groups && (rc = fetch(k + 1)) != MOLE_OK) return rc;  // queued before group k's layers: they overlap
+        mole_offload_ctx::Buffer &Bk = c->buf[k & 1];
+        MOLE_CUDA_TRY(cudaStreamWaitEvent(st, Bk.ready, 0));
+        const int l0 = k * g, n = (l0 + g <= L) ? g : L - l0;
+        for (int l = l0; l < l0 + n; ++l) {
+            void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
+            StepLaunch a;
+            a.hidden = src;
+            a.residual = nullptr;
+            a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
+            a.lut = Bk.staging + static_cast<long long>(l - l0) * area;
+            a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
+            a.out = dst;
+            a.gates_out = nullptr;
+            a.status = status;
+            a.lut_stride = 0;
+            a.wr_stride = 0;
+            a.M = M;
+            a.L = 1;
+            a.N = c->N;
+            a.d = c->d;
+            a.rows = M;  // a slot never exceeds the number of distinct ids
+            a.dtype = c->dtype;
+            a.flags = l > l0 ? MOLE_FLAG_CHAIN : 0;  // inside a group the layers follow one another directly
+            a.d_split = 0;
+            a.stream = st;
+            rc = launch_step(a);
+            if (rc != MOLE_OK) return rc;
+            src = dst;
+        }
+        MOLE_CUDA_TRY(cudaEventRecord(Bk.consumed, st));
     }
     return MOLE_OK;
 }

@@ -195,14 +195,17 @@ def test_offload_bad_ids_and_size_checks():
         host.free()
 
 
-@pytest.mark.parametrize("M,L", [(1, 3), (8, 5), (64, 4), (300, 2), (5, 1)])
-def test_offload_decode_step_equals_resident_layers(M, L):
-    """The whole offload step in one call (one dedup, fetch of layer l+1 under layer l's combine)
-    gives the bytes of L resident single-layer calls; repeated steps on one context stay correct."""
+@pytest.mark.parametrize("M,L,cap", [(1, 3, 1), (8, 5, 8), (64, 4, 64), (300, 2, 300), (5, 1, 5),
+                                     (1, 7, 64), (5, 7, 64), (24, 5, 64), (9, 6, 20), (33, 3, 64)])
+def test_offload_decode_step_equals_resident_layers(M, L, cap):
+    """The whole offload step in one call (one dedup, the next fetch under the current layers' combine)
+    gives the bytes of L resident single-layer calls; repeated steps on one context stay correct.
+    `cap` = the context's max_tokens: with room for cap / M layers' rows in a staging area, one fetch
+    launch brings several layers (all 7, groups of 2 + 2 + 1, 2 + 2 + 2, or one at a time)."""
     N, d, V = 16, 1024, 700
     g = torch.Generator().manual_seed(100 + M)
     host = mole.HostTable((L, V, N, d), torch.bfloat16)
-    ctx = mole.OffloadContext(max_tokens=M, N=N, d=d, V=V, n_buffers=2)
+    ctx = mole.OffloadContext(max_tokens=cap, N=N, d=d, V=V, n_buffers=2)
     side = torch.cuda.Stream()
     try:
         host.tensor.copy_(torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16))
