@@ -462,7 +462,8 @@ def run_mole(args):
     line["e2e"] = {"value": whole_job_tokens_per_s(world, M, e2e_steps, ms_e2e), "unit": UNIT,
                    "h2d_bytes_per_step": M * sh.d * 2 + M * 4, "d2h_bytes_per_step": M * sh.d * 2,
                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
-                   "how": "mole_decode_step_host: pinned host hidden+ids -> device, L chained layers, result -> "
+                   "how": "mole_decode_step_host: pinned host hidden+ids -> device, the step as mole_decode_step launches "
+                          "it by itself (one fused launch over all layers up to 4096 tokens, no CUDA graph), result -> "
                           "pinned host, stream synchronised after every step"}
 
     # ---- sweep over the configuration's batch sizes: chained step + isolated launches -----------------------
