@@ -509,8 +509,12 @@ def run_mole(args):
             for cold in (False, True):
                 ts = []
                 for r in range(reps):
+                    # keep the GPU busy while the host queues the events and the launch, so that the interval
+                    # between the events holds the launch alone: an L2 flush (cold) or a spin that touches no memory
                     if cold:
                         flush.fill_(r & 0xFF)
+                    else:
+                        torch.cuda._sleep(100000)
                     ts.append(timed_ms(torch, lambda: mole.layer_forward(hid, bl[r % N_BATCHES], luts[0], wrs[0], out)))
                 iso.append(statistics.median(ts) * 1e3)
             nbytes = sh.layer_bytes(m)
