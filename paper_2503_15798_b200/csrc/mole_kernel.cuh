@@ -566,7 +566,8 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 // resident, one chunk per item; 3 = router chunks in the ring, several chunks per item, the rows
 // cut by experts (K divides N) instead of by columns.
 // SHAPE: the layer widths of the paper's Table 2 with d, the chunk width and the number of compute
-// threads as constants (0 = any): 1: d = 768; 2: d = 1024; 3: d = 2048 in chunks of 512.
+// threads as constants (0 = any): 1: d = 768; 2: d = 1024; 3: d = 2048 in chunks of 512; 4: d = 2048 in
+// chunks of 1024 (fused steps of at most one token per SM).
 // DIRECT: the compute warps load the hidden state of the block's first token themselves, with plain
 // 16-byte loads, instead of waiting for the producer's bulk copy (a variant of its own because any
 // growth of the loop body costs the other launches 2 - 6 %).
@@ -576,7 +577,7 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 template <int SHAPE>
 struct ShapeOf {
     static constexpr int d = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 2048);
-    static constexpr int dcc = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 512);
+    static constexpr int dcc = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : (SHAPE == 3 ? 512 : 1024));
     static constexpr int consumers = SHAPE == 1 ? 96 : 128;
 };
 template <typename T, int NFAST, int P, int MODE, int SHAPE, int DIRECT = 0, int NORM = 0>
