@@ -92,10 +92,10 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
         if (total_smem(K, 2) > static_cast<uint32_t>(kSmemPerBlockMax)) return MOLE_ERR_UNSUPPORTED_SHAPE;
     } else {
         // the fewest chunks that keep one chunk at or under 32 KB (and a ring of two in shared memory).  A
-        // fused step of at most one token per SM has the SM's whole shared memory for one block: chunks of up
+        // launch of at most one token per SM has the SM's whole shared memory for one block: chunks of up
         // to 64 KB in a ring of three then halve the per-chunk bookkeeping (measured on d = 2048, N = 32,
-        // 16 layers, 1 to 148 tokens: 84 -> 66 us per step; a single-layer launch does not gain)
-        const bool roomy = L > 1 && M <= kNumSMs;
+        // 16 layers, 1 to 148 tokens: 84 -> 56-62 us per step; chained single-layer launches 3 - 12 % less)
+        const bool roomy = M <= kNumSMs && (L > 1 || in_ring);
         const long long chunk_cap = roomy ? 64 * 1024 : 32 * 1024;
         const int ring_min = roomy ? 3 : 2;
         K = 1;
