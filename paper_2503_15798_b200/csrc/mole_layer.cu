@@ -222,12 +222,14 @@ static StepKernel pick_norm_n(int n_fast)
     }
 }
 // ... and, for the single-layer launches of the paper's three layer widths, with the sizes compiled in
-static StepKernel pick_norm_shape_kernel(const StepPlan &plan, int dtype, int d)
+static StepKernel pick_norm_shape_kernel(const StepPlan &plan, int dtype, int d, bool direct)
 {
     if (dtype != MOLE_DTYPE_BF16) return nullptr;
     if (plan.n_fast == 16 && plan.lanes == 1 && plan.d_split == 1 && !plan.wr_in_ring) {
-        if (d == 768 && plan.consumers == 96) return mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 0, 1>;
-        if (d == 1024 && plan.consumers == 128) return mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 0, 1>;
+        if (d == 768 && plan.consumers == 96)
+            return direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 0, 1>;
+        if (d == 1024 && plan.consumers == 128)
+            return direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 0, 1>;
     }
     if (plan.n_fast == 32 && plan.lanes == 2 && plan.d_split == 4 && d == 2048 && plan.dc == 512 && plan.consumers == 128 &&
         plan.rows_by_expert)
@@ -299,19 +301,20 @@ int launch_step(const StepLaunch &a)
     if (norm && a.L != 1) return MOLE_ERR_INVALID_ARG;
     int rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan);
     if (rc != MOLE_OK) return rc;
-    StepKernel k_norm = nullptr;
-    if (norm && !(k_norm = pick_norm_shape_kernel(plan, a.dtype, a.d))) {
-        rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan, true);  // the general kernels cut the rows by columns
-        if (rc != MOLE_OK) return rc;
-        k_norm = pick_norm_kernel(a.dtype, plan.n_fast, plan.lanes);
-    }
     if (a.M * a.L > 0x3fffffffLL) return MOLE_ERR_TOO_LARGE;
     int sms = kNumSMs;
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
+    StepKernel k_norm = nullptr;
+    const bool direct = a.M >= 128 && a.M <= 4LL * sms;  // see pick_kernel
+    if (norm && !(k_norm = pick_norm_shape_kernel(plan, a.dtype, a.d, direct))) {
+        rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan, true);  // the general kernels cut the rows by columns
+        if (rc != MOLE_OK) return rc;
+        k_norm = pick_norm_kernel(a.dtype, plan.n_fast, plan.lanes);
+    }
     StepKernel k = norm ? k_norm
                         : pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
-                                      plan.rows_by_expert, a.M >= 128 && a.M <= 4LL * sms);
+                                      plan.rows_by_expert, direct);
     if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
     rc = ensure_smem(k, plan.smem);
     if (rc != MOLE_OK) return rc;
