@@ -67,3 +67,34 @@ def test_last_row_of_a_table_beyond_4GiB_is_addressed_correctly():
     torch.cuda.synchronize()
     for k, v in enumerate(marks.values()):  # uniform gates over equal rows: out == the mark exactly
         assert (out[k].float() == v).all()
+
+
+@pytest.mark.parametrize("name,M,n_sample", [("160m", 256, 96), ("410m", 256, 64)])
+def test_full_shape_decode_step_chained_and_fused(name, M, n_sample):
+    """Three layers of the full-size tables as the bench launches them (chained with programmatic
+    dependent launch, and the single fused launch): sampled tokens against the oracle's chain on the
+    rows they reference."""
+    sh = inputs.SHAPES[name]
+    L = 3
+    luts = torch.empty((L, sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=DEV)
+    for l in range(L):
+        inputs.make_table(sh.V, sh.N, sh.d, seed=20 + l, device=DEV, out=luts[l])
+    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=30 + l, device=DEV) for l in range(L)])
+    hidden = inputs.make_hidden(M, sh.d, seed=5, device=DEV)
+    ids = inputs.make_ids(M, sh.V, seed=6, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sample = torch.from_numpy(np.sort(np.random.default_rng(1).permutation(M)[:n_sample])).to(DEV)
+    h = hidden[sample].contiguous()
+    ids_s = ids[sample].contiguous()
+    everyone = torch.arange(n_sample, device=DEV)
+    for l in range(L):  # the oracle's chain, each layer fed the storage-type rounding of the previous one
+        ref, _ = _oracle_on_compact_rows(h, ids_s, luts[l], wrs[l], everyone)
+        h = torch.from_numpy(ref).to(torch.bfloat16).to(DEV)
+    want = h.cpu().to(torch.float64).numpy()
+    for mode in (mole.STEP_CHAINED, mole.STEP_FUSED):
+        out = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status, mode=mode)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got = out[sample].cpu().to(torch.float64).numpy()
+        assert (np.abs(got - want) <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(want))).all(), mode
+    del luts
