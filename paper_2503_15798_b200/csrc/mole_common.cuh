@@ -26,11 +26,11 @@ inline int elem_bytes(int dtype) { return dtype == MOLE_DTYPE_BF16 ? 2 : 4; }
 
 // Launch description of the fused kernel (filled by plan_step, pure host arithmetic).
 // A block owns whole tokens; it walks over its tokens and, for every token, over the L layers,
-// pulling the router matrix (L > 1) and the table rows of each (token, layer) item, cut into
-// d_split column chunks, through a ring of `stages` shared-memory slots.
+// pulling the router matrix (when it streams) and the table rows of each (token, layer) item, cut
+// into d_split chunks, through a ring of `stages` shared-memory slots.
 struct StepPlan {
-    int d_split;        // column chunks per token
-    int dc;             // columns per chunk
+    int d_split;        // chunks per item (of the router matrix, and of the rows)
+    int dc;             // columns per router chunk (and per rows chunk when the rows are cut by columns)
     int consumers;      // threads that compute (a multiple of 32); one more warp issues the copies
     int threads;        // consumers + 32
     int stages;         // ring depth, in chunks

@@ -9,18 +9,19 @@
 // type after every layer exactly as a layer-by-layer execution would round it.  There is no
 // communication between blocks.
 //
-// Data movement.  An item is cut into K column chunks of dcc = d / K columns.  Everything it
-// needs is pulled through a ring of shared-memory slots, one chunk per slot, by bulk
-// asynchronous copies (TMA engine, untiled, no multicast) that one extra "producer" warp issues
-// `stages` chunks ahead: first (when L > 1) the K chunks [dcc][N] of the layer's router matrix,
-// then the K chunks of the token's table rows -- [N][dcc], N short pieces per chunk, or, where K
-// divides N (MODE 3), the whole rows [N/K][d] of N/K experts in one contiguous copy, which the
-// copy engine moves three times as fast.  The rows depend only on the id, so they
-// run ahead of the arithmetic and, in a chained launch, ahead of the previous kernel.  A
-// token's hidden state arrives with its first chunk in a small ring of its own (the block's first
-// token excepted: the compute warps load it themselves).  Completion is
-// counted on one mbarrier per slot ("full"); the consumer warps hand a slot back through a
-// second one ("empty").  With L == 1 the router matrix is loaded once per block instead.
+// Data movement.  An item is cut into K chunks.  Everything it needs is pulled through a ring of
+// shared-memory slots, one chunk per slot, by bulk asynchronous copies (TMA engine, untiled, no
+// multicast) that one extra "producer" warp issues `stages` chunks ahead: first (when the router
+// matrix streams: L > 1, or a matrix too large to stay resident) the K chunks [dcc][N] of the
+// layer's router matrix, dcc = d / K columns each, then the K chunks of the token's table rows --
+// [N][dcc], N short pieces per chunk, or, where K divides N (MODE 3), the whole rows [N/K][d] of
+// N/K experts in one contiguous copy, which the copy engine moves three times as fast.  The rows
+// depend only on the id, so they run ahead of the arithmetic and, in a chained launch, ahead of
+// the previous kernel.  A token's hidden state arrives with its first chunk in a small ring of
+// its own (in DIRECT kernels the block's first token excepted: the compute warps load it
+// themselves).  Completion is counted on one mbarrier per slot ("full"); the consumer warps hand
+// a slot back through a second one ("empty").  Otherwise (L == 1, small matrix) the router matrix
+// is loaded once per block and stays.
 //
 // Arithmetic per item (consumer warps): a conflict-free linear sweep over the router chunks in
 // shared memory gives per-lane partial logits, a shuffle reduce-scatter sums them over the warp
