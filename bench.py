@@ -651,7 +651,7 @@ def run_offload(args):
         rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                      "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                      "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 1 + L + -(-L // min(L, max(1, 64 // M))),  # dedup + layers + fetch groups
+                     "launches_per_step": 1 + 2 * -(-L // min(L, max(1, 64 // M))),  # dedup + (fetch + layers) per group
                      "us_per_step_without_graph": us_calls})
         ctx.destroy()
     top = rows[-1]

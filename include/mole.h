@@ -282,13 +282,15 @@ MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const vo
  * layers are fetched from their host tables on side_stream while the current layers combine on
  * stream (the paper issues the row transfer first so that it overlaps the rest of the layer, App. A.2
  * listing).  A staging area holds max_tokens rows, so with B*T tokens one fetch launch brings the rows
- * of max_tokens / (B*T) consecutive layers (at least one): a context created for the largest batch
- * serves small batches with few, large fetches.  Needs a context with n_buffers >= 2.
+ * of max_tokens / (B*T) consecutive layers (at least one), and one fused launch then runs those layers:
+ * a context created for the largest batch serves small batches with few, large fetches and few launches.
+ * Needs a context with n_buffers >= 2.
  *   hidden_in device [M][d], read only;  out device [M][d] final result;  tmp device [M][d]
  *   scratch (may be NULL when L == 1);  lut_host_base HOST pointer (pinned + mapped) of layer 0's
  *   table, layer l at + l*lut_layer_stride_bytes;  w_router_base device, layer l at
  *   + l*wr_layer_stride_bytes.
- * Output is bit-identical to L calls of mole_layer_forward.  stream and side_stream must differ.
+ * Output is bit-identical to L calls of mole_layer_forward when the rows travel in one chunk (see
+ * d_split; otherwise equal up to the order of the fp32 sums).  stream and side_stream must differ.
  * The call may be captured into a CUDA graph (stream capturing, side_stream an ordinary stream: it
  * joins the capture and is joined back before the call returns).  While capturing, the call does not
  * wait for the events of the previous call on the same context -- a captured stream may not depend on

@@ -395,32 +395,32 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
         mole_offload_ctx::Buffer &Bk = c->buf[k & 1];
         MOLE_CUDA_TRY(cudaStreamWaitEvent(st, Bk.ready, 0));
         const int l0 = k * g, n = (l0 + g <= L) ? g : L - l0;
-        for (int l = l0; l < l0 + n; ++l) {
-            void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
-            StepLaunch a;
-            a.hidden = src;
-            a.residual = nullptr;
-            a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
-            a.lut = Bk.staging + static_cast<long long>(l - l0) * area;
-            a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
-            a.out = dst;
-            a.gates_out = nullptr;
-            a.status = status;
-            a.lut_stride = 0;
-            a.wr_stride = 0;
-            a.M = M;
-            a.L = 1;
-            a.N = c->N;
-            a.d = c->d;
-            a.rows = M;  // a slot never exceeds the number of distinct ids
-            a.dtype = c->dtype;
-            a.flags = l > l0 ? MOLE_FLAG_CHAIN : 0;  // inside a group the layers follow one another directly
-            a.d_split = 0;
-            a.stream = st;
-            rc = launch_step(a);
-            if (rc != MOLE_OK) return rc;
-            src = dst;
-        }
+        // the group's layers in ONE launch: their rows lie `area` bytes apart in the staging area, which is
+        // all the fused step kernel needs (a token's chain through the n layers stays on chip)
+        void *dst = (groups - 1 - k) % 2 == 0 ? out : tmp;
+        StepLaunch a;
+        a.hidden = src;
+        a.residual = nullptr;
+        a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
+        a.lut = Bk.staging;
+        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l0) * wr_layer_stride_bytes;
+        a.out = dst;
+        a.gates_out = nullptr;
+        a.status = status;
+        a.lut_stride = area;
+        a.wr_stride = wr_layer_stride_bytes;
+        a.M = M;
+        a.L = n;
+        a.N = c->N;
+        a.d = c->d;
+        a.rows = M;  // a slot never exceeds the number of distinct ids
+        a.dtype = c->dtype;
+        a.flags = 0;
+        a.d_split = 0;
+        a.stream = st;
+        rc = launch_step(a);
+        if (rc != MOLE_OK) return rc;
+        src = dst;
         MOLE_CUDA_TRY(cudaEventRecord(Bk.consumed, st));
     }
     return MOLE_OK;
