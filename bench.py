@@ -36,6 +36,7 @@ if ROOT not in sys.path:
 METRIC = "MoLE layer tokens/s (L-layer decode step) and achieved HBM GB/s"
 UNIT = "tokens/s"
 N_BATCHES = 32          # distinct id batches the steps rotate through
+OFFLOAD_CONTEXT_TOKENS = 256  # offload mode: the context (staging areas) is sized for this many tokens
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
@@ -561,6 +562,16 @@ def run_mole(args):
 # offload mode: table in pinned host memory (410M-shaped by default), one JSON line of its own
 # ------------------------------------------------------------------------------------------------------
 
+def offload_groups(L: int, M: int, row_bytes: int) -> int:
+    """Groups of layers mole_offload_decode_step forms on a context of OFFLOAD_CONTEXT_TOKENS tokens (one
+    fetch launch and one fused layer launch per group): as many layers as the staging area holds, but at
+    least three groups unless the whole step's rows are at most 1 MB."""
+    g = min(L, max(1, OFFLOAD_CONTEXT_TOKENS // M))
+    if M * row_bytes * L > (1 << 20):
+        g = min(g, (L + 2) // 3)
+    return -(-L // g)
+
+
 def run_offload(args):
     """Per decode step and layer: dedup the ids on the device, let the GPU fetch the distinct rows
     from the pinned host table into an HBM staging buffer (side stream), combine from staging (main
@@ -608,9 +619,10 @@ def run_offload(args):
     rows = []
     side = torch.cuda.Stream()
     for M in (1, 8, 64):
-        # one context sized for the largest batch, as a server would hold it: at the smaller batches a staging
-        # area has room for several layers' rows and the step fetches them in one launch
-        ctx = mole.OffloadContext(64, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
+        # one context sized for a server's largest batch (256 tokens: two staging areas of 8 MB): at the batches
+        # timed here a staging area has room for several layers' rows, fetched in one launch and run as one
+        # fused launch
+        ctx = mole.OffloadContext(OFFLOAD_CONTEXT_TOKENS, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
         hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
         bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
         id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
@@ -651,7 +663,7 @@ def run_offload(args):
         rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                      "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                      "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 1 + 2 * -(-L // min(L, max(1, 64 // M))),  # dedup + (fetch + layers) per group
+                     "launches_per_step": 1 + 2 * offload_groups(L, M, row_bytes),  # dedup + (fetch + layers) per group
                      "us_per_step_without_graph": us_calls})
         ctx.destroy()
     top = rows[-1]
@@ -664,7 +676,7 @@ def run_offload(args):
                                f"memory, L={L}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
                    "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": 64,
                    "l2": "rows come from host memory; 32 rotating id batches, one CUDA graph per batch"},
-        "gpu_launches": (1 + 2 * L) * max(20, min(args.steps, 400)),
+        "gpu_launches": top["launches_per_step"] * max(20, min(args.steps, 400)),
         "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": link_fetch, "unit": "GB/s",
                      "frac": top["frac_of_link"], "traffic": None, "kernel": "mole_fetch_kernel",
                      "peak_source": "measured in this run: GPU-initiated read of 8192 rows of the pinned table "

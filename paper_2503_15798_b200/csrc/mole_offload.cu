@@ -375,6 +375,9 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
     // bound by the launch + PCIe round trip of every fetch, not by the link.
     int g = static_cast<int>(c->max_tokens / M);
     g = g < 1 ? 1 : (g > L ? L : g);
+    // ... but unless the whole step's rows are a small transfer (<= 1 MB), keep at least three groups so
+    // that all fetches but the first run under the previous group's layers
+    if (M * c->row_bytes * L > (1LL << 20) && g > (L + 2) / 3) g = (L + 2) / 3;
     const int groups = (L + g - 1) / g;
     const long long area = M * c->row_bytes;  // one layer's rows inside a staging area
     auto fetch = [&](int k) -> int {
