@@ -10,8 +10,9 @@
 // communication between blocks.
 //
 // Data movement.  An item is cut into K chunks.  Everything it needs is pulled through a ring of
-// shared-memory slots, one chunk per slot, by bulk asynchronous copies (TMA engine, untiled, no
-// multicast) that one extra "producer" warp issues `stages` chunks ahead: first (when the router
+// shared-memory slots, one chunk per slot, by bulk asynchronous copies (TMA engine, untiled, every
+// copy into the block's own shared memory) that one extra "producer" warp issues `stages` chunks
+// ahead: first (when the router
 // matrix streams: L > 1, or a matrix too large to stay resident) the K chunks [dcc][N] of the
 // layer's router matrix, dcc = d / K columns each, then the K chunks of the token's table rows --
 // [N][dcc], N short pieces per chunk, or, where K divides N (MODE 3), the whole rows [N/K][d] of
