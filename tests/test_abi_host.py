@@ -57,6 +57,9 @@ def test_plan_shapes():
     # few tokens: one block per SM may use all of its shared memory for a deep ring
     B = binding.DTYPE_BF16
     assert P(64, 16, 768, B, 0, 12)[3] > P(16384, 16, 768, B, 0, 12)[3] and P(64, 16, 768, B, 0, 12)[4] == 1
+    # at most one token per SM and a streaming router: chunks of up to 64 KB in a ring of three
+    assert P(64, 32, 2048, B, 0, 16)[0] == 2 and P(64, 32, 2048, B, 0, 16)[3] >= 3 and P(148, 32, 2048, B, 0, 1)[0] == 2
+    assert P(149, 32, 2048, B, 0, 16)[0] == 4 and P(64, 16, 1024, B, 0, 24)[0] == 1
     # an explicit number of chunks is honoured
     assert P(64, 16, 768, binding.DTYPE_BF16, 4)[0] == 4 and P(64, 16, 768, binding.DTYPE_BF16, 1)[0] == 1
     # never a deeper ring than the chunks a block will see
