@@ -51,6 +51,47 @@ FUSED_TRAFFIC = {
 }
 
 
+def offload_groups(L: int, M: int, row_bytes: int) -> int:
+    """Groups of layers mole_offload_decode_step forms on a context of OFFLOAD_CONTEXT_TOKENS tokens (one
+    fetch launch and one fused layer launch per group): as many layers as the staging area holds, but at
+    least three groups unless the whole step's rows are at most 1 MB."""
+    g = min(L, max(1, OFFLOAD_CONTEXT_TOKENS // M))
+    if M * row_bytes * L > (1 << 20):
+        g = min(g, (L + 2) // 3)
+    return -(-L // g)
+
+
+OFFLOAD_BATCHES = (1, 8, 64)
+
+
+def timed_launch_shapes():
+    """Every launch shape a timed region of this file issues, as dicts (what, M, N, d, L, norm, kernel):
+    the parity tests walk this list and require a parity case for the kernel instantiation of each."""
+    from paper_2503_15798_b200 import inputs
+
+    shapes = []
+    for name in ("160m", "410m", "1b"):
+        sh = inputs.SHAPES[name]
+        for M in sh.batches:
+            for norm in (False, True):
+                tag = " norm" if norm else ""
+                shapes.append({"what": f"{name} batch {M} chained{tag}", "M": M, "N": sh.N, "d": sh.d, "L": 1, "norm": norm,
+                               "kernel": 0})
+                if M <= 4096:
+                    shapes.append({"what": f"{name} batch {M} fused{tag}", "M": M, "N": sh.N, "d": sh.d, "L": sh.L,
+                                   "norm": norm, "kernel": 0})
+            shapes.append({"what": f"{name} batch {M} chained, ring kernel", "M": M, "N": sh.N, "d": sh.d, "L": 1,
+                           "norm": False, "kernel": 1})
+    sh = inputs.SHAPES["410m"]
+    for M in OFFLOAD_BATCHES:
+        groups = offload_groups(sh.L, M, sh.row_bytes)
+        per = -(-sh.L // groups)
+        for L in {per, sh.L - per * (groups - 1)}:
+            shapes.append({"what": f"410m offload batch {M}, group of {L} layers", "M": M, "N": sh.N, "d": sh.d, "L": L,
+                           "norm": False, "kernel": 0})
+    return shapes
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -561,16 +602,6 @@ def run_mole(args):
 # ------------------------------------------------------------------------------------------------------
 # offload mode: table in pinned host memory (410M-shaped by default), one JSON line of its own
 # ------------------------------------------------------------------------------------------------------
-
-def offload_groups(L: int, M: int, row_bytes: int) -> int:
-    """Groups of layers mole_offload_decode_step forms on a context of OFFLOAD_CONTEXT_TOKENS tokens (one
-    fetch launch and one fused layer launch per group): as many layers as the staging area holds, but at
-    least three groups unless the whole step's rows are at most 1 MB."""
-    g = min(L, max(1, OFFLOAD_CONTEXT_TOKENS // M))
-    if M * row_bytes * L > (1 << 20):
-        g = min(g, (L + 2) // 3)
-    return -(-L // g)
-
 
 def run_offload(args):
     """Per decode step and layer: dedup the ids on the device, let the GPU fetch the distinct rows

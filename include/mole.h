@@ -46,7 +46,7 @@
 extern "C" {
 #endif
 
-#define MOLE_VERSION 210
+#define MOLE_VERSION 300
 
 /* every entry point is exported from the shared library with default visibility */
 #if defined(__GNUC__)
@@ -78,6 +78,12 @@ extern "C" {
                                   on the stream has finished; it reads hidden / residual only      \
                                   after it has.  Only valid if ids, lut and w_router are not       \
                                   written by that previous kernel. */
+
+/* which kernel family runs a single-layer launch (mole_args.kernel, mole_step_args.kernel) */
+#define MOLE_KERNEL_AUTO 0   /* the library's choice */
+#define MOLE_KERNEL_RING 1   /* persistent blocks, rows and router chunks streamed through a shared-memory ring: any shape */
+#define MOLE_KERNEL_DECODE 2 /* one block per token, rows held in registers, built for decode batches: bf16, N of 4, 8, \
+                                16 or 32, d a multiple of 128 up to 2048 (1024 for N = 32), d_split 0 */
 
 /* mole_decode_step_ex mode: how the L layers of a step are launched */
 #define MOLE_STEP_AUTO 0    /* fused unless the batch is large (then chained) */
@@ -118,7 +124,11 @@ typedef struct mole_args {
     uint32_t *status;      /* device status word (MOLE_STATUS_* bits OR-ed in), or NULL */
     int32_t B, T, N, d, V;
     int32_t dtype;         /* MOLE_DTYPE_* */
-    int32_t reserved;      /* must be 0 */
+    int32_t kernel;        /* MOLE_KERNEL_*; AUTO takes the decode kernel for up to 2048 tokens where it exists and
+                              d_split is 0, the ring kernel otherwise.  The two families add the same fp32 terms in a
+                              different order, so their outputs may differ in a rounding decision; within one family
+                              and launch shape a token's result is the same bits whatever batch it is in.
+                              MOLE_ERR_UNSUPPORTED_SHAPE if DECODE is asked for a shape it does not cover. */
     int32_t d_split;       /* chunks a token's router matrix and rows are streamed in (1, 2, 4, 8 or 16; d/d_split must
                               stay a multiple of the vector width); 0 = auto: the fewest chunks of at most 32 KB.
                               The router matrix is cut by columns.  The rows are cut by experts (whole rows of
@@ -161,7 +171,8 @@ MOLE_API int mole_layer_forward_ex(const mole_args *args);
  *    l+1's first row gathers are in flight while layer l finishes.  This is what a model that
  *    runs other work between the layers gets by calling mole_layer_forward_ex per layer.
  * mole_decode_step picks FUSED up to 4096 tokens and CHAINED above; _ex lets the caller choose
- * and force d_split (0 = auto).
+ * and force d_split (0 = auto).  The first launch of a step waits for everything before it on the
+ * stream (see mole_decode_step_args for the flag that lets it start early).
  */
 MOLE_API int mole_decode_step(const void *hidden_in, const int32_t *ids, const void *lut_base,
                      int64_t lut_layer_stride_bytes, const void *w_router_base,
@@ -171,6 +182,43 @@ MOLE_API int mole_decode_step_ex(const void *hidden_in, const int32_t *ids, cons
                      int64_t lut_layer_stride_bytes, const void *w_router_base,
                      int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status, int L, int B,
                      int T, int N, int d, int V, int dtype, int mode, int d_split, void *stream);
+
+/*
+ * mole_decode_step_args -- the L-layer step with every option, among them the decoder layer of the
+ * paper's App. A.2 listing in every layer: with norm_weight_base set, layer l's router reads
+ * RMSNorm(hidden) with the scale vector at norm_weight_base + l*norm_layer_stride_bytes (see
+ * mole_args.norm_weight) while the residual stays the un-normalised hidden state.  Both modes take it.
+ * The first launch of a step is an ordinary launch: it starts after everything that precedes it on the
+ * stream.  MOLE_FLAG_CHAIN in `flags` lets it start early as well (programmatic dependent launch); only
+ * valid if the kernel before it on the stream writes none of ids, the tables, the router weights and the
+ * norm weights.  Later layers of a CHAINED step are always chained to their predecessor.
+ */
+typedef struct mole_step_args {
+    uint32_t struct_size;  /* sizeof(mole_step_args), checked */
+    uint32_t flags;        /* 0 or MOLE_FLAG_CHAIN */
+    const void *hidden_in; /* device [M][d], dtype, read only */
+    const void *ids;       /* device int32 [M] */
+    const void *lut_base;  /* device; layer l's table [V][N][d] at + l*lut_layer_stride_bytes */
+    int64_t lut_layer_stride_bytes;
+    const void *w_router_base; /* device; layer l's router [d][N] at + l*wr_layer_stride_bytes */
+    int64_t wr_layer_stride_bytes;
+    const void *norm_weight_base; /* device [d] per layer, dtype, or NULL: routers read hidden itself */
+    int64_t norm_layer_stride_bytes;
+    void *out;             /* device [M][d] */
+    void *tmp;             /* device [M][d] scratch of CHAINED mode (NULL when L == 1 or FUSED) */
+    uint32_t *status;      /* device status word or NULL */
+    int32_t L, B, T, N, d, V;
+    int32_t dtype;         /* MOLE_DTYPE_* */
+    int32_t mode;          /* MOLE_STEP_* */
+    int32_t d_split;       /* as mole_args.d_split */
+    int32_t kernel;        /* as mole_args.kernel, for the single-layer launches of CHAINED mode; a FUSED step of
+                              several layers always runs on the ring kernel */
+    float norm_eps;        /* >= 0; read only with norm_weight_base */
+    int32_t reserved;      /* must be 0 */
+    void *stream;          /* cudaStream_t */
+} mole_step_args;
+
+MOLE_API int mole_decode_step_args(const mole_step_args *args);
 
 /*
  * mole_decode_step_host -- mole_decode_step for a caller whose activations live in HOST
@@ -187,8 +235,8 @@ MOLE_API int mole_decode_step_host(const void *hidden_host, const int32_t *ids_h
                           int V, int dtype, void *stream);
 
 /* ---------------------------------------------------------------------------------------
- * Offload mode: the table stays in pinned host memory (the paper keeps it "offloaded to the
- * storage device" and moves only the looked-up rows, Sec. 3.3 and the inference listing).
+ * Offload mode: the table lives off the accelerator, in pinned host memory, and only the
+ * looked-up rows move (Sec. 3.3 and the inference listing of App. A.2).
  * Per step the distinct ids are found on the device and only their rows cross the host link.
  * ------------------------------------------------------------------------------------- */
 
@@ -271,7 +319,7 @@ MOLE_API int mole_offload_prefetch(mole_offload_ctx *ctx, int buf, const int32_t
  * mole_layer_forward_offload -- on stream: wait for buffer `buf`'s ready event, run the fused
  * layer with the gather reading staging[slot[t]], record the buffer's consumed event.
  * B*T must equal the M given to the matching prefetch.  Output is bit-identical to
- * mole_layer_forward on the same inputs.
+ * mole_layer_forward on the same inputs (the same kernel choice, the same order of sums).
  */
 MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const void *hidden, const void *w_router, void *out,
                                uint32_t *status, int B, int T, void *stream);
@@ -290,8 +338,9 @@ MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const vo
  *   scratch (may be NULL when L == 1);  lut_host_base HOST pointer (pinned + mapped) of layer 0's
  *   table, layer l at + l*lut_layer_stride_bytes;  w_router_base device, layer l at
  *   + l*wr_layer_stride_bytes.
- * Output is bit-identical to L calls of mole_layer_forward when the rows travel in one chunk (see
- * d_split; otherwise equal up to the order of the fp32 sums).  stream and side_stream must differ.
+ * Every group runs on the ring kernel: the output is bit-identical to L single-layer calls with
+ * kernel = MOLE_KERNEL_RING when the rows travel in one chunk (see d_split; otherwise equal up to the order
+ * of the fp32 sums).  stream and side_stream must differ.
  * The call may be captured into a CUDA graph (stream capturing, side_stream an ordinary stream: it
  * joins the capture and is joined back before the call returns).  While capturing, the call does not
  * wait for the events of the previous call on the same context -- a captured stream may not depend on
@@ -314,19 +363,33 @@ MOLE_API const char *mole_last_cuda_error(void);
 MOLE_API int mole_version(void);
 
 /*
- * Debugging aids.  Every launch reads these environment variables (unset or 0: no effect); they override
- * parts of the launch plan and never change what is computed beyond the order of fp32 sums:
+ * Debugging aids.  The library reads these environment variables ONCE, at the first launch or plan
+ * (unset or 0: no effect); mole_reload_debug_env() reads them again (tests flip them between launches).
+ * They override parts of the launch plan and never change what is computed beyond the order of fp32 sums:
  *   MOLE_FORCE_STAGES (2..8: ring depth), MOLE_FORCE_TARGET_BLOCKS (resident blocks per SM aimed at),
  *   MOLE_FORCE_BLOCKS_PER_SM (upper bound on the grid), MOLE_FORCE_LANES (1, 2, 4: lanes per column
  *   group in the combine), MOLE_FORCE_COLUMN_CHUNKS (1: cut the rows by columns even where the expert
- *   cut exists; the tests use it to run both cuts on the same inputs).
+ *   cut exists), MOLE_FORCE_KERNEL (1, 2: MOLE_KERNEL_* for launches that leave the choice open).
+ * One of them shortens the bounded waits inside the kernels, to let a test see a wait run out:
+ *   MOLE_DEBUG_WAIT_LIMIT (n >= 1: a wait gives up after n polls; negative: after none -- any wait that
+ *   is not satisfied at once gives up).  The launch then returns normally with MOLE_STATUS_TIMEOUT in
+ *   the status word and undefined outputs; nothing faults and the stream stays usable.
  */
+MOLE_API int mole_reload_debug_env(void);
 
-/* launch shape the library would pick for M tokens and L layers in one launch (L = 1: a single
+/* launch shape the ring kernel would get for M tokens and L layers in one launch (L = 1: a single
  * layer): column chunks per token, threads per block, dynamic shared memory, depth of the ring,
- * resident blocks per SM.  Pure host arithmetic, no CUDA call. */
+ * resident blocks per SM.  Host arithmetic only; the SM count is the current device's if there is
+ * one, else the 148 of a B200. */
 MOLE_API int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads,
               int *out_smem_bytes, int *out_stages, int *out_blocks_per_sm);
+
+/* Name of the kernel instantiation a launch of this shape runs ("decode<N,NORM>" or
+ * "step<storage,N,P,MODE,SHAPE,DIRECT,NORM>"), with its block size and dynamic shared memory: lets a
+ * test list which instantiations a workload reaches.  norm != 0: with a normalised router; kernel as
+ * mole_args.kernel.  name receives at most name_bytes - 1 characters and a terminator.  Launches nothing. */
+MOLE_API int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, char *name,
+                 int name_bytes, int *out_threads, int *out_smem_bytes);
 
 #ifdef __cplusplus
 }

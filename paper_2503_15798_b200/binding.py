@@ -21,6 +21,7 @@ STATUS_BAD_ID, STATUS_TIMEOUT = 1, 2
 DTYPE_BF16, DTYPE_F32 = 0, 1
 FLAG_IDS_INT64, FLAG_CHAIN = 1, 2
 STEP_AUTO, STEP_FUSED, STEP_CHAINED = 0, 1, 2
+KERNEL_AUTO, KERNEL_RING, KERNEL_DECODE = 0, 1, 2
 
 # every symbol include/mole.h declares
 EXPORTS = (
@@ -28,7 +29,8 @@ EXPORTS = (
     "mole_dedup_ids", "mole_dedup_ids_static", "mole_fetch_rows", "mole_host_alloc", "mole_host_free", "mole_offload_create",
     "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_decode_step",
     "mole_offload_buffers",
-    "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan",
+    "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan", "mole_variant", "mole_reload_debug_env",
+    "mole_decode_step_args",
 )
 
 
@@ -38,9 +40,23 @@ class MoleArgs(ctypes.Structure):
         ("hidden", c_void_p), ("ids", c_void_p), ("lut", c_void_p), ("w_router", c_void_p), ("out", c_void_p),
         ("residual", c_void_p), ("gates_out", c_void_p), ("status", c_void_p),
         ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
-        ("dtype", c_int32), ("reserved", c_int32), ("d_split", c_int32),
+        ("dtype", c_int32), ("kernel", c_int32), ("d_split", c_int32),
         ("stream", c_void_p),
         ("norm_weight", c_void_p), ("norm_eps", ctypes.c_float), ("reserved2", c_int32),
+    ]
+
+
+class MoleStepArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", c_uint32), ("flags", c_uint32),
+        ("hidden_in", c_void_p), ("ids", c_void_p), ("lut_base", c_void_p), ("lut_layer_stride_bytes", c_int64),
+        ("w_router_base", c_void_p), ("wr_layer_stride_bytes", c_int64),
+        ("norm_weight_base", c_void_p), ("norm_layer_stride_bytes", c_int64),
+        ("out", c_void_p), ("tmp", c_void_p), ("status", c_void_p),
+        ("L", c_int32), ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
+        ("dtype", c_int32), ("mode", c_int32), ("d_split", c_int32), ("kernel", c_int32),
+        ("norm_eps", ctypes.c_float), ("reserved", c_int32),
+        ("stream", c_void_p),
     ]
 
 
@@ -93,6 +109,10 @@ def lib() -> ctypes.CDLL:
         L.mole_version.argtypes = []
         L.mole_plan.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
                                 POINTER(c_int), POINTER(c_int), POINTER(c_int)]
+        L.mole_variant.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, ctypes.c_char_p, c_int,
+                                   POINTER(c_int), POINTER(c_int)]
+        L.mole_reload_debug_env.argtypes = []
+        L.mole_decode_step_args.argtypes = [POINTER(MoleStepArgs)]
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is not c_char_p:
@@ -133,7 +153,7 @@ def _dev(t: torch.Tensor, name: str):
 
 def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_out=None, status=None,
                   d_split: int = 0, chain: bool = False, stream=None, B=None, T=None, norm_weight=None,
-                  norm_eps: float = 1e-6):
+                  norm_eps: float = 1e-6, kernel: int = KERNEL_AUTO):
     """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d],
     w_router [d][N]; returns out (allocated like hidden if not given).  norm_weight [d]: the router
     reads RMSNorm(hidden) with that scale and norm_eps, the residual stays un-normalised."""
@@ -164,7 +184,7 @@ def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_
     a.hidden, a.ids, a.lut, a.w_router, a.out = _ptr(hidden), _ptr(ids), _ptr(lut), _ptr(w_router), _ptr(out)
     a.residual, a.gates_out, a.status = _ptr(residual), _ptr(gates_out), _ptr(status)
     a.B, a.T, a.N, a.d, a.V = B, T, N, d, V
-    a.dtype, a.reserved, a.d_split = tag, 0, d_split
+    a.dtype, a.kernel, a.d_split = tag, kernel, d_split
     a.stream = _stream(stream)
     if norm_weight is not None:
         _dev(norm_weight, "norm_weight")
@@ -195,6 +215,32 @@ def decode_step(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, str
                                      _ptr(w_routers), w_routers.stride(0) * w_routers.element_size(), _ptr(out),
                                      _ptr(tmp), _ptr(status), L, M, 1, N, d, V, tag, mode, d_split, _stream(stream)),
            "mole_decode_step_ex")
+    return out
+
+
+def decode_step_args(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None, mode: int = STEP_AUTO,
+                     d_split: int = 0, norm_weights=None, norm_eps: float = 1e-6, kernel: int = KERNEL_AUTO,
+                     chain_first: bool = False):
+    """mole_decode_step_args: decode_step with every option; norm_weights [L][d] puts RMSNorm(hidden) in
+    front of every layer's router."""
+    L, V, N, d = luts.shape
+    a = MoleStepArgs()
+    a.struct_size = ctypes.sizeof(MoleStepArgs)
+    a.flags = FLAG_CHAIN if chain_first else 0
+    a.hidden_in, a.ids, a.lut_base = _ptr(hidden_in), _ptr(ids), _ptr(luts)
+    a.lut_layer_stride_bytes = luts.stride(0) * luts.element_size()
+    a.w_router_base, a.wr_layer_stride_bytes = _ptr(w_routers), w_routers.stride(0) * w_routers.element_size()
+    if norm_weights is not None:
+        _dev(norm_weights, "norm_weights")
+        if norm_weights.dtype != hidden_in.dtype or tuple(norm_weights.shape) != (L, d):
+            raise ValueError("norm_weights must be [L][d] of the element type of hidden")
+        a.norm_weight_base, a.norm_layer_stride_bytes = _ptr(norm_weights), norm_weights.stride(0) * norm_weights.element_size()
+    a.out, a.tmp, a.status = _ptr(out), _ptr(tmp), _ptr(status)
+    a.L, a.B, a.T, a.N, a.d, a.V = L, ids.numel(), 1, N, d, V
+    a.dtype, a.mode, a.d_split, a.kernel = _dtype_tag(hidden_in), mode, d_split, kernel
+    a.norm_eps, a.reserved = float(norm_eps), 0
+    a.stream = _stream(stream)
+    _check(lib().mole_decode_step_args(ctypes.byref(a)), "mole_decode_step_args")
     return out
 
 
@@ -347,6 +393,40 @@ def plan(M: int, N: int, d: int, dtype: int = DTYPE_BF16, d_split: int = 0, L: i
     _check(lib().mole_plan(M, L, N, d, dtype, d_split, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
                            ctypes.byref(e), ctypes.byref(f)), "mole_plan")
     return a.value, b.value, c.value, e.value, f.value
+
+
+def variant(M: int, N: int, d: int, dtype: int = DTYPE_BF16, d_split: int = 0, L: int = 1, norm: bool = False,
+            kernel: int = KERNEL_AUTO):
+    """mole_variant: (name, threads, smem_bytes) of the kernel instantiation a launch of this shape runs."""
+    buf = ctypes.create_string_buffer(96)
+    th, sm = c_int(), c_int()
+    _check(lib().mole_variant(M, L, N, d, dtype, d_split, int(norm), kernel, buf, len(buf), ctypes.byref(th),
+                              ctypes.byref(sm)), "mole_variant")
+    return buf.value.decode(), th.value, sm.value
+
+
+class debug_env:
+    """Context manager: set MOLE_FORCE_* / MOLE_DEBUG_* variables, make the library read them, and put
+    the environment back (and make the library read it again) on exit."""
+
+    def __init__(self, **variables):
+        self.variables = {k: str(v) for k, v in variables.items()}
+        self.saved = {}
+
+    def __enter__(self):
+        for k, v in self.variables.items():
+            self.saved[k] = os.environ.get(k)
+            os.environ[k] = v
+        _check(lib().mole_reload_debug_env(), "mole_reload_debug_env")
+        return self
+
+    def __exit__(self, *exc):
+        for k, old in self.saved.items():
+            if old is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = old
+        _check(lib().mole_reload_debug_env(), "mole_reload_debug_env")
 
 
 def version() -> int:

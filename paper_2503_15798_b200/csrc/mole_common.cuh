@@ -44,7 +44,9 @@ struct StepPlan {
     int lanes;          // combine: lanes per 16-byte column group (by columns) or column groups per lane (by experts)
 };
 // `by_columns`: never cut the rows by experts (kernel variants that exist for the column cut only)
-int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns = false);
+// `sms`: SM count the plan is laid out for (< 1: the nominal 148 of a B200); `norm`: room for RMSNorm(hidden)
+int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns = false, int sms = 0,
+              bool norm = false);
 
 // One launch of the fused kernel over L chained layers (L == 1: a single layer).
 // `row_index` is ids (resident mode) or slot (offload mode); `rows` the number of table rows
@@ -62,8 +64,10 @@ struct StepLaunch {
     uint32_t flags;
     int d_split;
     cudaStream_t stream;
-    const void *norm_weight = nullptr;  // [d], dtype: the router reads RMSNorm(hidden) (single layer only); NULL: hidden
+    const void *norm_weight = nullptr;  // [d], dtype: the router reads RMSNorm(hidden); NULL: hidden itself
+    long long norm_stride = 0;          // bytes between the scale vectors of consecutive layers
     float norm_eps = 0.f;
+    int kernel = 0;  // MOLE_KERNEL_*: which kernel family runs the launch (0: the library's choice)
 };
 int launch_step(const StepLaunch &a);
 

@@ -44,12 +44,13 @@ constexpr int kMaxStages = 8;       // ring depth
 constexpr int kBarLogits = 1;       // named barriers of the consumer warps: partial logits written,
 constexpr int kBarGates = 2;        // softmax numerators written,
 constexpr int kBarHidden = 3;       // running hidden state written
-constexpr uint32_t kWaitPolls = 1u << 24;   // >= 1 s of polling before a wait gives up
+constexpr uint32_t kWaitPolls = 1u << 24;   // default poll limit: >= 1 s of polling before a wait gives up
 constexpr uint32_t kDrainPolls = 1u << 14;  // after a failure: short waits for copies still in flight
 
 struct StepParams {
     const void *hidden, *residual, *row_index, *lut, *w_router;
     const void *norm_weight;  // [d] scale of the RMSNorm in front of the router (NORM kernels), else unused
+    long long norm_stride;    // bytes between the scale vectors of consecutive layers
     float norm_eps;
     void *out;
     float *gates_out;
@@ -59,17 +60,18 @@ struct StepParams {
     int N, d, K, dcc, L;
     int stages, hring, wr_in_ring, consumers;
     uint32_t flags;
+    uint32_t wait_polls;  // polls after which a wait on the ring gives up (kWaitPolls unless a test shortens it)
 };
 
 // Shared-memory map, computed the same way on the host (for the size) and in the kernel.
 struct SmemMap {
     uint32_t chunk_bytes;  // one ring slot: a [dcc][N] router chunk or an [N][dcc] rows chunk
     uint32_t hid_bytes;    // one hidden state: d elements
-    uint32_t off_wr, off_hring, off_hid, off_partial, off_gates, off_meta, off_bars, total;
+    uint32_t off_wr, off_hring, off_hid, off_norm, off_partial, off_gates, off_meta, off_bars, total;
 };
 __host__ __device__ inline uint32_t up128(uint32_t x) { return (x + 127u) & ~127u; }
 __host__ __device__ inline SmemMap smem_map(int N, int d, int dcc, int eb, int stages, int hring, int wr_in_ring,
-                                            int consumers)
+                                            int consumers, int norm)
 {
     SmemMap m;
     m.chunk_bytes = static_cast<uint32_t>(N) * dcc * eb;
@@ -78,7 +80,8 @@ __host__ __device__ inline SmemMap smem_map(int N, int d, int dcc, int eb, int s
     m.off_wr = stages * up128(m.chunk_bytes);                                             // resident router matrix (L == 1)
     m.off_hring = m.off_wr + (wr_in_ring ? 0u : up128(static_cast<uint32_t>(d) * N * eb));  // hidden states of the tokens in flight
     m.off_hid = m.off_hring + hring * up128(m.hid_bytes);                                 // running hidden state between layers
-    m.off_partial = m.off_hid + up128(m.hid_bytes);
+    m.off_norm = m.off_hid + up128(m.hid_bytes);                                          // RMSNorm(hidden), what a normalised router reads
+    m.off_partial = m.off_norm + (norm ? up128(m.hid_bytes) : 0u);
     m.off_gates = m.off_partial + up128(warps * N * 4);
     m.off_meta = m.off_gates + up128(N * 4);
     m.off_bars = m.off_meta + up128((kMaxStages + 3) * 4);
@@ -550,11 +553,12 @@ __device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
 // for a warp that has given up -- a short wait that lets copies already issued land, so that none
 // is in flight when the block exits.
 __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volatile int *dead, bool alive, bool issued,
-                                          uint32_t *status, int lane)
+                                          uint32_t *status, int lane, uint32_t polls)
 {
     if (alive) {
-        if (wait_or_give_up(bar, parity, dead, kWaitPolls)) return true;
+        if (wait_or_give_up(bar, parity, dead, polls)) return true;
         if (lane == 0) report_timeout(dead, status);
+        if (issued) (void)wait_or_give_up(bar, parity, dead + 2, kDrainPolls);  // this chunk's copies may still be on their way
         return false;
     }
     if (issued) (void)wait_or_give_up(bar, parity, dead + 2, kDrainPolls);
@@ -573,9 +577,9 @@ __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volati
 // DIRECT: the compute warps load the hidden state of the block's first token themselves, with plain
 // 16-byte loads, instead of waiting for the producer's bulk copy (a variant of its own because any
 // growth of the loop body costs the other launches 2 - 6 %).
-// NORM (single-layer launches, MODE 0): the router reads RMSNorm(hidden) -- normalised in shared
-// memory after the hidden state has landed -- while the residual stays the hidden state itself
-// (App. A.2 listing).
+// NORM: the router reads RMSNorm(hidden) -- normalised into a buffer of its own in shared memory
+// after the hidden state has landed (layer l of a fused step with the l-th scale vector) -- while
+// the residual stays the hidden state itself (App. A.2 listing).
 template <int SHAPE>
 struct ShapeOf {
     static constexpr int d = SHAPE == 1 ? 768 : (SHAPE == 2 ? 1024 : 2048);
@@ -598,7 +602,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
     const int nc = SHAPE ? ShapeOf<SHAPE>::consumers : p.consumers;
     const bool ring = MODE == 0 ? (p.wr_in_ring != 0) : (MODE != 2);  // router chunks travel through the ring
     constexpr bool kRowsByExpert = MODE == 3;  // rows chunk kk = the whole rows of experts kk*N/K ..
-    const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, ring, nc);
+    const SmemMap m = smem_map(N, d, dcc, EB, stages, HR, ring, nc, NORM);
     const uint32_t slot_bytes = up128(m.chunk_bytes), hid_stride = up128(m.hid_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long G = gridDim.x, b0 = blockIdx.x;
@@ -725,7 +729,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         for (long long ci = pre; ci < total; ++ci) {
             int ok = 1;
             if (lane == 0) {
-                ok = wait_or_give_up(empty + pst, pph, dead, kWaitPolls, true);
+                ok = wait_or_give_up(empty + pst, pph, dead, p.wait_polls, true);
                 if (!ok) report_timeout(dead, p.status);
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -740,7 +744,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         float *partial = reinterpret_cast<float *>(smem + m.off_partial);  // [nwarps][N]
         float *gates = reinterpret_cast<float *>(smem + m.off_gates);      // [N] softmax numerators of the current item
         const uint32_t smem_base = smem_u32(smem);
-        const uint32_t hid_s = smem_base + m.off_hid, gates_s = smem_u32(gates);
+        const uint32_t hid_s = smem_base + m.off_hid, norm_s = smem_base + m.off_norm, gates_s = smem_u32(gates);
         const uint32_t chunk_cols_bytes = static_cast<uint32_t>(dcc) * EB;
         // After a wait has timed out (`alive` false) the warp stops waiting but keeps going through the
         // arithmetic and the barriers on whatever the slots hold -- every address stays inside shared
@@ -758,10 +762,13 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
         long long ci = 0;  // chunks consumed so far
         auto acquire = [&](int st, uint32_t ph) {
             if (alive && mbar_try_wait(full + st, ph)) return;  // the usual case: the copies have landed
-            alive = acquire_slow(full + st, ph, dead, alive, ci < *issued, p.status, lane);
+            alive = acquire_slow(full + st, ph, dead, alive, ci < *issued, p.status, lane, p.wait_polls);
         };
         if (!ring && ntok > 0) {
-            if (!wait_or_give_up(wrbar, 0, dead, kWaitPolls)) give_up();
+            if (!wait_or_give_up(wrbar, 0, dead, p.wait_polls)) {
+                give_up();
+                (void)wait_or_give_up(wrbar, 0, dead + 2, kDrainPolls);  // let the router matrix land before the block can exit
+            }
         }
 
         int st = 0, he = 0;  // ring slot of the next chunk, hidden-ring entry of the current token
@@ -795,7 +802,8 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 }
 
                 // ---- router: partial logits over all d columns ----
-                const uint32_t raddr = NORM ? hid_s : haddr;  // what the router reads: RMSNorm(hidden) or hidden itself
+                const uint32_t raddr = NORM ? norm_s : haddr;  // what the router reads: RMSNorm(hidden) or hidden itself
+                const void *norm_w = static_cast<const unsigned char *>(p.norm_weight) + static_cast<size_t>(l) * p.norm_stride;
                 sweep.clear();
                 if (ring) {
 #pragma unroll 1
@@ -803,7 +811,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                         acquire(st, ph);
                         if constexpr (NORM) {  // the hidden state came with the item's first chunk
                             if (q == 0)
-                                rmsnorm_to_shared<T>(haddr, hid_s, p.norm_weight, p.norm_eps, d, partial, kBarHidden, tid, nc, lane,
+                                rmsnorm_to_shared<T>(haddr, norm_s, norm_w, p.norm_eps, d, partial, kBarHidden, tid, nc, lane,
                                                      warp, nwarps);
                         }
                         {
@@ -816,7 +824,7 @@ __global__ void __launch_bounds__(kMaxConsumers + 32) mole_step_kernel(const Ste
                 } else {
                     if (k > 0 || !direct) acquire(st, ph);  // the first rows chunk brings the hidden state with it
                     if constexpr (NORM)
-                        rmsnorm_to_shared<T>(haddr, hid_s, p.norm_weight, p.norm_eps, d, partial, kBarHidden, tid, nc, lane, warp,
+                        rmsnorm_to_shared<T>(haddr, norm_s, norm_w, p.norm_eps, d, partial, kBarHidden, tid, nc, lane, warp,
                                              nwarps);
                     {
                         if constexpr (NFAST > 0) sweep.chunk(smem_base + m.off_wr, raddr, d, tid, nc);

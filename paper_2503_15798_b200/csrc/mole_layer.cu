@@ -2,9 +2,12 @@
 // for a single layer and for a chained L-layer decode step (Eq. 4 and Eq. 8 of arXiv
 // 2503.15798).  The kernel itself is in mole_kernel.cuh.
 #include <atomic>
+#include <mutex>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
+#include "mole_decode.cuh"
 #include "mole_kernel.cuh"
 
 namespace mole {
@@ -21,25 +24,67 @@ void set_cuda_error(cudaError_t e)
 
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-constexpr int kNumSMs = 148;                  // B200; the launch asks the device for its own count
+constexpr int kNumSMs = 148;                  // B200; used when no device can be asked (mole_plan on a machine without one)
 constexpr int kSmemPerBlockMax = 227 * 1024;  // opt-in limit per block
 constexpr int kSmemPerSM = 228 * 1024;        // per SM, of which every resident block reserves 1 KB
 constexpr long long kFusedMaxTokens = 4096;   // above this a step runs as L chained launches
+constexpr long long kDecodeKernelMaxTokens = 2048;  // single-layer launches up to here take the one-block-per-token kernel
+
+// ---- debugging aids: the MOLE_FORCE_* / MOLE_DEBUG_* variables, read once ---------------------------
+struct DebugEnv {
+    int lanes, column_chunks, target_blocks, stages, blocks_per_sm, kernel;
+    long long wait_limit;
+};
+static std::mutex g_env_mutex;
+static DebugEnv g_env;
+static std::atomic<int> g_env_generation{0};  // 0: not read yet; bumped by every (re)load
+
+static int env_int(const char *name)
+{
+    const char *f = getenv(name);
+    return f ? atoi(f) : 0;
+}
+static void load_env_locked()
+{
+    g_env.lanes = env_int("MOLE_FORCE_LANES");
+    g_env.column_chunks = env_int("MOLE_FORCE_COLUMN_CHUNKS");
+    g_env.target_blocks = env_int("MOLE_FORCE_TARGET_BLOCKS");
+    g_env.stages = env_int("MOLE_FORCE_STAGES");
+    g_env.blocks_per_sm = env_int("MOLE_FORCE_BLOCKS_PER_SM");
+    g_env.kernel = env_int("MOLE_FORCE_KERNEL");
+    const char *w = getenv("MOLE_DEBUG_WAIT_LIMIT");
+    g_env.wait_limit = w ? atoll(w) : 0;
+    g_env_generation.fetch_add(1);
+}
+static DebugEnv debug_env(int *generation = nullptr)
+{
+    std::lock_guard<std::mutex> lock(g_env_mutex);
+    if (g_env_generation.load() == 0) load_env_locked();
+    if (generation) *generation = g_env_generation.load();
+    return g_env;
+}
+// polls after which a device-side wait gives up: the default, or what MOLE_DEBUG_WAIT_LIMIT says
+// (n >= 1: n polls; negative: none at all, every wait that is not satisfied at once gives up)
+static uint32_t wait_polls_from(const DebugEnv &e)
+{
+    if (e.wait_limit < 0) return 0u;
+    if (e.wait_limit > 0) return e.wait_limit > 0x7fffffffLL ? 0x7fffffffu : static_cast<uint32_t>(e.wait_limit);
+    return kWaitPolls;
+}
 
 // Lanes per 16-byte column group in the combine (1, 2 or 4).
-static int env_int(const char *name);
-static int lanes_per_group(int dcc, int vec)
+static int lanes_per_group(int dcc, int vec, const DebugEnv &env)
 {
     const int groups = dcc / vec;
-    const int forced = env_int("MOLE_FORCE_LANES");  // debugging aid
+    const int forced = env.lanes;
     if ((forced == 1 || forced == 2 || forced == 4) && groups * forced <= kMaxConsumers) return forced;
     // about four compute warps -- one per SM sub-partition -- measured best: more warps repeat the
     // per-item bookkeeping, fewer lengthen the chain of an item
     return groups * 4 <= 128 ? 4 : (groups * 2 <= 128 ? 2 : 1);
 }
-static int consumers_for(int dcc, int vec)
+static int consumers_for(int dcc, int vec, const DebugEnv &env)
 {
-    const int lanes = (dcc / vec) * lanes_per_group(dcc, vec);
+    const int lanes = (dcc / vec) * lanes_per_group(dcc, vec, env);
     return round_up(lanes < kMaxConsumers ? lanes : kMaxConsumers, 32);
 }
 // Several chunks per item: the rows are cut by experts -- whole rows, one bulk copy per chunk --
@@ -51,11 +96,11 @@ static int groups_per_lane(int d, int vec)
     const int groups = d / vec;
     return groups <= 128 ? 1 : (groups <= 256 ? 2 : 4);
 }
-static bool rows_by_expert(int dtype, int N, int d, int K, int in_ring, bool by_columns = false)
+static bool rows_by_expert(int dtype, int N, int d, int K, int in_ring, bool by_columns, const DebugEnv &env)
 {
     if (by_columns) return false;
     const bool n_fast = N == 4 || N == 8 || N == 16 || N == 32 || N == 64;
-    if (env_int("MOLE_FORCE_COLUMN_CHUNKS") > 0) return false;  // debugging aid
+    if (env.column_chunks > 0) return false;  // debugging aid
     return dtype == MOLE_DTYPE_BF16 && n_fast && K > 1 && N % K == 0 && in_ring && d / 8 <= 4 * 128;
 }
 static int consumers_by_expert(int d, int vec)
@@ -63,16 +108,13 @@ static int consumers_by_expert(int d, int vec)
     const int gpl = groups_per_lane(d, vec);
     return round_up((d / vec + gpl - 1) / gpl, 32);
 }
-static int env_int(const char *name)  // debugging aids: MOLE_FORCE_* override parts of the plan
-{
-    const char *f = getenv(name);
-    return f ? atoi(f) : 0;
-}
 
-int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns)
+int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan *plan, bool by_columns, int sms, bool norm)
 {
     if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
     if (L < 1 || M < 0) return MOLE_ERR_INVALID_ARG;
+    if (sms < 1) sms = kNumSMs;
+    const DebugEnv env = debug_env();
     const int eb = elem_bytes(dtype), vec = 16 / eb;
     if (N < 1 || N > kMaxN || d < vec || d % vec != 0) return MOLE_ERR_UNSUPPORTED_SHAPE;
     // the router matrix stays resident only for a single layer, and only if it leaves room for the ring
@@ -81,8 +123,9 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     auto total_smem = [&](int K, int stages) {
         const int dcc = d / K;
         const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
-        const int consumers = rows_by_expert(dtype, N, d, K, in_ring, by_columns) ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
-        return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers).total;
+        const int consumers = rows_by_expert(dtype, N, d, K, in_ring, by_columns, env) ? consumers_by_expert(d, vec)
+                                                                                         : consumers_for(dcc, vec, env);
+        return smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers, norm ? 1 : 0).total;
     };
     int K;
     if (d_split != 0) {
@@ -95,7 +138,7 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
         // launch of at most one token per SM has the SM's whole shared memory for one block: chunks of up
         // to 64 KB in a ring of three then halve the per-chunk bookkeeping (measured on d = 2048, N = 32,
         // 16 layers, 1 to 148 tokens: 84 -> 56-62 us per step; chained single-layer launches 3 - 12 % less)
-        const bool roomy = M <= kNumSMs && (L > 1 || in_ring);
+        const bool roomy = M <= sms && (L > 1 || in_ring);
         const long long chunk_cap = roomy ? 64 * 1024 : 32 * 1024;
         const int ring_min = roomy ? 3 : 2;
         K = 1;
@@ -109,32 +152,34 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
         }
     }
     const int dcc = d / K;
-    const bool by_expert = rows_by_expert(dtype, N, d, K, in_ring, by_columns);
-    const int consumers = by_expert ? consumers_by_expert(d, vec) : consumers_for(dcc, vec);
+    const bool by_expert = rows_by_expert(dtype, N, d, K, in_ring, by_columns, env);
+    const int consumers = by_expert ? consumers_by_expert(d, vec) : consumers_for(dcc, vec, env);
     // Resident blocks per SM aimed at: one per token while tokens are few (each with the deepest ring
     // that fits), up to four token chains per SM when there are many (shallower rings, more overlap).
-    int want = static_cast<int>((M + kNumSMs - 1) / kNumSMs);
+    int want = static_cast<int>((M + sms - 1) / sms);
     want = want < 1 ? 1 : (want > 4 ? 4 : want);
-    if (env_int("MOLE_FORCE_TARGET_BLOCKS") > 0) want = env_int("MOLE_FORCE_TARGET_BLOCKS");
+    if (env.target_blocks > 0) want = env.target_blocks;
     int stages = 0;
     for (; want >= 1 && stages == 0; --want) {
         const uint32_t budget = static_cast<uint32_t>(kSmemPerSM / want - 1024);
-        for (int s = kMaxStages; s >= 2; --s)
-            if (total_smem(K, s) <= budget && total_smem(K, s) <= static_cast<uint32_t>(kSmemPerBlockMax)) {
+        for (int s = kMaxStages; s >= 2; --s) {
+            const uint32_t need = total_smem(K, s);
+            if (need <= budget && need <= static_cast<uint32_t>(kSmemPerBlockMax)) {
                 stages = s;
                 break;
             }
+        }
     }
     if (stages == 0) stages = 2;  // total_smem(K, 2) fits a block (checked above)
     // no deeper than the chunks a block will see
-    const long long cap = static_cast<long long>(kNumSMs) * 4;
+    const long long cap = static_cast<long long>(sms) * 4;
     const long long blocks = M < cap ? (M > 0 ? M : 1) : cap;
     const long long chunks = ((M + blocks - 1) / blocks) * per_tok * K;
     if (stages > chunks) stages = chunks < 2 ? 2 : static_cast<int>(chunks);
-    const int forced = env_int("MOLE_FORCE_STAGES");
+    const int forced = env.stages;
     if (forced >= 2 && forced <= kMaxStages && total_smem(K, forced) <= static_cast<uint32_t>(kSmemPerBlockMax)) stages = forced;
     const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;
-    const SmemMap m = smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers);
+    const SmemMap m = smem_map(N, d, dcc, eb, stages, hring, in_ring, consumers, norm ? 1 : 0);
     plan->d_split = K;
     plan->dc = dcc;
     plan->consumers = consumers;
@@ -150,101 +195,141 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     if (per_sm < 1) per_sm = 1;
     plan->blocks_per_sm = per_sm;
     plan->rows_by_expert = by_expert ? 1 : 0;
-    plan->lanes = by_expert ? groups_per_lane(d, vec) : lanes_per_group(dcc, vec);
+    plan->lanes = by_expert ? groups_per_lane(d, vec) : lanes_per_group(dcc, vec, env);
     plan->n_fast = (N == 4 || N == 8 || N == 16 || N == 32 || N == 64) ? N : 0;
     return MOLE_OK;
 }
 
+// A kernel instantiation and its name ("step<storage,NFAST,P,MODE,SHAPE,DIRECT,NORM>" for the ring
+// kernel, "decode<N,NORM>" for the one-block-per-token kernel): what mole_variant() reports, so that a
+// test can tell which instantiations a workload reaches.
 typedef void (*StepKernel)(const StepParams);
+typedef void (*DecodeKernel)(const DecodeParams);
+struct Variant {
+    StepKernel fn;
+    const char *name;
+};
+#define MOLE_V(T, TN, NF, P, MODE, SHAPE, DIRECT, NORM) \
+    Variant { mole_step_kernel<T, NF, P, MODE, SHAPE, DIRECT, NORM>, "step<" TN "," #NF "," #P "," #MODE "," #SHAPE "," #DIRECT "," #NORM ">" }
+#define MOLE_VB(NF, P, MODE, SHAPE, DIRECT, NORM) MOLE_V(__nv_bfloat16, "bf16", NF, P, MODE, SHAPE, DIRECT, NORM)
+#define MOLE_VF(NF, P, MODE, SHAPE, DIRECT, NORM) MOLE_V(float, "f32", NF, P, MODE, SHAPE, DIRECT, NORM)
+static const Variant kNoVariant = {nullptr, "none"};
 
-template <typename T, int P, int MODE>
-static StepKernel pick_n(int n_fast)
-{
-    switch (n_fast) {
-        case 4: return mole_step_kernel<T, 4, P, MODE, 0>;
-        case 8: return mole_step_kernel<T, 8, P, MODE, 0>;
-        case 16: return mole_step_kernel<T, 16, P, MODE, 0>;
-        case 32: return mole_step_kernel<T, 32, P, MODE, 0>;
-        case 64: return mole_step_kernel<T, 64, P, MODE, 0>;
-        default: return nullptr;
+// bf16, compile-time launch flags (MODE 1, 2, 3), any of the unrolled N
+#define MOLE_PICK_N_BF16(P, MODE, NORM)                      \
+    switch (n_fast) {                                        \
+        case 4: return MOLE_VB(4, P, MODE, 0, 0, NORM);      \
+        case 8: return MOLE_VB(8, P, MODE, 0, 0, NORM);      \
+        case 16: return MOLE_VB(16, P, MODE, 0, 0, NORM);    \
+        case 32: return MOLE_VB(32, P, MODE, 0, 0, NORM);    \
+        case 64: return MOLE_VB(64, P, MODE, 0, 0, NORM);    \
+        default: return kNoVariant;                          \
     }
-}
-
-template <typename T, int MODE>
-static StepKernel pick_p(int n_fast, int lanes)
+#define MOLE_PICK_N_F32(P, MODE, NORM)                       \
+    switch (n_fast) {                                        \
+        case 4: return MOLE_VF(4, P, MODE, 0, 0, NORM);      \
+        case 8: return MOLE_VF(8, P, MODE, 0, 0, NORM);      \
+        case 16: return MOLE_VF(16, P, MODE, 0, 0, NORM);    \
+        case 32: return MOLE_VF(32, P, MODE, 0, 0, NORM);    \
+        case 64: return MOLE_VF(64, P, MODE, 0, 0, NORM);    \
+        default: return kNoVariant;                          \
+    }
+template <int MODE>
+static Variant pick_bf16(int n_fast, int lanes)
 {
-    return lanes == 4 ? pick_n<T, 4, MODE>(n_fast) : (lanes == 2 ? pick_n<T, 2, MODE>(n_fast) : pick_n<T, 1, MODE>(n_fast));
+    if (lanes == 4) { MOLE_PICK_N_BF16(4, MODE, 0) }
+    if (lanes == 2) { MOLE_PICK_N_BF16(2, MODE, 0) }
+    MOLE_PICK_N_BF16(1, MODE, 0)
+}
+static Variant pick_f32(int n_fast, int lanes)
+{
+    if (lanes == 4) { MOLE_PICK_N_F32(4, 0, 0) }
+    if (lanes == 2) { MOLE_PICK_N_F32(2, 0, 0) }
+    MOLE_PICK_N_F32(1, 0, 0)
 }
 
 // The generic-N router and the fp32 storage type exist only with run-time flags (MODE 0); bf16 with
-// a compiled-in N also in the three specialised shapes.
-static StepKernel pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers,
-                              int by_expert, bool direct)
+// a compiled-in N also in the specialised shapes.
+static Variant pick_kernel(int dtype, int n_fast, int lanes, int chunks, int in_ring, int d, int dcc, int consumers,
+                           int by_expert, bool direct)
 {
     // the layer widths of the paper's Table 2 (160M, 410M and 1B models) with their sizes compiled in;
     // `direct`: single-layer launches of 128 tokens up to one token per resident block, where the compute
     // warps loading the hidden state themselves measured 6 % faster per chained layer (slower below)
     if (dtype == MOLE_DTYPE_BF16) {
         if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 768 && consumers == 96)
-            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 1>
-                           : (direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1>);
+            return in_ring ? MOLE_VB(16, 1, 1, 1, 0, 0) : (direct ? MOLE_VB(16, 1, 2, 1, 1, 0) : MOLE_VB(16, 1, 2, 1, 0, 0));
         if (n_fast == 16 && lanes == 1 && chunks == 1 && d == 1024 && consumers == 128)
-            return in_ring ? mole_step_kernel<__nv_bfloat16, 16, 1, 1, 2>
-                           : (direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2>);
+            return in_ring ? MOLE_VB(16, 1, 1, 2, 0, 0) : (direct ? MOLE_VB(16, 1, 2, 2, 1, 0) : MOLE_VB(16, 1, 2, 2, 0, 0));
         if (n_fast == 32 && lanes == 2 && chunks == 4 && d == 2048 && dcc == 512 && consumers == 128 && by_expert)
-            return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 3>;
+            return MOLE_VB(32, 2, 3, 3, 0, 0);
         if (n_fast == 32 && lanes == 2 && chunks == 2 && d == 2048 && dcc == 1024 && consumers == 128 && by_expert)
-            return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 4>;
-        if (by_expert) return pick_p<__nv_bfloat16, 3>(n_fast, lanes);
+            return MOLE_VB(32, 2, 3, 4, 0, 0);
+        if (by_expert) return pick_bf16<3>(n_fast, lanes);
     }
     if (n_fast == 0) {
         if (dtype == MOLE_DTYPE_BF16)
-            return lanes == 4 ? mole_step_kernel<__nv_bfloat16, 0, 4, 0, 0> : (lanes == 2 ? mole_step_kernel<__nv_bfloat16, 0, 2, 0, 0> : mole_step_kernel<__nv_bfloat16, 0, 1, 0, 0>);
-        return lanes == 4 ? mole_step_kernel<float, 0, 4, 0, 0> : (lanes == 2 ? mole_step_kernel<float, 0, 2, 0, 0> : mole_step_kernel<float, 0, 1, 0, 0>);
+            return lanes == 4 ? MOLE_VB(0, 4, 0, 0, 0, 0) : (lanes == 2 ? MOLE_VB(0, 2, 0, 0, 0, 0) : MOLE_VB(0, 1, 0, 0, 0, 0));
+        return lanes == 4 ? MOLE_VF(0, 4, 0, 0, 0, 0) : (lanes == 2 ? MOLE_VF(0, 2, 0, 0, 0, 0) : MOLE_VF(0, 1, 0, 0, 0, 0));
     }
-    if (dtype != MOLE_DTYPE_BF16) return pick_p<float, 0>(n_fast, lanes);
-    if (chunks == 1) return in_ring ? pick_p<__nv_bfloat16, 1>(n_fast, lanes) : pick_p<__nv_bfloat16, 2>(n_fast, lanes);
-    return pick_p<__nv_bfloat16, 0>(n_fast, lanes);
+    if (dtype != MOLE_DTYPE_BF16) return pick_f32(n_fast, lanes);
+    if (chunks == 1) return in_ring ? pick_bf16<1>(n_fast, lanes) : pick_bf16<2>(n_fast, lanes);
+    return pick_bf16<0>(n_fast, lanes);
 }
 
-// The kernels whose router reads RMSNorm(hidden): run-time launch flags, rows cut by columns.
-template <typename T, int P>
-static StepKernel pick_norm_n(int n_fast)
+// The kernels whose router reads RMSNorm(hidden): run-time launch flags, rows cut by columns ...
+static Variant pick_norm_kernel(int dtype, int n_fast, int lanes)
 {
-    switch (n_fast) {
-        case 0: return mole_step_kernel<T, 0, P, 0, 0, 0, 1>;
-        case 4: return mole_step_kernel<T, 4, P, 0, 0, 0, 1>;
-        case 8: return mole_step_kernel<T, 8, P, 0, 0, 0, 1>;
-        case 16: return mole_step_kernel<T, 16, P, 0, 0, 0, 1>;
-        case 32: return mole_step_kernel<T, 32, P, 0, 0, 0, 1>;
-        case 64: return mole_step_kernel<T, 64, P, 0, 0, 0, 1>;
-        default: return nullptr;
+    if (dtype == MOLE_DTYPE_BF16) {
+        if (n_fast == 0) return lanes == 4 ? MOLE_VB(0, 4, 0, 0, 0, 1) : (lanes == 2 ? MOLE_VB(0, 2, 0, 0, 0, 1) : MOLE_VB(0, 1, 0, 0, 0, 1));
+        if (lanes == 4) { MOLE_PICK_N_BF16(4, 0, 1) }
+        if (lanes == 2) { MOLE_PICK_N_BF16(2, 0, 1) }
+        MOLE_PICK_N_BF16(1, 0, 1)
     }
+    if (n_fast == 0) return lanes == 4 ? MOLE_VF(0, 4, 0, 0, 0, 1) : (lanes == 2 ? MOLE_VF(0, 2, 0, 0, 0, 1) : MOLE_VF(0, 1, 0, 0, 0, 1));
+    if (lanes == 4) { MOLE_PICK_N_F32(4, 0, 1) }
+    if (lanes == 2) { MOLE_PICK_N_F32(2, 0, 1) }
+    MOLE_PICK_N_F32(1, 0, 1)
 }
 // ... and, for the single-layer launches of the paper's three layer widths, with the sizes compiled in
-static StepKernel pick_norm_shape_kernel(const StepPlan &plan, int dtype, int d, bool direct)
+static Variant pick_norm_shape_kernel(const StepPlan &plan, int dtype, int d, bool direct)
 {
-    if (dtype != MOLE_DTYPE_BF16) return nullptr;
+    if (dtype != MOLE_DTYPE_BF16) return kNoVariant;
     if (plan.n_fast == 16 && plan.lanes == 1 && plan.d_split == 1 && !plan.wr_in_ring) {
-        if (d == 768 && plan.consumers == 96)
-            return direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 1, 0, 1>;
-        if (d == 1024 && plan.consumers == 128)
-            return direct ? mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 1, 1> : mole_step_kernel<__nv_bfloat16, 16, 1, 2, 2, 0, 1>;
+        if (d == 768 && plan.consumers == 96) return direct ? MOLE_VB(16, 1, 2, 1, 1, 1) : MOLE_VB(16, 1, 2, 1, 0, 1);
+        if (d == 1024 && plan.consumers == 128) return direct ? MOLE_VB(16, 1, 2, 2, 1, 1) : MOLE_VB(16, 1, 2, 2, 0, 1);
     }
     if (plan.n_fast == 32 && plan.lanes == 2 && plan.d_split == 4 && d == 2048 && plan.dc == 512 && plan.consumers == 128 &&
         plan.rows_by_expert)
-        return mole_step_kernel<__nv_bfloat16, 32, 2, 3, 3, 0, 1>;
-    return nullptr;
+        return MOLE_VB(32, 2, 3, 3, 0, 1);
+    return kNoVariant;
 }
-static StepKernel pick_norm_kernel(int dtype, int n_fast, int lanes)
+
+// The one-block-per-token kernel (mole_decode.cuh): bf16, N of 4, 8, 16 or 32, d a multiple of 128
+// with d / 4 threads, a single layer, the launch's own chunking (d_split 0), up to 2048 tokens.
+struct DecodeVariant {
+    DecodeKernel fn;
+    const char *name;
+};
+static bool decode_shape_ok(int dtype, int N, int d)
 {
-    if (dtype == MOLE_DTYPE_BF16)
-        return lanes == 4 ? pick_norm_n<__nv_bfloat16, 4>(n_fast) : (lanes == 2 ? pick_norm_n<__nv_bfloat16, 2>(n_fast) : pick_norm_n<__nv_bfloat16, 1>(n_fast));
-    return lanes == 4 ? pick_norm_n<float, 4>(n_fast) : (lanes == 2 ? pick_norm_n<float, 2>(n_fast) : pick_norm_n<float, 1>(n_fast));
+    if (dtype != MOLE_DTYPE_BF16 || d % 128 != 0) return false;
+    if (N != 4 && N != 8 && N != 16 && N != 32) return false;
+    return d / 4 <= decode_max_threads(N) && decode_smem_bytes(N, d) <= static_cast<uint32_t>(kSmemPerBlockMax);
+}
+static DecodeVariant pick_decode(int N, bool norm)
+{
+    switch (N) {
+        case 4: return norm ? DecodeVariant{mole_decode_kernel<4, 1>, "decode<4,1>"} : DecodeVariant{mole_decode_kernel<4, 0>, "decode<4,0>"};
+        case 8: return norm ? DecodeVariant{mole_decode_kernel<8, 1>, "decode<8,1>"} : DecodeVariant{mole_decode_kernel<8, 0>, "decode<8,0>"};
+        case 16: return norm ? DecodeVariant{mole_decode_kernel<16, 1>, "decode<16,1>"} : DecodeVariant{mole_decode_kernel<16, 0>, "decode<16,0>"};
+        case 32: return norm ? DecodeVariant{mole_decode_kernel<32, 1>, "decode<32,1>"} : DecodeVariant{mole_decode_kernel<32, 0>, "decode<32,0>"};
+        default: return DecodeVariant{nullptr, "none"};
+    }
 }
 
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
-static int ensure_smem(StepKernel k, int smem)
+static int ensure_smem(const void *fn, int smem)
 {
     if (smem <= 48 * 1024) return MOLE_OK;
     struct Slot {
@@ -252,10 +337,9 @@ static int ensure_smem(StepKernel k, int smem)
         std::atomic<int> dev{-1};
         std::atomic<int> bytes{0};
     };
-    static Slot slots[128];
+    static Slot slots[256];
     int dev = 0;
     MOLE_CUDA_TRY(cudaGetDevice(&dev));
-    const void *fn = reinterpret_cast<const void *>(k);
     for (auto &sl : slots) {
         if (sl.fn.load() == fn && sl.dev.load() == dev && sl.bytes.load() >= smem) return MOLE_OK;
     }
@@ -276,11 +360,12 @@ static int ensure_smem(StepKernel k, int smem)
 }
 
 // SM count of the current device, asked once per device.
-static int sm_count(int *out)
+static int sm_count(int *out, int *dev_out = nullptr)
 {
     static std::atomic<int> cache[64];
     int dev = 0;
     MOLE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev_out) *dev_out = dev;
     if (dev >= 0 && dev < 64 && cache[dev].load() > 0) {
         *out = cache[dev].load();
         return MOLE_OK;
@@ -293,40 +378,168 @@ static int sm_count(int *out)
     return MOLE_OK;
 }
 
+// Everything about a launch that depends only on its shape: found once, then looked up.
+struct ShapeKey {
+    long long M;
+    int L, N, d, dtype, d_split, norm, kernel, dev, env_generation;
+    bool operator==(const ShapeKey &o) const
+    {
+        return M == o.M && L == o.L && N == o.N && d == o.d && dtype == o.dtype && d_split == o.d_split && norm == o.norm &&
+               kernel == o.kernel && dev == o.dev && env_generation == o.env_generation;
+    }
+};
+struct LaunchChoice {
+    bool decode;        // the one-block-per-token kernel; otherwise the ring kernel with `plan`
+    StepPlan plan;
+    StepKernel step_fn;
+    DecodeKernel decode_fn;
+    const char *name;
+    int threads, smem;
+    long long grid;
+    uint32_t wait_polls;
+};
+
+// `sms` / `dev` < 0: no device is asked (nominal B200 figures, nothing is prepared for a launch).
+static int choose_launch(long long M, int L, int N, int d, int dtype, int d_split, bool norm, int kernel, int sms, bool prepare,
+                         LaunchChoice *c)
+{
+    int generation = 0;
+    const DebugEnv env = debug_env(&generation);
+    if (kernel == MOLE_KERNEL_AUTO && env.kernel > 0) kernel = env.kernel;
+    if (kernel != MOLE_KERNEL_AUTO && kernel != MOLE_KERNEL_RING && kernel != MOLE_KERNEL_DECODE) return MOLE_ERR_INVALID_ARG;
+    c->wait_polls = wait_polls_from(env);
+    StepPlan plan;
+    int rc = plan_step(M, L, N, d, dtype, d_split, &plan, false, sms, norm);  // also validates the shape
+    if (rc != MOLE_OK) return rc;
+    const bool decode_ok = L == 1 && d_split == 0 && decode_shape_ok(dtype, N, d);
+    if (kernel == MOLE_KERNEL_DECODE && !decode_ok) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    if (decode_ok && (kernel == MOLE_KERNEL_DECODE || (kernel == MOLE_KERNEL_AUTO && M <= kDecodeKernelMaxTokens))) {
+        const DecodeVariant v = pick_decode(N, norm);
+        if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        c->decode = true;
+        c->plan = plan;
+        c->step_fn = nullptr;
+        c->decode_fn = v.fn;
+        c->name = v.name;
+        c->threads = d / 4;
+        c->smem = static_cast<int>(decode_smem_bytes(N, d));
+        c->grid = M;
+        if (prepare) return ensure_smem(reinterpret_cast<const void *>(v.fn), c->smem);
+        return MOLE_OK;
+    }
+    const bool direct = M >= 128 && M <= 4LL * sms;  // see pick_kernel
+    Variant v = kNoVariant;
+    if (norm) {
+        if (L == 1) v = pick_norm_shape_kernel(plan, dtype, d, direct);
+        if (!v.fn) {
+            rc = plan_step(M, L, N, d, dtype, d_split, &plan, true, sms, true);  // the general kernels cut the rows by columns
+            if (rc != MOLE_OK) return rc;
+            v = pick_norm_kernel(dtype, plan.n_fast, plan.lanes);
+        }
+    } else {
+        v = pick_kernel(dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, d, plan.dc, plan.consumers, plan.rows_by_expert,
+                        direct);
+    }
+    if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    c->decode = false;
+    c->plan = plan;
+    c->step_fn = v.fn;
+    c->decode_fn = nullptr;
+    c->name = v.name;
+    c->threads = plan.threads;
+    c->smem = plan.smem;
+    int per_sm = plan.blocks_per_sm;
+    if (prepare) {
+        rc = ensure_smem(reinterpret_cast<const void *>(v.fn), plan.smem);
+        if (rc != MOLE_OK) return rc;
+        // a persistent grid: as many blocks as fit at once, never more than the tokens
+        MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, v.fn, plan.threads, plan.smem));
+    }
+    if (per_sm < 1) per_sm = 1;
+    if (env.blocks_per_sm >= 1 && env.blocks_per_sm < per_sm) per_sm = env.blocks_per_sm;
+    c->grid = static_cast<long long>(per_sm) * sms;
+    if (c->grid > M) c->grid = M;
+    return MOLE_OK;
+}
+
+// The calling thread's last few shapes (a decoding loop repeats a handful of them).
+static int cached_launch(const StepLaunch &a, const LaunchChoice **out)
+{
+    constexpr int kEntries = 32;
+    struct Entry {
+        bool used = false;
+        ShapeKey key;
+        LaunchChoice choice;
+    };
+    thread_local Entry cache[kEntries];
+    thread_local int next = 0;
+    int sms = kNumSMs, dev = 0;
+    int rc = sm_count(&sms, &dev);
+    if (rc != MOLE_OK) return rc;
+    int generation = 0;
+    (void)debug_env(&generation);
+    const ShapeKey key = {a.M, a.L, a.N, a.d, a.dtype, a.d_split, a.norm_weight ? 1 : 0, a.kernel, dev, generation};
+    for (int i = 0; i < kEntries; ++i)
+        if (cache[i].used && cache[i].key == key) {
+            *out = &cache[i].choice;
+            return MOLE_OK;
+        }
+    LaunchChoice c;
+    rc = choose_launch(a.M, a.L, a.N, a.d, a.dtype, a.d_split, a.norm_weight != nullptr, a.kernel, sms, true, &c);
+    if (rc != MOLE_OK) return rc;
+    Entry &e = cache[next];
+    next = (next + 1) % kEntries;
+    e.used = true;
+    e.key = key;
+    e.choice = c;
+    *out = &e.choice;
+    return MOLE_OK;
+}
+
 int launch_step(const StepLaunch &a)
 {
     if (a.M == 0) return MOLE_OK;
-    StepPlan plan;
-    const bool norm = a.norm_weight != nullptr;
-    if (norm && a.L != 1) return MOLE_ERR_INVALID_ARG;
-    int rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan);
-    if (rc != MOLE_OK) return rc;
     if (a.M * a.L > 0x3fffffffLL) return MOLE_ERR_TOO_LARGE;
-    int sms = kNumSMs;
-    rc = sm_count(&sms);
+    const LaunchChoice *c = nullptr;
+    int rc = cached_launch(a, &c);
     if (rc != MOLE_OK) return rc;
-    StepKernel k_norm = nullptr;
-    const bool direct = a.M >= 128 && a.M <= 4LL * sms;  // see pick_kernel
-    if (norm && !(k_norm = pick_norm_shape_kernel(plan, a.dtype, a.d, direct))) {
-        rc = plan_step(a.M, a.L, a.N, a.d, a.dtype, a.d_split, &plan, true);  // the general kernels cut the rows by columns
-        if (rc != MOLE_OK) return rc;
-        k_norm = pick_norm_kernel(a.dtype, plan.n_fast, plan.lanes);
-    }
-    StepKernel k = norm ? k_norm
-                        : pick_kernel(a.dtype, plan.n_fast, plan.lanes, plan.d_split, plan.wr_in_ring, a.d, plan.dc, plan.consumers,
-                                      plan.rows_by_expert, direct);
-    if (!k) return MOLE_ERR_UNSUPPORTED_SHAPE;
-    rc = ensure_smem(k, plan.smem);
-    if (rc != MOLE_OK) return rc;
-    // a persistent grid: as many blocks as fit at once never more than the tokens
-    int per_sm = 0;
-    MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, plan.threads, plan.smem));
-    if (per_sm < 1) per_sm = 1;
-    if (env_int("MOLE_FORCE_BLOCKS_PER_SM") >= 1 && env_int("MOLE_FORCE_BLOCKS_PER_SM") < per_sm)
-        per_sm = env_int("MOLE_FORCE_BLOCKS_PER_SM");
-    long long grid = static_cast<long long>(per_sm) * sms;
-    if (grid > a.M) grid = a.M;
 
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(c->grid), 1, 1);
+    cfg.blockDim = dim3(c->threads, 1, 1);
+    cfg.dynamicSmemBytes = c->smem;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attrs[1];
+    unsigned na = 0;
+    if (a.flags & MOLE_FLAG_CHAIN) {
+        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = na;
+
+    if (c->decode) {
+        DecodeParams p;
+        p.hidden = a.hidden;
+        p.residual = a.residual;
+        p.row_index = a.row_index;
+        p.lut = a.lut;
+        p.w_router = a.w_router;
+        p.norm_weight = a.norm_weight;
+        p.out = a.out;
+        p.gates_out = a.gates_out;
+        p.status = a.status;
+        p.rows = a.rows;
+        p.d = a.d;
+        p.norm_eps = a.norm_eps;
+        p.flags = a.flags;
+        p.wait_polls = c->wait_polls;
+        MOLE_CUDA_TRY(cudaLaunchKernelEx(&cfg, c->decode_fn, p));
+        return MOLE_OK;
+    }
+    const StepPlan &plan = c->plan;
     StepParams p;
     p.hidden = a.hidden;
     p.residual = a.residual;
@@ -334,6 +547,7 @@ int launch_step(const StepLaunch &a)
     p.lut = a.lut;
     p.w_router = a.w_router;
     p.norm_weight = a.norm_weight;
+    p.norm_stride = a.norm_stride;
     p.norm_eps = a.norm_eps;
     p.out = a.out;
     p.gates_out = a.gates_out;
@@ -352,23 +566,8 @@ int launch_step(const StepLaunch &a)
     p.wr_in_ring = plan.wr_in_ring;
     p.consumers = plan.consumers;
     p.flags = a.flags;
-
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
-    cfg.blockDim = dim3(plan.threads, 1, 1);
-    cfg.dynamicSmemBytes = plan.smem;
-    cfg.stream = a.stream;
-    cudaLaunchAttribute attrs[1];
-    unsigned na = 0;
-    if (a.flags & MOLE_FLAG_CHAIN) {
-        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attrs[na].val.programmaticStreamSerializationAllowed = 1;
-        ++na;
-    }
-    cfg.attrs = attrs;
-    cfg.numAttrs = na;
-    MOLE_CUDA_TRY(cudaLaunchKernelEx(&cfg, k, p));
+    p.wait_polls = c->wait_polls;
+    MOLE_CUDA_TRY(cudaLaunchKernelEx(&cfg, c->step_fn, p));
     return MOLE_OK;
 }
 
@@ -396,7 +595,8 @@ int mole_layer_forward_ex(const mole_args *a)
 {
     if (!a || a->struct_size != sizeof(mole_args)) return MOLE_ERR_INVALID_ARG;
     if (a->flags & ~(MOLE_FLAG_IDS_INT64 | MOLE_FLAG_CHAIN)) return MOLE_ERR_INVALID_ARG;
-    if (a->reserved != 0 || a->reserved2 != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->reserved2 != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->kernel != MOLE_KERNEL_AUTO && a->kernel != MOLE_KERNEL_RING && a->kernel != MOLE_KERNEL_DECODE) return MOLE_ERR_INVALID_ARG;
     if (a->norm_weight && (!aligned16(a->norm_weight) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f)) return MOLE_ERR_INVALID_ARG;
     int rc = check_common(a->hidden, a->ids, a->lut, a->w_router, a->out, a->residual, a->B, a->T, a->N, a->d, a->V,
                           a->dtype);
@@ -426,6 +626,7 @@ int mole_layer_forward_ex(const mole_args *a)
     s.stream = static_cast<cudaStream_t>(a->stream);
     s.norm_weight = a->norm_weight;
     s.norm_eps = a->norm_eps;
+    s.kernel = a->kernel;
     return launch_step(s);
 }
 
@@ -450,59 +651,106 @@ int mole_layer_forward(const void *hidden, const int32_t *ids, const void *lut, 
     return mole_layer_forward_ex(&a);
 }
 
-int mole_decode_step_ex(const void *hidden_in, const int32_t *ids, const void *lut_base, int64_t lut_layer_stride_bytes,
-                        const void *w_router_base, int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status,
-                        int L, int B, int T, int N, int d, int V, int dtype, int mode, int d_split, void *stream)
+int mole_decode_step_args(const mole_step_args *a)
 {
+    if (!a || a->struct_size != sizeof(mole_step_args)) return MOLE_ERR_INVALID_ARG;
+    if ((a->flags & ~MOLE_FLAG_CHAIN) || a->reserved != 0) return MOLE_ERR_INVALID_ARG;
+    const int L = a->L;
+    int mode = a->mode;
     if (L < 1 || mode < MOLE_STEP_AUTO || mode > MOLE_STEP_CHAINED) return MOLE_ERR_INVALID_ARG;
-    int rc = check_common(hidden_in, ids, lut_base, w_router_base, out, nullptr, B, T, N, d, V, dtype);
+    if (a->kernel != MOLE_KERNEL_AUTO && a->kernel != MOLE_KERNEL_RING && a->kernel != MOLE_KERNEL_DECODE) return MOLE_ERR_INVALID_ARG;
+    int rc = check_common(a->hidden_in, a->ids, a->lut_base, a->w_router_base, a->out, nullptr, a->B, a->T, a->N, a->d, a->V,
+                          a->dtype);
     if (rc != MOLE_OK) return rc;
-    const long long M = static_cast<long long>(B) * T;
+    const long long M = static_cast<long long>(a->B) * a->T;
     if (M == 0) return MOLE_OK;
-    if ((lut_layer_stride_bytes & 15) || (wr_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if ((a->lut_layer_stride_bytes & 15) || (a->wr_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if (a->norm_weight_base &&
+        (!aligned16(a->norm_weight_base) || (a->norm_layer_stride_bytes & 15) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f))
+        return MOLE_ERR_INVALID_ARG;
     if (mode == MOLE_STEP_AUTO) mode = (L > 1 && M > kFusedMaxTokens) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
 
-    StepLaunch a;
-    a.residual = nullptr;
-    a.row_index = ids;
-    a.gates_out = nullptr;
-    a.status = status;
-    a.lut_stride = lut_layer_stride_bytes;
-    a.wr_stride = wr_layer_stride_bytes;
-    a.M = M;
-    a.N = N;
-    a.d = d;
-    a.rows = V;
-    a.dtype = dtype;
-    a.d_split = d_split;
-    a.stream = static_cast<cudaStream_t>(stream);
+    StepLaunch s;
+    s.residual = nullptr;
+    s.row_index = a->ids;
+    s.gates_out = nullptr;
+    s.status = a->status;
+    s.lut_stride = a->lut_layer_stride_bytes;
+    s.wr_stride = a->wr_layer_stride_bytes;
+    s.norm_stride = a->norm_layer_stride_bytes;
+    s.norm_eps = a->norm_eps;
+    s.M = M;
+    s.N = a->N;
+    s.d = a->d;
+    s.rows = a->V;
+    s.dtype = a->dtype;
+    s.d_split = a->d_split;
+    s.kernel = a->kernel;
+    s.stream = static_cast<cudaStream_t>(a->stream);
     if (mode == MOLE_STEP_FUSED) {
         // one launch: every block walks its tokens through all L layers
-        a.hidden = hidden_in;
-        a.lut = lut_base;
-        a.w_router = w_router_base;
-        a.out = out;
-        a.L = L;
-        a.flags = 0;
-        return launch_step(a);
+        s.hidden = a->hidden_in;
+        s.lut = a->lut_base;
+        s.w_router = a->w_router_base;
+        s.norm_weight = a->norm_weight_base;
+        s.out = a->out;
+        s.L = L;
+        s.flags = a->flags & MOLE_FLAG_CHAIN;
+        if (L > 1 && s.kernel == MOLE_KERNEL_DECODE) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        return launch_step(s);
     }
-    if (L > 1 && (!tmp || !aligned16(tmp) || out == hidden_in || tmp == hidden_in || tmp == out))
+    if (L > 1 && (!a->tmp || !aligned16(a->tmp) || a->out == a->hidden_in || a->tmp == a->hidden_in || a->tmp == a->out))
         return MOLE_ERR_INVALID_ARG;
-    // L launches; ping-pong so that the last layer writes `out` and hidden_in is never written
-    const void *src = hidden_in;
+    // L launches; ping-pong so that the last layer writes `out` and hidden_in is never written.  Layers after
+    // the first are chained to their predecessor with programmatic dependent launch (they read nothing but
+    // the previous layer's output from it); the first layer only if the caller says so (MOLE_FLAG_CHAIN):
+    // whatever precedes it on the stream may be producing ids, tables or router weights.
+    const void *src = a->hidden_in;
     for (int l = 0; l < L; ++l) {
-        void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
-        a.hidden = src;
-        a.lut = static_cast<const unsigned char *>(lut_base) + static_cast<int64_t>(l) * lut_layer_stride_bytes;
-        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
-        a.out = dst;
-        a.L = 1;
-        a.flags = MOLE_FLAG_CHAIN;
-        rc = launch_step(a);
+        void *dst = ((L - 1 - l) % 2 == 0) ? a->out : a->tmp;
+        s.hidden = src;
+        s.lut = static_cast<const unsigned char *>(a->lut_base) + static_cast<int64_t>(l) * a->lut_layer_stride_bytes;
+        s.w_router = static_cast<const unsigned char *>(a->w_router_base) + static_cast<int64_t>(l) * a->wr_layer_stride_bytes;
+        s.norm_weight = a->norm_weight_base
+                            ? static_cast<const unsigned char *>(a->norm_weight_base) + static_cast<int64_t>(l) * a->norm_layer_stride_bytes
+                            : nullptr;
+        s.out = dst;
+        s.L = 1;
+        s.flags = l > 0 ? MOLE_FLAG_CHAIN : (a->flags & MOLE_FLAG_CHAIN);
+        rc = launch_step(s);
         if (rc != MOLE_OK) return rc;
         src = dst;
     }
     return MOLE_OK;
+}
+
+int mole_decode_step_ex(const void *hidden_in, const int32_t *ids, const void *lut_base, int64_t lut_layer_stride_bytes,
+                        const void *w_router_base, int64_t wr_layer_stride_bytes, void *out, void *tmp, uint32_t *status,
+                        int L, int B, int T, int N, int d, int V, int dtype, int mode, int d_split, void *stream)
+{
+    mole_step_args a;
+    memset(&a, 0, sizeof a);
+    a.struct_size = sizeof a;
+    a.hidden_in = hidden_in;
+    a.ids = ids;
+    a.lut_base = lut_base;
+    a.lut_layer_stride_bytes = lut_layer_stride_bytes;
+    a.w_router_base = w_router_base;
+    a.wr_layer_stride_bytes = wr_layer_stride_bytes;
+    a.out = out;
+    a.tmp = tmp;
+    a.status = status;
+    a.L = L;
+    a.B = B;
+    a.T = T;
+    a.N = N;
+    a.d = d;
+    a.V = V;
+    a.dtype = dtype;
+    a.mode = mode;
+    a.d_split = d_split;
+    a.stream = stream;
+    return mole_decode_step_args(&a);
 }
 
 int mole_decode_step(const void *hidden_in, const int32_t *ids, const void *lut_base, int64_t lut_layer_stride_bytes,
@@ -518,32 +766,76 @@ int mole_decode_step_host(const void *hidden_host, const int32_t *ids_host, void
                           int64_t lut_layer_stride_bytes, const void *w_router_base, int64_t wr_layer_stride_bytes,
                           uint32_t *status, int L, int B, int T, int N, int d, int V, int dtype, void *stream)
 {
-    if (B < 0 || T < 0 || (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32)) return MOLE_ERR_INVALID_ARG;
+    // every check the step itself would make, before the first copy is queued
+    if (L < 1) return MOLE_ERR_INVALID_ARG;
+    int rc = check_common(dev_hidden, dev_ids, lut_base, w_router_base, dev_out, nullptr, B, T, N, d, V, dtype);
+    if (rc != MOLE_OK) return rc;
     const long long M = static_cast<long long>(B) * T;
     if (M == 0) return MOLE_OK;
-    if (!hidden_host || !ids_host || !out_host || !dev_hidden || !dev_ids || !dev_out) return MOLE_ERR_INVALID_ARG;
+    if (!hidden_host || !ids_host || !out_host) return MOLE_ERR_INVALID_ARG;
+    if ((lut_layer_stride_bytes & 15) || (wr_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if (M * L > 0x3fffffffLL) return MOLE_ERR_TOO_LARGE;
+    const bool chained = L > 1 && M > kFusedMaxTokens;
+    if (chained && (!dev_tmp || !aligned16(dev_tmp) || dev_out == dev_hidden || dev_tmp == dev_hidden || dev_tmp == dev_out))
+        return MOLE_ERR_INVALID_ARG;
+    {
+        StepPlan plan;
+        rc = plan_step(M, chained ? 1 : L, N, d, dtype, 0, &plan);
+        if (rc != MOLE_OK) return rc;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t act_bytes = static_cast<size_t>(M) * d * elem_bytes(dtype);
     MOLE_CUDA_TRY(cudaMemcpyAsync(dev_ids, ids_host, static_cast<size_t>(M) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     MOLE_CUDA_TRY(cudaMemcpyAsync(dev_hidden, hidden_host, act_bytes, cudaMemcpyHostToDevice, st));
-    int rc = mole_decode_step(dev_hidden, dev_ids, lut_base, lut_layer_stride_bytes, w_router_base, wr_layer_stride_bytes,
-                              dev_out, dev_tmp, status, L, B, T, N, d, V, dtype, stream);
+    rc = mole_decode_step(dev_hidden, dev_ids, lut_base, lut_layer_stride_bytes, w_router_base, wr_layer_stride_bytes,
+                          dev_out, dev_tmp, status, L, B, T, N, d, V, dtype, stream);
     if (rc != MOLE_OK) return rc;
     MOLE_CUDA_TRY(cudaMemcpyAsync(out_host, dev_out, act_bytes, cudaMemcpyDeviceToHost, st));
     return MOLE_OK;
+}
+
+// SM count of the current device if there is one, the nominal B200 figure otherwise (no error is kept)
+static int sms_or_nominal()
+{
+    int sms = kNumSMs;
+    if (sm_count(&sms) != MOLE_OK) {
+        (void)cudaGetLastError();
+        sms = kNumSMs;
+    }
+    return sms;
 }
 
 int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads, int *out_smem_bytes,
               int *out_stages, int *out_blocks_per_sm)
 {
     StepPlan plan;
-    int rc = plan_step(M, L, N, d, dtype, d_split, &plan);
+    int rc = plan_step(M, L, N, d, dtype, d_split, &plan, false, sms_or_nominal());
     if (rc != MOLE_OK) return rc;
     if (out_d_split) *out_d_split = plan.d_split;
     if (out_threads) *out_threads = plan.threads;
     if (out_smem_bytes) *out_smem_bytes = plan.smem;
     if (out_stages) *out_stages = plan.stages;
     if (out_blocks_per_sm) *out_blocks_per_sm = plan.blocks_per_sm;
+    return MOLE_OK;
+}
+
+int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, char *name, int name_bytes, int *out_threads,
+                 int *out_smem_bytes)
+{
+    if (M < 1 || !name || name_bytes < 1) return MOLE_ERR_INVALID_ARG;
+    LaunchChoice c;
+    int rc = choose_launch(M, L, N, d, dtype, d_split, norm != 0, kernel, sms_or_nominal(), false, &c);
+    if (rc != MOLE_OK) return rc;
+    snprintf(name, static_cast<size_t>(name_bytes), "%s", c.name);
+    if (out_threads) *out_threads = c.threads;
+    if (out_smem_bytes) *out_smem_bytes = c.smem;
+    return MOLE_OK;
+}
+
+int mole_reload_debug_env(void)
+{
+    std::lock_guard<std::mutex> lock(g_env_mutex);
+    load_env_locked();
     return MOLE_OK;
 }
 

@@ -420,6 +420,7 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
         a.dtype = c->dtype;
         a.flags = 0;
         a.d_split = 0;
+        a.kernel = MOLE_KERNEL_RING;  // every group on one kernel family: the step's bits do not depend on how it is grouped
         a.stream = st;
         rc = launch_step(a);
         if (rc != MOLE_OK) return rc;

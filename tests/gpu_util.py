@@ -63,16 +63,28 @@ def check_gates(gates: torch.Tensor, ref: np.ndarray):
     assert np.abs(g.sum(axis=1) - 1.0).max() <= 1e-6
 
 
+def near_tie_slack(normed: np.ndarray, wr: torch.Tensor, dtype=torch.bfloat16) -> np.ndarray:
+    """Per token, how far the gates may move because the normalised state is rounded to the storage type
+    in fp32 on the GPU and in fp64 by the oracle.  Only an element whose exact (fp64) value lies within fp32
+    noise (2^-20 relative) of a rounding tie can land on the other neighbour; that moves logit j by one
+    storage-type ulp of THAT element times W_r[c][j], and a softmax moves by at most half of its largest
+    logit change.  A token without such an element gets no slack at all."""
+    if dtype != torch.bfloat16:
+        return np.zeros(normed.shape[0])  # fp32 storage: a last-place difference moves a logit by ~1e-7
+    a = np.abs(normed)
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(a, 1e-300))) - 7)  # bf16: 8 significant bits
+    frac = (a / ulp) % 1.0
+    near = np.abs(frac - 0.5) * ulp <= 2.0 ** -20 * a
+    wmax = np.abs(wr.detach().cpu().to(torch.float64).numpy()).max(axis=1)  # [d]
+    return 0.5 * (near * ulp * wmax[None, :]).sum(axis=1)
+
+
 def check_gates_normed_router(gates: torch.Tensor, ref: np.ndarray, normed: np.ndarray, wr: torch.Tensor, dtype=torch.bfloat16):
-    """Gates of the layer whose router reads RMSNorm(hidden) rounded to the storage type.  That rounding
-    is a decision taken in fp32 on the GPU and in fp64 by the oracle: an element within fp32 noise of a
-    tie (about one in ten thousand) lands on the neighbouring value, which moves a logit by one
-    storage-type ulp of that element times a router weight and a gate by at most a quarter of that.
-    So: every gate within two such flips of the oracle's, and all but a few within the plain 1e-5."""
+    """Gates of the layer whose router reads RMSNorm(hidden) rounded to the storage type: within 1e-5 of
+    the oracle's, plus -- only for tokens that have an element on a rounding tie -- what those elements'
+    flips can move (near_tie_slack).  `normed`: the oracle's normalised state in fp64, before rounding."""
     g = gates.detach().cpu().to(torch.float64).numpy()
     err = np.abs(g - ref)
-    ulp = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -24
-    flip = 0.25 * ulp * float(np.abs(normed).max()) * float(wr.abs().max())
-    assert err.max() <= 1e-5 + 2 * flip, (float(err.max()), flip)
-    assert (err <= 1e-5).mean() >= 0.97, float((err <= 1e-5).mean())
+    slack = near_tie_slack(normed, wr, dtype)
+    assert (err <= 1e-5 + slack[:, None]).all(), (float(err.max()), float(slack.max()), int((slack > 0).sum()))
     assert np.abs(g.sum(axis=1) - 1.0).max() <= 1e-6

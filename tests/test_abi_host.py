@@ -33,15 +33,29 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_version_and_status_strings(lib):
-    assert lib.mole_version() == 210
+    assert lib.mole_version() == 300
     seen = {lib.mole_status_string(c).decode() for c in range(6)}
     assert len(seen) == 6 and "ok" in seen
     assert lib.mole_status_string(99).decode() == "unknown status"
 
 
-def test_args_struct_layout_matches_header(lib):
-    # 2 x u32, 8 pointers, 8 x i32, 2 pointers, 1 float, 1 i32
-    assert ctypes.sizeof(binding.MoleArgs) == 8 + 8 * 8 + 8 * 4 + 2 * 8 + 4 + 4
+def test_variant_names_and_kernel_choice(lib):
+    V = binding.variant
+    # decode batches of the paper's 160M / 410M widths: the one-block-per-token kernel, d / 4 threads
+    assert V(256, 16, 768) == ("decode<16,0>", 192, V(256, 16, 768)[2]) and V(64, 16, 1024)[:2] == ("decode<16,0>", 256)
+    assert V(256, 16, 768, norm=True)[0] == "decode<16,1>"
+    # beyond 2048 tokens, with an explicit chunk count, for several layers, or on request: the ring kernel
+    assert V(16384, 16, 1024)[0] == "step<bf16,16,1,2,2,0,0>"
+    assert V(256, 16, 768, d_split=1)[0] == "step<bf16,16,1,2,1,1,0>"
+    assert V(256, 16, 768, L=12)[0] == "step<bf16,16,1,1,1,0,0>"
+    assert V(256, 16, 768, kernel=binding.KERNEL_RING)[0] == "step<bf16,16,1,2,1,1,0>"
+    # the 1B width (512 column groups of 8 bytes, N = 32) is outside the decode kernel: ring kernel, rows cut by experts
+    assert V(256, 32, 2048)[0] == "step<bf16,32,2,3,3,0,0>" and V(64, 32, 2048, L=16)[0] == "step<bf16,32,2,3,4,0,0>"
+    with pytest.raises(binding.MoleError) as e:
+        V(256, 32, 2048, kernel=binding.KERNEL_DECODE)
+    assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    assert V(64, 32, 1024)[0] == "decode<32,0>" and V(64, 5, 768)[0].startswith("step<bf16,0,")
+    assert V(64, 4, 64, binding.DTYPE_F32)[0].startswith("step<f32,4,")
 
 
 def test_plan_shapes():
@@ -125,9 +139,9 @@ def test_ex_rejects_bad_struct(lib):
     a.residual = good + 0x100
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
     a.residual = None
-    a.reserved = 9
+    a.kernel = 9
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
-    a.reserved = 0
+    a.kernel = 0
     a.reserved2 = 1
     assert lib.mole_layer_forward_ex(ctypes.byref(a)) == binding.ERR_INVALID_ARG
     a.reserved2 = 0
@@ -151,6 +165,29 @@ def test_decode_step_and_offload_argument_checks(lib):
     assert dx(good, good, good, 16, good, 16, good + 0x100, None, None, 2, 4, 1, 16, 768, 100, 0, CH, 0, None) == binding.ERR_INVALID_ARG
     assert dx(good, good, good, 16, good, 16, good, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, CH, 0, None) == binding.ERR_INVALID_ARG
     assert dx(good, good, good, 16, good, 16, good + 0x100, good + 0x200, None, 2, 4, 1, 16, 768, 100, 0, 7, 0, None) == binding.ERR_INVALID_ARG
+    # the host-buffer form validates everything before it queues its first copy
+    dh = lib.mole_decode_step_host
+    assert dh(good, good, good, good, good, good + 0x100, good + 0x200, good, 16, good, 16, None, 2, 4, 1, 16, 772, 100, 0,
+              None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert dh(good, good, good, good, good, good + 0x100, good + 0x200, good, 16, good, 16, None, 2, 4, 1, 16, -8, 100, 0,
+              None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert dh(good, good, good, good, good, good + 0x100, good + 0x200, good, 8, good, 16, None, 2, 4, 1, 16, 768, 100, 0,
+              None) == binding.ERR_INVALID_ARG
+    assert dh(None, good, good, good, good, good + 0x100, good + 0x200, good, 16, good, 16, None, 2, 4, 1, 16, 768, 100, 0,
+              None) == binding.ERR_INVALID_ARG
+    sa = binding.MoleStepArgs()
+    assert lib.mole_decode_step_args(None) == binding.ERR_INVALID_ARG
+    assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG  # struct_size 0
+    sa.struct_size = ctypes.sizeof(binding.MoleStepArgs)
+    sa.hidden_in = sa.ids = sa.lut_base = sa.w_router_base = good
+    sa.out, sa.tmp = good + 0x100, good + 0x200
+    sa.L, sa.B, sa.T, sa.N, sa.d, sa.V = 2, 4, 1, 16, 768, 100
+    sa.norm_weight_base, sa.norm_eps = good + 8, 1e-5  # misaligned scale vectors
+    assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG
+    sa.norm_weight_base, sa.norm_eps = good, -1.0
+    assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG
+    sa.norm_eps, sa.flags = 1e-5, 1  # only MOLE_FLAG_CHAIN is a flag of a step
+    assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG
     dd = lib.mole_dedup_ids
     assert dd(good, -1, 10, good, good, good, good, None, None) == binding.ERR_INVALID_ARG
     assert dd(good, (1 << 20) + 1, 10, good, good, good, good, None, None) == binding.ERR_TOO_LARGE

@@ -46,9 +46,12 @@ def test_full_shape_layer_against_oracle(name, batches, n_sample):
         check_out(out[sample], ref)
         check_gates(gates[sample], gref)
         # token independence at full size: the sampled tokens alone give the same bytes
-        if M > 1:
-            alone = mole.layer_forward(hidden[sample].contiguous(), ids[sample].contiguous(), lut, wr,
-                                       d_split=mole.plan(M, sh.N, sh.d)[0])
+        if M > 1:  # ... in the same kernel family and launch shape
+            if mole.variant(M, sh.N, sh.d)[0].startswith("decode"):
+                how = {"kernel": mole.KERNEL_DECODE}
+            else:
+                how = {"kernel": mole.KERNEL_RING, "d_split": mole.plan(M, sh.N, sh.d)[0]}
+            alone = mole.layer_forward(hidden[sample].contiguous(), ids[sample].contiguous(), lut, wr, **how)
             assert torch.equal(alone, out[sample])
     del lut
 
@@ -69,7 +72,7 @@ def test_last_row_of_a_table_beyond_4GiB_is_addressed_correctly():
         assert (out[k].float() == v).all()
 
 
-@pytest.mark.parametrize("name,M,n_sample", [("160m", 256, 96), ("410m", 256, 64)])
+@pytest.mark.parametrize("name,M,n_sample", [("160m", 256, 96), ("410m", 256, 64), ("1b", 256, 48), ("1b", 64, 32)])
 def test_full_shape_decode_step_chained_and_fused(name, M, n_sample):
     """Three layers of the full-size tables as the bench launches them (chained with programmatic
     dependent launch, and the single fused launch): sampled tokens against the oracle's chain on the

@@ -302,11 +302,8 @@ def test_rows_cut_by_experts_single_layer(M, N, d, split):
     assert status == 0
     check_out(out, ref)
     check_gates(gates, gref)
-    os.environ["MOLE_FORCE_COLUMN_CHUNKS"] = "1"  # the same launch with the rows cut by columns
-    try:
+    with mole.debug_env(MOLE_FORCE_COLUMN_CHUNKS=1):  # the same launch with the rows cut by columns
         out2, gates2, status2 = run_gpu(hidden, ids, lut, wr, d_split=split)
-    finally:
-        del os.environ["MOLE_FORCE_COLUMN_CHUNKS"]
     assert status2 == 0
     check_out(out2, ref)
     check_gates(gates2, gref)
@@ -345,13 +342,10 @@ def test_decode_step_fused_and_chained_equal_layer_after_layer(M, N, d, L, split
     # The fused launch sums an item's experts in the same order as the single layers when the rows
     # arrive cut by columns (always with one chunk); cut by experts (several chunks, bf16, K | N) the
     # order of the fp32 sum differs, and with it now and then a rounding decision.
-    os.environ["MOLE_FORCE_COLUMN_CHUNKS"] = "1"
-    try:
+    with mole.debug_env(MOLE_FORCE_COLUMN_CHUNKS=1):
         by_columns = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), None, status=status,
                                       mode=mole.STEP_FUSED, d_split=split)
         torch.cuda.synchronize()
-    finally:
-        del os.environ["MOLE_FORCE_COLUMN_CHUNKS"]
     assert torch.equal(by_columns, h)
     if split == 1:
         assert torch.equal(fused, h)

@@ -222,7 +222,7 @@ def test_offload_decode_step_equals_resident_layers(M, L, cap):
             ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, status=status, side_stream=side)
             h = hidden
             for l in range(L):
-                h = mole.layer_forward(h, ids, luts_dev[l], wrs[l])
+                h = mole.layer_forward(h, ids, luts_dev[l], wrs[l], kernel=mole.KERNEL_RING)
             torch.cuda.synchronize()
             assert torch.equal(out, h)
             if step == 2 and M > 2:
@@ -268,6 +268,53 @@ def test_offload_decode_step_replayed_from_cuda_graphs():
             graphs[k % 3].replay()
         torch.cuda.synchronize()
         assert torch.equal(out, want[29 % 3]) and int(status.item()) == 0
+    finally:
+        ctx.destroy()
+        host.free()
+
+
+@pytest.mark.parametrize("M", [1, 8, 64])
+def test_offload_decode_step_at_the_benchmarked_shape(M):
+    """The offload configuration as bench.py times it: 410M-shaped host tables (V = 50304, 32 KB rows; three
+    layers, 4.9 GB pinned, a layer stride of 1.65 GB), a context of 256 tokens (so one fetch launch brings
+    several layers' rows), Zipf ids.  Bitwise equal to resident ring-kernel layers on a device copy of the
+    same tables, and element by element within the chain bound of the oracle on the referenced rows."""
+    sh = inputs.SHAPES["410m"]
+    L, N, d, V = 3, sh.N, sh.d, sh.V
+    host = mole.HostTable((L, V, N, d), torch.bfloat16)
+    ctx = mole.OffloadContext(max_tokens=256, N=N, d=d, V=V, n_buffers=2)
+    side = torch.cuda.Stream()
+    try:
+        dev_tables = torch.empty((L, V, N, d), dtype=torch.bfloat16, device=DEV)
+        for l in range(L):
+            inputs.make_table(V, N, d, seed=50 + l, device=DEV, out=dev_tables[l])
+            host.tensor[l].copy_(dev_tables[l])
+        torch.cuda.synchronize()
+        wrs = torch.stack([inputs.make_router(d, N, seed=60 + l, device=DEV) for l in range(L)])
+        hidden = inputs.make_hidden(M, d, seed=M, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        for step in range(2):
+            ids = inputs.make_ids(M, V, seed=70 + step + M, device=DEV)
+            out, tmp = torch.empty_like(hidden), torch.empty_like(hidden)
+            ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, status=status, side_stream=side)
+            h = hidden
+            for l in range(L):
+                h = mole.layer_forward(h, ids, dev_tables[l], wrs[l], kernel=mole.KERNEL_RING)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            assert torch.equal(out, h)
+            # the oracle's chain on the rows this batch references (plain torch index on the pinned host table)
+            ids_np = ids.cpu().numpy()
+            uniq, inv = np.unique(ids_np, return_inverse=True)
+            ho = hidden.cpu()
+            for l in range(L):
+                rows = host.tensor[l][torch.from_numpy(uniq).long()]
+                ref, _, bad = oracle.layer_lookup(bits(ho), inv, bits(rows), bits(wrs[l]))
+                assert bad == 0
+                ho = torch.from_numpy(ref).to(torch.bfloat16)
+            err = np.abs(out.cpu().double().numpy() - ref)
+            assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))).all(), float(err.max())
+        del dev_tables
     finally:
         ctx.destroy()
         host.free()

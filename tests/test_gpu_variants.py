@@ -1,0 +1,122 @@
+"""Every kernel instantiation that bench.py times has a parity case here, element by element against the
+fp64 oracle, at the token count, width and expert count the bench uses (the table itself is small: the
+instantiation does not depend on the number of table rows).  The CPU half of the file walks the launch
+shapes bench.py declares and fails if one of them resolves to an instantiation without a case below."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import oracle
+from gpu_util import as_f64, bits, check_gates, check_gates_normed_router, check_out, oracle_layer
+from paper_2503_15798_b200 import binding as mole
+
+DEV = "cuda"
+RING, DECODE, AUTO = mole.KERNEL_RING, mole.KERNEL_DECODE, mole.KERNEL_AUTO
+
+# instantiation -> launches that reach it: (M, N, d, L, norm, kernel)
+CASES = {
+    # single-layer launches of the chained step
+    "decode<16,0>": [(256, 16, 768, 1, False, AUTO), (64, 16, 1024, 1, False, AUTO), (1, 16, 768, 1, False, AUTO),
+                     (2048, 16, 1024, 1, False, AUTO)],
+    "decode<16,1>": [(256, 16, 768, 1, True, AUTO), (256, 16, 1024, 1, True, AUTO), (8, 16, 768, 1, True, AUTO)],
+    "decode<32,0>": [(70, 32, 1024, 1, False, AUTO)],
+    "decode<32,1>": [(70, 32, 512, 1, True, AUTO)],
+    "decode<8,0>": [(33, 8, 256, 1, False, AUTO)],
+    "decode<8,1>": [(33, 8, 384, 1, True, AUTO)],
+    "decode<4,0>": [(19, 4, 128, 1, False, AUTO)],
+    "decode<4,1>": [(19, 4, 2048, 1, True, AUTO)],
+    "step<bf16,16,1,2,1,1,0>": [(256, 16, 768, 1, False, RING)],
+    "step<bf16,16,1,2,1,0,0>": [(64, 16, 768, 1, False, RING), (3000, 16, 768, 1, False, AUTO)],
+    "step<bf16,16,1,2,2,1,0>": [(256, 16, 1024, 1, False, RING)],
+    "step<bf16,16,1,2,2,0,0>": [(64, 16, 1024, 1, False, RING), (2500, 16, 1024, 1, False, AUTO)],
+    "step<bf16,16,1,2,1,1,1>": [(256, 16, 768, 1, True, RING)],
+    "step<bf16,16,1,2,1,0,1>": [(700, 16, 768, 1, True, RING)],
+    "step<bf16,16,1,2,2,1,1>": [(256, 16, 1024, 1, True, RING)],
+    "step<bf16,16,1,2,2,0,1>": [(2500, 16, 1024, 1, True, AUTO)],
+    "step<bf16,32,2,3,3,0,0>": [(256, 32, 2048, 1, False, AUTO), (256, 32, 2048, 3, False, AUTO)],
+    "step<bf16,32,2,3,4,0,0>": [(64, 32, 2048, 1, False, AUTO), (64, 32, 2048, 3, False, AUTO), (148, 32, 2048, 2, False, AUTO)],
+    "step<bf16,32,2,3,3,0,1>": [(256, 32, 2048, 1, True, AUTO)],
+    "step<bf16,32,1,0,0,0,1>": [(16, 32, 2048, 1, True, AUTO), (16, 32, 2048, 2, True, AUTO)],
+    "step<bf16,32,2,0,0,0,1>": [(256, 32, 2048, 2, True, AUTO)],
+    # fused steps
+    "step<bf16,16,1,1,1,0,0>": [(256, 16, 768, 3, False, AUTO), (64, 16, 768, 12, False, AUTO)],
+    "step<bf16,16,1,1,2,0,0>": [(256, 16, 1024, 3, False, AUTO), (64, 16, 1024, 4, False, AUTO), (8, 16, 1024, 8, False, AUTO)],
+    "step<bf16,16,1,0,0,0,1>": [(256, 16, 768, 3, True, AUTO), (64, 16, 1024, 2, True, AUTO)],
+}
+FLAT = [(name,) + c for name, cs in CASES.items() for c in cs]
+
+
+def test_every_launch_shape_the_bench_times_has_a_parity_case():
+    missing = {}
+    for sh in bench.timed_launch_shapes():
+        name = mole.variant(sh["M"], sh["N"], sh["d"], L=sh["L"], norm=sh["norm"], kernel=sh["kernel"])[0]
+        if name not in CASES:
+            missing.setdefault(name, []).append(sh["what"])
+    assert not missing, missing
+
+
+def _oracle_chain(hidden, ids, luts, wrs, gammas, eps):
+    """The oracle layer after layer, each fed the storage-type rounding of the previous one; with gammas the
+    router of every layer reads the rounded RMSNorm of its input.  Returns the last layer's fp64 output, its
+    gates, the (fp64) normalised state of the last layer."""
+    h = hidden
+    for l in range(luts.shape[0]):
+        if gammas is None:
+            ref, gref, _ = oracle_layer(h, ids, luts[l], wrs[l])
+            normed = None
+        else:
+            h64, g64 = as_f64(h), as_f64(gammas[l])
+            normed = np.stack([oracle.rmsnorm(h64[t], g64, eps) for t in range(h64.shape[0])])
+            ref, gref, _ = oracle.layer_lookup(bits(torch.from_numpy(normed).to(torch.bfloat16)), ids.cpu().numpy(),
+                                               bits(luts[l]), bits(wrs[l]), residual=bits(h))
+        h = torch.from_numpy(ref).to(torch.bfloat16)
+    return ref, gref, normed
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,M,N,d,L,norm,kernel", FLAT)
+def test_variant_against_the_oracle(name, M, N, d, L, norm, kernel):
+    assert mole.variant(M, N, d, L=L, norm=norm, kernel=kernel)[0] == name
+    V = 97
+    g = torch.Generator().manual_seed(M + 7 * d + L)
+    luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16)
+    wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16)
+    hidden = (1.5 * torch.empty(M, d).normal_(0, 1, generator=g)).to(torch.bfloat16)
+    ids = torch.randint(0, V, (M,), generator=g, dtype=torch.int32)
+    gammas = (1.0 + 0.2 * torch.empty(L, d).normal_(0, 1, generator=g)).to(torch.bfloat16) if norm else None
+    eps = 1e-5
+    ref, gref, normed = _oracle_chain(hidden, ids, luts, wrs, gammas, eps)
+    hd, idd, ld, wd = hidden.to(DEV), ids.to(DEV), luts.to(DEV), wrs.to(DEV)
+    gd = gammas.to(DEV) if norm else None
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    if L == 1:
+        gates = torch.zeros(M, N, dtype=torch.float32, device=DEV)
+        out = mole.layer_forward(hd, idd, ld[0], wd[0], gates_out=gates, status=status, kernel=kernel, chain=True,
+                                 norm_weight=None if gd is None else gd[0], norm_eps=eps)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        if norm:
+            check_gates_normed_router(gates, gref, normed, wrs[0])
+            dg = np.abs(as_f64(gates) - gref).sum(axis=1, keepdims=True)
+            err = np.abs(as_f64(out) - ref)
+            assert (err <= 2.0 ** -8 * np.abs(ref) + 2e-5 + dg * float(luts.abs().max())).all()
+        else:
+            check_gates(gates, gref)
+            check_out(out, ref)
+        return
+    outs = []
+    for mode in (mole.STEP_FUSED, mole.STEP_CHAINED):
+        out = mole.decode_step_args(hd, idd, ld, wd, torch.empty_like(hd), torch.empty_like(hd), status=status, mode=mode,
+                                    norm_weights=gd, norm_eps=eps, kernel=kernel)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        err = np.abs(as_f64(out) - ref)
+        slack = 0.0
+        if norm:  # a rounding tie in a normalised element moves a gate (see gpu_util.near_tie_slack): per layer, a few 1e-4
+            slack = L * 1e-3 * float(luts.abs().max()) * N
+        assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref)) + slack).all(), (mode, float(err.max()))
+        outs.append(out)
+    if not norm:
+        # the two ways of launching a step differ only in the order of fp32 sums
+        assert (np.abs(as_f64(outs[0]) - as_f64(outs[1])) <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))).all()
