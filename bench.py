@@ -2,19 +2,28 @@
 """Benchmark of the fused MoLE layer (arXiv 2503.15798, Eq. 4 + Eq. 8) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 160m|410m|1b] [--batch M]
-                    [--impl mole|reference] [--no-sweep] [--no-cpu]
+                    [--impl mole|reference] [--headline-only] [--no-cpu] [--no-offload] [--offload]
 
-A "step" is one decode step of the whole hot path: all L layers of the configuration applied
-to one batch of M tokens (router, softmax over all experts, row gather, weighted sum,
-residual), chained with programmatic dependent launch and replayed from a CUDA graph.  The
-metric is tokens/s for the L-layer step; the roofline block reports the layer kernel's
-algorithmic GB/s (gathered rows + hidden in/out + router weights) against the measured HBM
-copy bandwidth.  Every step uses a different pre-generated Zipf(1.1) id batch, and the table
-(GBs) is far larger than L2.  Beside it, as an extra ("fused_step"), the same step as a single
-launch that walks every token through all L layers on chip.
+A "step" is one decode step of the whole hot path: all L layers of the configuration applied to
+one batch of M tokens (router, softmax over all experts, row gather, weighted sum, residual).
+The headline times it as a model that runs other work between the layers gets it: one launch per
+layer, chained with programmatic dependent launch, the L launches of a step replayed from a CUDA
+graph.  The metric is tokens/s for the L-layer step; the roofline block reports the layer
+kernel's algorithmic GB/s (gathered rows + hidden in/out + router weights) against the measured
+HBM copy bandwidth.  Every step uses a different pre-generated Zipf(1.1) id batch, and the tables
+(GBs) are far larger than L2.  The timed region of exactly K steps is repeated until the repeats
+span a quarter of a second; the value is the median repeat.
 
-With N > 1 (torchrun) every rank holds its own replica of the tables and its own batches
-(tokens are independent, so there is no collective on the data path): weak scaling.
+Beside the headline (one GPU): the same step as a single fused launch ("fused_step"), with
+RMSNorm in front of every router, end to end from host buffers through the C ABI ("e2e"), a
+sweep over the configuration's batch sizes with isolated-launch times, and a `configs` block with
+the chained and fused rows of the other workload shapes, the quantised (NF4 / NF3) tables and the
+offload mode.  The CPU oracle is timed on the host cores on a bounded sample of the same
+workload, and its outputs are compared with the GPU's for the last timed step.
+
+With N > 1 (torchrun) every rank holds its own replica of the tables and its own batches (tokens
+are independent, so there is no collective on the data path): weak scaling; only the headline,
+the fused step and the end-to-end number are measured.
 
 --impl reference times the CPU oracle (oracle/, plain C, fp64) on the host cores instead.
 """
@@ -23,6 +32,7 @@ from __future__ import annotations
 import argparse
 import dataclasses
 import json
+import math
 import os
 import statistics
 import sys
@@ -35,20 +45,18 @@ if ROOT not in sys.path:
 
 METRIC = "MoLE layer tokens/s (L-layer decode step) and achieved HBM GB/s"
 UNIT = "tokens/s"
-N_BATCHES = 32          # distinct id batches the steps rotate through
+N_BATCHES = 32          # distinct id batches the headline's steps rotate through
+N_BATCHES_EXTRA = 16    # ... and the rows beside it
+MIN_SPAN_S = 0.25       # the timed region is repeated until the repeats span this long
 OFFLOAD_CONTEXT_TOKENS = 256  # offload mode: the context (staging areas) is sized for this many tokens
+OFFLOAD_BATCHES = (1, 8, 64)
 FALLBACK_HBM_GBS = 6650.0
+QUANT_BLOCKS = {"160m": {"nf4": 768, "nf3": 128}, "410m": {"nf4": 1024, "nf3": 128}, "1b": {"nf4": 1024, "nf3": 128}}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
-TRAFFIC = {
-    # profiles/mole_step_kernel_single_layer_160m_batch256.md: mean of three captured launches (one layer each)
-    ("160m", 256, 12): 4.43e6,
-}
-# the same for the fused all-layers launch reported as an extra
-FUSED_TRAFFIC = {
-    # profiles/mole_step_kernel_fused_160m_batch256.md: 7.59 MB per 2-layer launch, x6 for the 12 layers of a full launch
-    ("160m", 256, 12): 45.5e6,
-}
+# of the kernel as it stands
+TRAFFIC = {}
+FUSED_TRAFFIC = {}
 
 
 def offload_groups(L: int, M: int, row_bytes: int) -> int:
@@ -61,53 +69,62 @@ def offload_groups(L: int, M: int, row_bytes: int) -> int:
     return -(-L // g)
 
 
-OFFLOAD_BATCHES = (1, 8, 64)
-
-
 def timed_launch_shapes():
-    """Every launch shape a timed region of this file issues, as dicts (what, M, N, d, L, norm, kernel):
-    the parity tests walk this list and require a parity case for the kernel instantiation of each."""
+    """Every launch shape a timed region of this file issues, as dicts (what, M, N, d, L, norm, kernel,
+    lut_format, lut_block): the parity tests walk this list and require a parity case for the kernel
+    instantiation of each."""
     from paper_2503_15798_b200 import inputs
 
     shapes = []
+
+    def add(what, M, sh, L, norm=False, kernel=0, fmt=0, block=0):
+        shapes.append({"what": what, "M": M, "N": sh.N, "d": sh.d, "L": L, "norm": norm, "kernel": kernel,
+                       "lut_format": fmt, "lut_block": block})
+
     for name in ("160m", "410m", "1b"):
         sh = inputs.SHAPES[name]
         for M in sh.batches:
             for norm in (False, True):
                 tag = " norm" if norm else ""
-                shapes.append({"what": f"{name} batch {M} chained{tag}", "M": M, "N": sh.N, "d": sh.d, "L": 1, "norm": norm,
-                               "kernel": 0})
+                add(f"{name} batch {M} chained{tag}", M, sh, 1, norm)
                 if M <= 4096:
-                    shapes.append({"what": f"{name} batch {M} fused{tag}", "M": M, "N": sh.N, "d": sh.d, "L": sh.L,
-                                   "norm": norm, "kernel": 0})
-            shapes.append({"what": f"{name} batch {M} chained, ring kernel", "M": M, "N": sh.N, "d": sh.d, "L": 1,
-                           "norm": False, "kernel": 1})
+                    add(f"{name} batch {M} fused{tag}", M, sh, sh.L, norm)
+            add(f"{name} batch {M} chained, ring kernel", M, sh, 1, kernel=1)
+            if M <= 4096:
+                add(f"{name} batch {M} fused, ring kernel", M, sh, sh.L, kernel=1)
+            for fmt, tag in ((1, "nf4"), (2, "nf3")):
+                add(f"{name} batch {M} chained, {tag} table", M, sh, 1, fmt=fmt, block=QUANT_BLOCKS[name][tag])
     sh = inputs.SHAPES["410m"]
     for M in OFFLOAD_BATCHES:
         groups = offload_groups(sh.L, M, sh.row_bytes)
         per = -(-sh.L // groups)
         for L in {per, sh.L - per * (groups - 1)}:
-            shapes.append({"what": f"410m offload batch {M}, group of {L} layers", "M": M, "N": sh.N, "d": sh.d, "L": L,
-                           "norm": False, "kernel": 0})
+            add(f"410m offload batch {M}, group of {L} layers", M, sh, L, kernel=1)
+        for fmt, tag in ((1, "nf4"), (2, "nf3")):
+            add(f"410m offload batch {M}, {tag} records", M, sh, 1, fmt=fmt, block=QUANT_BLOCKS["410m"][tag])
     return shapes
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
-    ap.add_argument("--warmup", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="mole", choices=["mole", "reference"])
     ap.add_argument("--config", default="160m", choices=["160m", "410m", "1b"])
     ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--headline-only", action="store_true",
+                    help="only the headline, the fused step and the end-to-end number (what N > 1 runs)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-batch sweep and the isolated-launch rows")
-    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-configs", action="store_true", help="skip the rows of the other workload shapes")
+    ap.add_argument("--no-offload", action="store_true", help="skip the offload-mode rows of the default run")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg (and its parity check)")
     ap.add_argument("--layers", type=int, default=0, help="override L (debugging; the line then says so)")
     ap.add_argument("--vocab", type=int, default=0,
                     help="override V, the number of table rows (small profiler captures; the line then says so)")
     ap.add_argument("--offload", action="store_true",
-                    help="offload mode instead: table in pinned host memory, per-step dedup + row fetch overlapped with "
-                         "the previous layer's combine; roofline = measured host-link GB/s")
+                    help="offload mode alone: table in pinned host memory, per-step dedup + row fetch overlapped with "
+                         "the previous layers' combine; roofline = measured host-link GB/s")
     return ap.parse_args()
 
 
@@ -123,7 +140,7 @@ def measured_peak():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self.period, self._stop, self._thread, self.h = period_s, threading.Event(), None, None
         try:
@@ -212,6 +229,11 @@ def reference_arm_runs_here(rank: int) -> bool:
     return rank == 0
 
 
+def repeats_for(ms_one: float, min_span_s: float = MIN_SPAN_S) -> int:
+    """How often a timed region of ms_one milliseconds is repeated to span min_span_s (at least 3, at most 4000)."""
+    return max(3, min(4000, int(math.ceil(min_span_s * 1e3 / max(ms_one, 1e-6)))))
+
+
 # ------------------------------------------------------------------------------------------------------
 # the CPU oracle leg (only bench.py's baseline leg and --impl reference execute oracle/)
 # ------------------------------------------------------------------------------------------------------
@@ -240,10 +262,36 @@ def host_bits(t):
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
+def oracle_chain_check(luts, wrs, hidden, ids, got, threads):
+    """Part of the CPU-baseline leg: the oracle's L-layer chain (each layer fed the bf16 rounding of the
+    previous one) on the rows this batch references, compared element by element with `got`, the GPU's
+    output for the same step.  Returns (max |err| / bound, seconds), bound = L * 2^-7 * max(1, |ref|): one
+    bf16 ulp per layer."""
+    import numpy as np
+    import torch
+
+    import oracle
+
+    t0 = time.perf_counter()
+    L = luts.shape[0]
+    ids_np = ids.cpu().numpy()
+    uniq, inv = np.unique(ids_np, return_inverse=True)
+    sel = torch.from_numpy(uniq).long().to(luts.device)
+    h = hidden.cpu()
+    ref = None
+    for l in range(L):
+        rows = luts[l][sel].cpu()  # plain torch index: the bytes the kernel gathered
+        ref, _, bad = oracle.layer_lookup(host_bits(h), inv, host_bits(rows), host_bits(wrs[l]), threads=threads)
+        assert bad == 0
+        h = torch.from_numpy(ref).to(torch.bfloat16)
+    err = np.abs(got.cpu().to(torch.float64).numpy() - ref)
+    bound = L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))
+    return float((err / bound).max()), time.perf_counter() - t0
+
+
 def run_reference(args):
     """--impl reference: the oracle, as it stands, on the host cores (rank 0 only)."""
     import numpy as np
-    import torch
 
     import oracle
     from paper_2503_15798_b200 import inputs
@@ -295,11 +343,10 @@ def workload_config(sh, L, M, args):
 # ------------------------------------------------------------------------------------------------------
 
 class StepGraphs:
-    """One CUDA graph per id batch; a graph holds the L chained layer launches of one step."""
+    """One CUDA graph per id batch; a graph holds the launches of one step.  `step(ids, out, tmp, status)`
+    issues them."""
 
-    def __init__(self, mole, luts, wrs, hidden, id_batches, mode=0):
-        import torch
-
+    def __init__(self, torch, step, hidden, id_batches):
         self.torch, self.graphs = torch, []
         self.out = torch.empty_like(hidden)
         self.tmp = torch.empty_like(hidden)
@@ -307,64 +354,169 @@ class StepGraphs:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            for ids in id_batches:  # warm-up launches outside capture (sets kernel attributes)
-                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status, mode=mode)
+            for ids in id_batches[:4]:  # launches outside capture first (they set kernel attributes)
+                step(ids, self.out, self.tmp, self.status)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         for ids in id_batches:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                mole.decode_step(hidden, ids, luts, wrs, self.out, self.tmp, status=self.status, mode=mode)
+                step(ids, self.out, self.tmp, self.status)
             self.graphs.append(g)
+        self.id_batches = id_batches
 
     def run(self, k0, k1):
         n = len(self.graphs)
         for k in range(k0, k1):
             self.graphs[k % n].replay()
 
-
-class NormStepGraphs(StepGraphs):
-    """The same chained step with the decoder layer of the paper's App. A.2 listing: every layer's
-    router reads RMSNorm(hidden) (fused into the kernel), the residual stays un-normalised."""
-
-    def __init__(self, mole, luts, wrs, gammas, hidden, id_batches, eps=1e-5):
-        import torch
-
-        self.torch, self.graphs = torch, []
-        self.out = torch.empty_like(hidden)
-        self.tmp = torch.empty_like(hidden)
-        self.status = torch.zeros(1, dtype=torch.int32, device=hidden.device)
-        L = luts.shape[0]
-
-        def step(ids):
-            src = hidden
-            for l in range(L):
-                dst = self.out if (L - 1 - l) % 2 == 0 else self.tmp
-                mole.layer_forward(src, ids, luts[l], wrs[l], dst, status=self.status, chain=l > 0,
-                                   norm_weight=gammas[l], norm_eps=eps)
-                src = dst
-
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            for ids in id_batches:
-                step(ids)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        for ids in id_batches:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                step(ids)
-            self.graphs.append(g)
+    def ok(self):
+        return int(self.status.item()) == 0
 
 
-def timed_ms(torch, fn):
+def event_ms(torch, fn):
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
     fn()
     b.record()
     b.synchronize()
     return a.elapsed_time(b)
+
+
+class _Null:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        return False
+
+
+def timed_steps(torch, run, steps, warmup, barrier=None, dist=None, dev=None, sampler=None):
+    """Warm-up, then the timed region of exactly `steps` steps (barrier + synchronise on both sides, CUDA
+    events on the launching stream), repeated until the repeats span MIN_SPAN_S; every repeat's time is
+    the maximum over ranks.  Returns (median ms of a repeat, dict with min / max / repeats)."""
+    sync = barrier if barrier else torch.cuda.synchronize
+    run(0, max(warmup, 3))
+    sync()
+    first = event_ms(torch, lambda: run(0, steps))
+    reps = repeats_for(max_over_ranks(first, dist, dev))
+    times = []
+    with (sampler if sampler is not None else _Null()):
+        for _ in range(reps):
+            sync()
+            times.append(event_ms(torch, lambda: run(0, steps)))
+    sync()
+    if dist is not None:
+        t = torch.tensor(times, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        times = [float(x) for x in t.cpu()]
+    med = statistics.median(times)
+    return med, {"repeats": reps, "ms_min": min(times), "ms_max": max(times), "span_s": sum(times) * 1e-3}
+
+
+def make_tables(torch, inputs, sh, L, rank, dev):
+    luts = torch.empty((L, sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        inputs.make_table(sh.V, sh.N, sh.d, seed=rank_seeds(rank, l)["table"], device=dev, out=luts[l])
+    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
+    return luts, wrs
+
+
+def config_rows(torch, mole, inputs, sh, L, luts, wrs, batches, steps, warmup, peak, dev, quant=True):
+    """Chained and fused rows of one workload shape (and, with `quant`, the chained step over its tables
+    quantised to NF4 and NF3): per batch the step time, tokens/s, algorithmic bytes and fraction of peak."""
+    rows = []
+    hidden_all = inputs.make_hidden(max(batches), sh.d, seed=3000, device=dev)
+    qtables = {}
+    if quant:
+        for tag, fmt in (("nf4", mole.LUT_NF4), ("nf3", mole.LUT_NF3)):
+            block = QUANT_BLOCKS[sh.name][tag]
+            rb = mole.quant_record_bytes(sh.N, sh.d, fmt, block)
+            packed = torch.zeros((L, sh.V, rb), dtype=torch.uint8, device=dev)
+            for l in range(L):
+                mole.QuantTable.quantize(luts[l], fmt, block, out=packed[l])
+            qtables[tag] = mole.QuantTable(packed, sh.N, sh.d, fmt, block)
+        torch.cuda.synchronize()
+    for m in batches:
+        hid = hidden_all[:m].contiguous()
+        bl = [inputs.make_ids(m, sh.V, seed=4000 + b + 7 * m, device=dev) for b in range(N_BATCHES_EXTRA)]
+        k = max(10, min(steps, int(2e6 // max(m * L, 64))))
+        row = {"batch": m, "steps": k}
+        modes = [("chained", mole.STEP_CHAINED, mole.KERNEL_AUTO, None),
+                 ("chained_ring_kernel", mole.STEP_CHAINED, mole.KERNEL_RING, None)]
+        if m <= 4096:
+            modes += [("fused", mole.STEP_FUSED, mole.KERNEL_AUTO, None), ("fused_ring_kernel", mole.STEP_FUSED, mole.KERNEL_RING, None)]
+        for tag in qtables:
+            modes.append(("chained_" + tag, mole.STEP_CHAINED, mole.KERNEL_AUTO, qtables[tag]))
+        for name, mode, kernel, qt in modes:
+            table = qt if qt is not None else luts
+
+            def step(ids, out, tmp, status, table=table, mode=mode, kernel=kernel):
+                mole.decode_step_args(hid, ids, table, wrs, out, tmp, status=status, mode=mode, kernel=kernel)
+
+            g = StepGraphs(torch, step, hid, bl)
+            ms, spread = timed_steps(torch, g.run, k, min(warmup, 20))
+            assert g.ok(), "a kernel reported a bad id or a timed-out wait"
+            us = ms * 1e3 / k
+            if qt is not None:
+                nbytes = L * (m * qt.record_bytes + 2 * m * sh.d * 2 + sh.d * sh.N * 2)
+            elif mode == mole.STEP_FUSED:
+                nbytes = sh.step_bytes(m, L)
+            else:
+                nbytes = L * sh.layer_bytes(m)
+            row[name] = {"us_per_step": us, "us_per_layer": us / L, "tokens_per_s": m / (us * 1e-6),
+                         "algorithmic_bytes_per_step": nbytes, "GBps": nbytes / us / 1e3, "frac_of_peak": nbytes / us / 1e3 / peak,
+                         "repeats": spread["repeats"],
+                         "kernel": mole.variant(m, sh.N, sh.d, L=L if mode == mole.STEP_FUSED else 1, kernel=kernel,
+                                                lut_format=qt.fmt if qt else 0, lut_block=qt.block if qt else 0)[0]}
+            del g
+        rows.append(row)
+    return rows
+
+
+def isolated_rows(torch, mole, inputs, sh, luts, wrs, batches, peak, dev):
+    """One layer alone (no chaining): `reps` launches inside one event pair, each preceded by a kernel that
+    keeps the GPU busy while the host queues the launch -- an L2 flush (cold) or a short spin (steady) --
+    minus the same region without the launches."""
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    rows = []
+    for m in batches:
+        if m * sh.d * 2 > 2**31:
+            continue
+        hid = inputs.make_hidden(m, sh.d, seed=3000, device=dev)
+        bl = [inputs.make_ids(m, sh.V, seed=4000 + b + 7 * m, device=dev) for b in range(N_BATCHES_EXTRA)]
+        out = torch.empty_like(hid)
+        reps = 100 if m <= 1024 else 20
+        res = {}
+        for cold in (False, True):
+            def filler(r):
+                if cold:
+                    flush.fill_(r & 0xFF)
+                else:
+                    torch.cuda._sleep(20000)
+
+            def with_launches():
+                for r in range(reps):
+                    filler(r)
+                    mole.layer_forward(hid, bl[r % N_BATCHES_EXTRA], luts[0], wrs[0], out)
+
+            def without():
+                for r in range(reps):
+                    filler(r)
+
+            with_launches()
+            torch.cuda.synchronize()
+            t1 = min(event_ms(torch, with_launches) for _ in range(3))
+            t0 = min(event_ms(torch, without) for _ in range(3))
+            res["cold" if cold else "steady"] = max(t1 - t0, 0.0) * 1e3 / reps
+        nbytes = sh.layer_bytes(m)
+        rows.append({"batch": m, "isolated_steady_us": res["steady"], "isolated_cold_us": res["cold"],
+                     "isolated_cold_GBps": nbytes / max(res["cold"], 1e-3) / 1e3,
+                     "isolated_cold_frac_of_peak": nbytes / max(res["cold"], 1e-3) / 1e3 / peak,
+                     "how": f"{reps} launches, each after an L2 flush (cold) or a spin (steady), inside one event pair, "
+                            "minus the region without the launches"})
+    del flush
+    return rows
 
 
 def run_mole(args):
@@ -397,88 +549,99 @@ def run_mole(args):
     L = args.layers or sh.L
     M = args.batch
     peak, peak_src = measured_peak()
+    extras = world == 1 and not args.headline_only
+    t_start = time.perf_counter()
 
-    # ---- resident inputs: L tables, routers, hidden, rotating id batches (per-rank seeds) ----------
-    luts = torch.empty((L, sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
-    for l in range(L):
-        inputs.make_table(sh.V, sh.N, sh.d, seed=rank_seeds(rank, l)["table"], device=dev, out=luts[l])
-    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
-    max_m = max([M] + ([b for b in sh.batches] if not args.no_sweep else []))
-    hidden_all = inputs.make_hidden(max_m, sh.d, seed=rank_seeds(rank)["hidden"], device=dev)
+    luts, wrs = make_tables(torch, inputs, sh, L, rank, dev)
+    hidden = inputs.make_hidden(M, sh.d, seed=rank_seeds(rank)["hidden"], device=dev)
 
-    def batches_for(m):
-        return [inputs.make_ids(m, sh.V, seed=rank_seeds(rank, 0, b, m)["ids"], device=dev) for b in range(N_BATCHES)]
+    def batches_for(m, n=N_BATCHES):
+        return [inputs.make_ids(m, sh.V, seed=rank_seeds(rank, 0, b, m)["ids"], device=dev) for b in range(n)]
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
+    def plain_step(mode, kernel=mole.KERNEL_AUTO):
+        def step(ids, out, tmp, status):
+            mole.decode_step_args(hidden, ids, luts, wrs, out, tmp, status=status, mode=mode, kernel=kernel)
+        return step
+
     # ---- headline: K steps of the L-layer decode step as a model that runs other work between the layers
     # gets it: one launch per layer, chained with programmatic dependent launch, the layer's output the next
     # layer's hidden state, the L launches of a step replayed from a CUDA graph -----------------------------
-    hidden = hidden_all[:M].contiguous()
-    fused = False
-    graphs = StepGraphs(mole, luts, wrs, hidden, batches_for(M), mode=mole.STEP_CHAINED)
-    graphs.run(0, max(args.warmup, 3))
-    barrier()
-    with ClockSampler(physical_gpu_index(local_rank)) as clocks:
-        ms = timed_ms(torch, lambda: graphs.run(0, args.steps))
-    barrier()
-    assert int(graphs.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
-    ms = max_over_ranks(ms, dist, dev)
+    graphs = StepGraphs(torch, plain_step(mole.STEP_CHAINED), hidden, batches_for(M))
+    clocks = ClockSampler(physical_gpu_index(local_rank))
+    ms, spread = timed_steps(torch, graphs.run, args.steps, args.warmup, barrier, dist, dev, sampler=clocks)
+    assert graphs.ok(), "a kernel reported a bad id or a timed-out wait"
+    last_ids = graphs.id_batches[(args.steps - 1) % N_BATCHES]
+    headline_out = graphs.out.clone()  # the last timed step's result (every repeat ends on the same id batch)
     ms_per_step = ms / args.steps
     value = whole_job_tokens_per_s(world, M, args.steps, ms)
-    launches = args.steps * (1 if fused else L)
-    launch_bytes = sh.step_bytes(M, L) if fused else sh.layer_bytes(M)
+    launches = args.steps * L
+    launch_bytes = sh.layer_bytes(M)
     achieved = launch_bytes / (ms * 1e-3 / launches) / 1e9
+    kernel_name = mole.variant(M, sh.N, sh.d)[0]
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(sh, L, M, args),
+        "timing": dict(spread, what=f"the timed region of {args.steps} steps repeated {spread['repeats']} times "
+                                    "(barrier + synchronise around each); value from the median repeat"),
         "tokens_per_s_per_layer": value * L,
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC.get((sh.name, M, L)), "kernel": "mole_step_kernel", "peak_source": peak_src,
+                     "traffic": TRAFFIC.get((sh.name, M, L)), "kernel": kernel_name, "peak_source": peak_src,
                      "launch": "one launch per layer (%d per step), chained with programmatic dependent launch" % L,
                      "algorithmic_bytes_per_launch": launch_bytes, "us_per_launch": ms * 1e3 / launches},
         "clocks": clocks.summary(),
     }
+    del graphs
 
     # ---- extra, never the headline: the same step as ONE launch that keeps a token's chain through all L
     # layers on chip (what mole_decode_step picks by itself up to 4096 tokens) ------------------------------
-    del graphs
+    fused_out = None
     if L > 1 and M <= 4096:
-        g = StepGraphs(mole, luts, wrs, hidden, batches_for(M), mode=mole.STEP_FUSED)
-        g.run(0, max(args.warmup, 3))
-        barrier()
-        ms_f = max_over_ranks(timed_ms(torch, lambda: g.run(0, args.steps)), dist, dev)
-        barrier()
-        assert int(g.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
+        g = StepGraphs(torch, plain_step(mole.STEP_FUSED), hidden, batches_for(M))
+        ms_f, spread_f = timed_steps(torch, g.run, args.steps, args.warmup, barrier, dist, dev)
+        assert g.ok(), "a kernel reported a bad id or a timed-out wait"
         fb = sh.step_bytes(M, L)
         gbs = fb / (ms_f * 1e-3 / args.steps) / 1e9
         line["fused_step"] = {"what": "all %d layers of a step in one launch (layer-batched), an extra beside the headline" % L,
                               "value": whole_job_tokens_per_s(world, M, args.steps, ms_f), "unit": UNIT,
                               "us_per_step": ms_f * 1e3 / args.steps, "algorithmic_bytes_per_launch": fb,
-                              "achieved": gbs, "frac": gbs / peak, "traffic": FUSED_TRAFFIC.get((sh.name, M, L))}
+                              "achieved": gbs, "frac": gbs / peak, "traffic": FUSED_TRAFFIC.get((sh.name, M, L)),
+                              "kernel": mole.variant(M, sh.N, sh.d, L=L)[0], "repeats": spread_f["repeats"]}
+        fused_out = g.out.clone()
         del g
 
-    # ---- extra: the chained step with RMSNorm fused in front of every layer's router (App. A.2 listing) ----
-    if rank == 0:
+    # ---- extra: the chained and the fused step with RMSNorm in front of every layer's router (App. A.2
+    # listing), through the same C entry point ---------------------------------------------------------------
+    if extras:
         gammas = torch.stack([inputs.make_router(sh.d, 1, seed=2500 + l, device=dev).reshape(sh.d) + 1.0 for l in range(L)])
-        g = NormStepGraphs(mole, luts, wrs, gammas, hidden, batches_for(M))
-        g.run(0, max(args.warmup, 3))
-        torch.cuda.synchronize()
-        steps_n = min(args.steps, 2000)
-        ms_n = timed_ms(torch, lambda: g.run(0, steps_n))
-        assert int(g.status.item()) == 0, "a kernel reported a bad id or a timed-out wait"
-        us_layer_n = ms_n * 1e3 / (steps_n * L)
-        line["norm_router_step"] = {"what": "chained step whose routers read RMSNorm(hidden), fused into the layer kernel",
-                                    "us_per_layer": us_layer_n, "value": M / (us_layer_n * L * 1e-6), "unit": UNIT,
-                                    "achieved": sh.layer_bytes(M) / us_layer_n / 1e3,
-                                    "frac": sh.layer_bytes(M) / us_layer_n / 1e3 / peak}
-        del g
+        norm = {}
+        for name, mode in (("chained", mole.STEP_CHAINED), ("fused", mole.STEP_FUSED)):
+            if mode == mole.STEP_FUSED and not (L > 1 and M <= 4096):
+                continue
+
+            def step(ids, out, tmp, status, mode=mode):
+                mole.decode_step_args(hidden, ids, luts, wrs, out, tmp, status=status, mode=mode, norm_weights=gammas,
+                                      norm_eps=1e-5)
+
+            g = StepGraphs(torch, step, hidden, batches_for(M, N_BATCHES_EXTRA))
+            k = min(args.steps, 500)
+            ms_n, _ = timed_steps(torch, g.run, k, min(args.warmup, 20))
+            assert g.ok(), "a kernel reported a bad id or a timed-out wait"
+            us = ms_n * 1e3 / k
+            nbytes = L * sh.layer_bytes(M) if mode == mole.STEP_CHAINED else sh.step_bytes(M, L)
+            norm[name] = {"us_per_step": us, "us_per_layer": us / L, "value": M / (us * 1e-6), "unit": UNIT,
+                          "achieved": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+                          "kernel": mole.variant(M, sh.N, sh.d, L=L if mode == mole.STEP_FUSED else 1, norm=True)[0]}
+            del g
+        line["norm_router_step"] = dict(norm, what="the step with every router reading RMSNorm(hidden), fused into the layer "
+                                                   "kernels (mole_decode_step_args with norm weights)")
 
     # ---- end to end: host buffers in, host buffer out, through the C ABI, every step ---------------------
     h_host = hidden.cpu().pin_memory()
@@ -486,7 +649,7 @@ def run_mole(args):
     ids_host = [b.cpu().pin_memory() for b in batches_for(M)]
     dev_bufs = [torch.empty_like(hidden) for _ in range(3)]
     dev_ids = torch.empty(M, dtype=torch.int32, device=dev)
-    e2e_steps = min(args.steps, 2000)
+    e2e_steps = min(args.steps, 1000)
 
     def e2e_call(k):
         mole.decode_step_host(h_host, ids_host[k % N_BATCHES], out_host, dev_bufs[0], dev_ids, dev_bufs[1],
@@ -502,95 +665,86 @@ def run_mole(args):
             e2e_call(k)
         e2e_graphs.append(g)
 
-    def e2e_run(n):
-        for k in range(n):
+    def e2e_run(k0, k1):
+        for k in range(k0, k1):
             e2e_graphs[k % N_BATCHES].replay()
             torch.cuda.current_stream().synchronize()  # the caller reads out_host after every step
 
-    e2e_run(max(3, min(args.warmup, 50)))
-    barrier()
-    t0 = time.perf_counter()
-    ms_e2e = timed_ms(torch, lambda: e2e_run(e2e_steps))
-    wall_e2e = time.perf_counter() - t0
-    barrier()
-    ms_e2e = max_over_ranks(ms_e2e, dist, dev)
+    ms_e2e, spread_e = timed_steps(torch, e2e_run, e2e_steps, min(args.warmup, 50), barrier, dist, dev)
     line["e2e"] = {"value": whole_job_tokens_per_s(world, M, e2e_steps, ms_e2e), "unit": UNIT,
                    "h2d_bytes_per_step": M * sh.d * 2 + M * 4, "d2h_bytes_per_step": M * sh.d * 2,
-                   "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
+                   "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps, "repeats": spread_e["repeats"],
                    "how": "mole_decode_step_host captured into one CUDA graph per id batch: pinned host hidden+ids -> device, "
                           "the step as mole_decode_step launches it by itself (one fused launch over all layers up to "
                           "4096 tokens), result -> pinned host; one graph launch and one stream synchronisation per step"}
+    e2e_out = out_host.clone()
+    del e2e_graphs
 
-    # ---- sweep over the configuration's batch sizes: chained step + isolated launches -----------------------
-    if not args.no_sweep and rank == 0:
-        sweep = []
-        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-        for m in sh.batches:
-            if m * sh.d * 2 > 2**31:
-                continue
-            hid = hidden_all[:m].contiguous()
-            bl = batches_for(m)
-            steps_m = max(50, min(args.steps, int(2e6 // max(m, 64))))
-            g = StepGraphs(mole, luts, wrs, hid, bl, mode=mole.STEP_CHAINED)
-            g.run(0, 20)
-            torch.cuda.synchronize()
-            ms_m = timed_ms(torch, lambda: g.run(0, steps_m))
-            us_layer = ms_m * 1e3 / (steps_m * L)
-            del g
-            us_fused = None
-            if m <= 4096:
-                g = StepGraphs(mole, luts, wrs, hid, bl, mode=mole.STEP_FUSED)
-                g.run(0, 20)
-                torch.cuda.synchronize()
-                us_fused = timed_ms(torch, lambda: g.run(0, steps_m)) * 1e3 / steps_m
-                del g
-            # isolated single launches of layer 0: steady (rotating ids) and cold (L2 flushed before each)
-            out = torch.empty_like(hid)
-            reps = 200 if m <= 1024 else 20
-            iso = []
-            for cold in (False, True):
-                ts = []
-                for r in range(reps):
-                    # keep the GPU busy while the host queues the events and the launch, so that the interval
-                    # between the events holds the launch alone: an L2 flush (cold) or a spin that touches no memory
-                    if cold:
-                        flush.fill_(r & 0xFF)
-                    else:
-                        torch.cuda._sleep(100000)
-                    ts.append(timed_ms(torch, lambda: mole.layer_forward(hid, bl[r % N_BATCHES], luts[0], wrs[0], out)))
-                iso.append(statistics.median(ts) * 1e3)
-            nbytes = sh.layer_bytes(m)
-            fb = sh.step_bytes(m, L)
-            sweep.append({
-                "batch": m,
-                "fused_us_per_step": us_fused, "fused_tokens_per_s_all_layers": (m / (us_fused * 1e-6)) if us_fused else None,
-                "fused_GBps": (fb / us_fused / 1e3) if us_fused else None,
-                "fused_frac_of_peak": (fb / us_fused / 1e3 / peak) if us_fused else None,
-                "chained_us_per_layer": us_layer, "tokens_per_s_all_layers": m / (us_layer * L * 1e-6),
-                "tokens_per_s_per_layer": m / (us_layer * 1e-6), "chained_GBps": nbytes / us_layer / 1e3,
-                "chained_frac_of_peak": nbytes / us_layer / 1e3 / peak,
-                "isolated_steady_us": iso[0], "isolated_cold_us": iso[1],
-                "isolated_cold_GBps": nbytes / iso[1] / 1e3,
-                "plan_layer": mole.plan(m, sh.N, sh.d), "plan_fused": mole.plan(m, sh.N, sh.d, mole.DTYPE_BF16, 0, L),
-            })
-        line["sweep"] = sweep
-        del flush
+    # ---- sweep over the configuration's batch sizes: chained + fused steps, isolated launches ---------------
+    if extras and not args.no_sweep:
+        rows = config_rows(torch, mole, inputs, sh, L, luts, wrs, sh.batches, args.steps, args.warmup, peak, dev)
+        iso = {r["batch"]: r for r in isolated_rows(torch, mole, inputs, sh, luts, wrs, sh.batches, peak, dev)}
+        for r in rows:
+            r.update({k: v for k, v in iso.get(r["batch"], {}).items() if k != "batch"})
+        line["sweep"] = rows
 
-    # ---- the CPU oracle beside it (rank 0, N = 1 only) ------------------------------------------------------
+    # ---- the CPU oracle beside it (rank 0, N = 1 only): timed on a bounded sample of the same workload, and
+    # its outputs compared with the GPU's for the last timed step ----------------------------------------------
     if not args.no_cpu and rank == 0 and world == 1:
         import oracle
 
         cores = oracle.effective_threads(len(os.sched_getaffinity(0)))
         table0 = host_bits(luts[0])
         ids_np = [b.cpu().numpy().astype(np.int64) for b in batches_for(M)]
-        v_all, calls, dt = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 12.0, cores)
-        v_one, calls1, dt1 = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 5.0, 1)
+        v_all, calls, dt = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 10.0, cores)
+        v_one, calls1, dt1 = time_oracle(table0, host_bits(wrs[0]), host_bits(hidden), ids_np, L, 4.0, 1)
+        del table0
+        parity = {}
+        ratio, secs = oracle_chain_check(luts, wrs, hidden, last_ids, headline_out, cores)
+        parity["chained_step"] = {"max_err_over_bound": ratio, "ok": ratio <= 1.0}
+        if fused_out is not None:
+            ratio_f, _ = oracle_chain_check(luts, wrs, hidden, last_ids, fused_out, cores)
+            parity["fused_step"] = {"max_err_over_bound": ratio_f, "ok": ratio_f <= 1.0}
+        e2e_ids = ids_host[(e2e_steps - 1) % N_BATCHES].to(dev)
+        ratio_e, _ = oracle_chain_check(luts, wrs, hidden, e2e_ids, e2e_out.to(dev), cores)
+        parity["e2e_step"] = {"max_err_over_bound": ratio_e, "ok": ratio_e <= 1.0}
         line["cpu_baseline"] = {
             "value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{calls} calls of the oracle's lookup-form layer (fp64) on a host copy of layer 0's table, "
                       f"{M} tokens each, {dt:.1f} s; tokens/s divided by L={L} for the L-layer step",
             "single_thread_value": v_one,
+            "parity_of_the_last_timed_step": dict(parity, what=f"the oracle's {L}-layer chain on all {M} tokens of the last timed "
+                                                  "step's id batch against the GPU's output, element by element; bound "
+                                                  f"{L} x 2^-7 x max(1, |ref|)"),
         }
+        assert all(v["ok"] for v in parity.values() if isinstance(v, dict)), parity
+
+    del luts, wrs
+    torch.cuda.empty_cache()
+
+    # ---- the other workload shapes, their quantised tables, the offload mode (one GPU only) ------------------
+    if extras and not args.no_configs:
+        configs = {}
+        for name in ("160m", "410m", "1b"):
+            if name == sh.name:
+                continue
+            osh = inputs.SHAPES[name]
+            try:
+                oluts, owrs = make_tables(torch, inputs, osh, osh.L, rank, dev)
+                rows = config_rows(torch, mole, inputs, osh, osh.L, oluts, owrs, osh.batches, args.steps, args.warmup, peak, dev)
+                configs[name] = {"V": osh.V, "d": osh.d, "N": osh.N, "L": osh.L,
+                                 "table_GB": osh.layer_table_bytes * osh.L / 1e9, "rows": rows}
+                del oluts, owrs
+            except Exception as e:  # e.g. not enough device memory for the 105 GB table on a smaller part
+                configs[name] = {"error": f"{type(e).__name__}: {e}"}
+            torch.cuda.empty_cache()
+        if not args.no_offload:
+            try:
+                configs["410m_offload"] = offload_rows(args, torch, mole, inputs, dev)
+            except Exception as e:
+                configs["410m_offload"] = {"error": f"{type(e).__name__}: {e}"}
+        line["configs"] = configs
+    line["bench_wall_s"] = time.perf_counter() - t_start
 
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -600,14 +754,113 @@ def run_mole(args):
 
 
 # ------------------------------------------------------------------------------------------------------
-# offload mode: table in pinned host memory (410M-shaped by default), one JSON line of its own
+# offload mode: table in pinned host memory (410M-shaped)
 # ------------------------------------------------------------------------------------------------------
 
-def run_offload(args):
-    """Per decode step and layer: dedup the ids on the device, let the GPU fetch the distinct rows
-    from the pinned host table into an HBM staging buffer (side stream), combine from staging (main
-    stream); layer l+1's fetch overlaps layer l's combine through two buffers (mole_offload_decode_step)."""
+def offload_rows(args, torch, mole, inputs, dev, formats=("bf16", "nf4", "nf3")):
+    """Per decode step: dedup the ids on the device, let the GPU fetch the distinct rows from the pinned host
+    table into an HBM staging buffer (side stream), combine from staging (main stream); the next layers'
+    fetch overlaps the current layers' combine through two buffers (mole_offload_decode_step).  Rows for the
+    bf16 host table and for the host table quantised to NF4 / NF3 (packed records cross the link)."""
     import numpy as np
+
+    sh = inputs.SHAPES["410m"]
+    L = args.layers or sh.L
+    result = {"V": sh.V, "d": sh.d, "N": sh.N, "L": L, "context_tokens": OFFLOAD_CONTEXT_TOKENS}
+    tmp = torch.empty((sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
+    side = torch.cuda.Stream()
+    link = None
+    for tag in formats:
+        fmt = {"bf16": mole.LUT_PLAIN, "nf4": mole.LUT_NF4, "nf3": mole.LUT_NF3}[tag]
+        block = QUANT_BLOCKS["410m"].get(tag, 0)
+        row_bytes = sh.row_bytes if fmt == mole.LUT_PLAIN else mole.quant_record_bytes(sh.N, sh.d, fmt, block)
+        # the host table, layer by layer (generated on the device, copied down once, outside any timed region)
+        packed = None
+        if fmt == mole.LUT_PLAIN:
+            host = mole.HostTable((L, sh.V, sh.N, sh.d), torch.bfloat16)
+        else:
+            host = mole.HostTable((L, sh.V, row_bytes), torch.uint8)
+            packed = torch.zeros((sh.V, row_bytes), dtype=torch.uint8, device=dev)
+        for l in range(L):
+            inputs.make_table(sh.V, sh.N, sh.d, seed=1000 + l, device=dev, out=tmp)
+            if fmt == mole.LUT_PLAIN:
+                host.tensor[l].copy_(tmp)
+            else:
+                mole.QuantTable.quantize(tmp, fmt, block, out=packed)
+                host.tensor[l].copy_(packed)
+        torch.cuda.synchronize()
+        if link is None:
+            # host link, measured: a large pinned host -> device copy, and the GPU-initiated read of the same bytes
+            nrows = 8192
+            big = torch.empty((nrows, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+            src = host.tensor[0][:nrows]
+            big.copy_(src, non_blocking=True)
+            torch.cuda.synchronize()
+            ms_copy = min(event_ms(torch, lambda: big.copy_(src, non_blocking=True)) for _ in range(5))
+            uniq_all = torch.arange(nrows, dtype=torch.int32, device=dev)
+            cnt_all = torch.tensor([nrows], dtype=torch.int32, device=dev)
+            mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)
+            torch.cuda.synchronize()
+            ms_fetch = min(event_ms(torch, lambda: mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)) for _ in range(5))
+            link = {"memcpy_GBps": nrows * sh.row_bytes / ms_copy / 1e6, "gpu_read_GBps": nrows * sh.row_bytes / ms_fetch / 1e6}
+            link["peak_GBps"] = max(link["memcpy_GBps"], link["gpu_read_GBps"])
+            link["peak_source"] = ("measured in this run: the faster of cudaMemcpyAsync and a GPU-initiated read of 8192 rows "
+                                   "of the pinned table")
+            del big
+        rows = []
+        for M in OFFLOAD_BATCHES:
+            # one context sized for a server's largest batch (256 tokens: two staging areas): at the batches timed
+            # here a staging area has room for several layers' rows, fetched in one launch
+            ctx = mole.OffloadContext(OFFLOAD_CONTEXT_TOKENS, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2, lut_format=fmt,
+                                      lut_block=block)
+            hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
+            bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
+            id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
+            status = torch.zeros(1, dtype=torch.int32, device=dev)
+            uniq_rows = float(np.mean([len(np.unique(b.cpu().numpy())) for b in id_batches]))
+
+            def step(k):  # one call per step: one dedup, the next layers' fetch under the current layers' combine
+                ctx.decode_step(hidden, id_batches[k % N_BATCHES], host.tensor, wrs, bufs[0], bufs[1], status=status,
+                                side_stream=side)
+
+            steps = max(20, min(args.steps, 200))
+            for k in range(max(min(args.warmup, 10), 3)):
+                step(k)
+            torch.cuda.synchronize()
+            us_calls = event_ms(torch, lambda: [step(k) for k in range(steps)]) * 1e3 / steps
+            torch.cuda.synchronize()
+            # the same steps replayed from CUDA graphs (one per id batch; the side stream joins the capture)
+            graphs = []
+            for k in range(N_BATCHES):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    step(k)
+                graphs.append(g)
+
+            def run(k0, k1):
+                for k in range(k0, k1):
+                    graphs[k % N_BATCHES].replay()
+
+            ms, spread = timed_steps(torch, run, steps, 5)
+            assert int(status.item()) == 0
+            del graphs
+            us_step = ms * 1e3 / steps
+            link_bytes = uniq_rows * row_bytes * L  # distinct rows only cross the link
+            rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
+                         "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
+                         "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link["peak_GBps"],
+                         "us_per_step_without_graph": us_calls, "repeats": spread["repeats"]})
+            ctx.destroy()
+        result[tag] = {"row_bytes": row_bytes, "host_table_GB": row_bytes * sh.V * L / 1e9, "rows": rows}
+        host.free()
+        del packed
+    result["host_link"] = link
+    return result
+
+
+def run_offload(args):
+    """--offload: the offload mode alone, one JSON line of its own."""
     import torch
 
     from paper_2503_15798_b200 import binding as mole
@@ -617,105 +870,24 @@ def run_offload(args):
     lib_build.build()
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    cfg = args.config if args.config != "160m" else "410m"
-    sh = inputs.SHAPES[cfg]
-    L = args.layers or sh.L
-    row_bytes = sh.row_bytes
-
-    # the host table, layer by layer (generated on the device, copied down once, outside any timed region)
-    host = mole.HostTable((L, sh.V, sh.N, sh.d), torch.bfloat16)
-    tmp = torch.empty((sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
-    for l in range(L):
-        inputs.make_table(sh.V, sh.N, sh.d, seed=1000 + l, device=dev, out=tmp)
-        host.tensor[l].copy_(tmp)
-    torch.cuda.synchronize()
-    wrs = torch.stack([inputs.make_router(sh.d, sh.N, seed=2000 + l, device=dev) for l in range(L)])
-
-    # host link, measured: a large pinned host -> device copy, and the GPU-initiated read of the same bytes
-    nrows = 8192
-    big = torch.empty((nrows, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
-    src = host.tensor[0][:nrows]
-    big.copy_(src, non_blocking=True)
-    torch.cuda.synchronize()
-    ms_copy = min(timed_ms(torch, lambda: big.copy_(src, non_blocking=True)) for _ in range(5))
-    link_copy = nrows * row_bytes / ms_copy / 1e6
-    uniq_all = torch.arange(nrows, dtype=torch.int32, device=dev)
-    cnt_all = torch.tensor([nrows], dtype=torch.int32, device=dev)
-    mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)
-    torch.cuda.synchronize()
-    ms_fetch = min(timed_ms(torch, lambda: mole.fetch_rows(host.tensor[0], uniq_all, cnt_all, nrows, big)) for _ in range(5))
-    link_fetch = nrows * row_bytes / ms_fetch / 1e6
-    del big
-
-    rows = []
-    side = torch.cuda.Stream()
-    for M in (1, 8, 64):
-        # one context sized for a server's largest batch (256 tokens: two staging areas of 8 MB): at the batches
-        # timed here a staging area has room for several layers' rows, fetched in one launch and run as one
-        # fused launch
-        ctx = mole.OffloadContext(OFFLOAD_CONTEXT_TOKENS, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2)
-        hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
-        bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
-        id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
-        status = torch.zeros(1, dtype=torch.int32, device=dev)
-        uniq_rows = float(np.mean([len(np.unique(b.cpu().numpy())) for b in id_batches]))
-
-        luts_host = host.tensor  # [L][V][N][d], pinned and device-mapped
-
-        def step(k):  # one call per step: one dedup, layer l+1's fetch under layer l's combine
-            ctx.decode_step(hidden, id_batches[k % N_BATCHES], luts_host, wrs, bufs[0], bufs[1], status=status,
-                            side_stream=side)
-
-        steps = max(20, min(args.steps, 400))
-        for k in range(max(args.warmup, 3)):
-            step(k)
-        torch.cuda.synchronize()
-        ms = timed_ms(torch, lambda: [step(k) for k in range(steps)])
-        torch.cuda.synchronize()
-        assert int(status.item()) == 0
-        us_calls = ms * 1e3 / steps
-        # the same steps replayed from CUDA graphs (one per id batch; the side stream joins the capture):
-        # at small batches the 2L+1 launches of a step are otherwise bound by the host's launch rate
-        graphs = []
-        for k in range(N_BATCHES):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                step(k)
-            graphs.append(g)
-        for k in range(max(args.warmup, 3)):
-            graphs[k % N_BATCHES].replay()
-        torch.cuda.synchronize()
-        ms = timed_ms(torch, lambda: [graphs[k % N_BATCHES].replay() for k in range(steps)])
-        torch.cuda.synchronize()
-        assert int(status.item()) == 0
-        del graphs
-        us_step = ms * 1e3 / steps
-        link_bytes = uniq_rows * row_bytes * L  # distinct rows only cross the link
-        rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
-                     "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
-                     "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link_fetch,
-                     "launches_per_step": 1 + 2 * offload_groups(L, M, row_bytes),  # dedup + (fetch + layers) per group
-                     "us_per_step_without_graph": us_calls})
-        ctx.destroy()
-    top = rows[-1]
+    res = offload_rows(args, torch, mole, inputs, dev)
+    top = res["bf16"]["rows"][-1]
+    steps = max(20, min(args.steps, 200))
     line = {
         "metric": "MoLE offload-mode tokens/s (L-layer decode step) and achieved host-link GB/s", "value": top["tokens_per_s"],
-        "unit": UNIT, "n_gpus": 1, "steps": max(20, min(args.steps, 400)), "warmup": max(args.warmup, 3),
+        "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": max(min(args.warmup, 10), 3),
         "ms_per_step": top["us_per_step"] / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{sh.name}-shaped offload decode: table {sh.layer_table_bytes * L / 1e9:.2f} GB in pinned host "
-                               f"memory, L={L}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
-                   "V": sh.V, "d": sh.d, "N": sh.N, "L": L, "batch": 64,
+        "config": {"workload": f"410m-shaped offload decode: table {res['bf16']['host_table_GB']:.2f} GB in pinned host "
+                               f"memory, L={res['L']}, batch 64x1 (sweep 1, 8, 64), ids Zipf(1.1)",
+                   "V": res["V"], "d": res["d"], "N": res["N"], "L": res["L"], "batch": 64,
                    "l2": "rows come from host memory; 32 rotating id batches, one CUDA graph per batch"},
-        "gpu_launches": top["launches_per_step"] * max(20, min(args.steps, 400)),
-        "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": link_fetch, "unit": "GB/s",
+        "gpu_launches": (1 + 2 * offload_groups(res["L"], 64, res["bf16"]["row_bytes"])) * steps,
+        "roofline": {"bound": "host-link", "achieved": top["link_GBps"], "peak": res["host_link"]["peak_GBps"], "unit": "GB/s",
                      "frac": top["frac_of_link"], "traffic": None, "kernel": "mole_fetch_kernel",
-                     "peak_source": "measured in this run: GPU-initiated read of 8192 rows of the pinned table "
-                                    f"({link_fetch:.1f} GB/s; cudaMemcpyAsync of the same bytes {link_copy:.1f} GB/s)"},
-        "host_link": {"memcpy_GBps": link_copy, "gpu_read_GBps": link_fetch},
-        "sweep": rows,
+                     "peak_source": res["host_link"]["peak_source"]},
+        "offload": res,
     }
-    host.free()
     print(json.dumps(line), flush=True)
 
 

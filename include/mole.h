@@ -62,6 +62,7 @@ extern "C" {
 #define MOLE_ERR_CUDA 3              /* a CUDA runtime call failed; see mole_last_cuda_error() */
 #define MOLE_ERR_NOMEM 4             /* an allocation inside create()/host_alloc() failed */
 #define MOLE_ERR_TOO_LARGE 5         /* size beyond a stated maximum */
+#define MOLE_ERR_IO 6                /* a table file could not be opened, read or written, or is not a table file */
 
 /* bits OR-ed by kernels into an optional device status word (uint32_t, caller zeroes it) */
 #define MOLE_STATUS_BAD_ID 1u  /* some id was outside [0, V) */
@@ -84,6 +85,11 @@ extern "C" {
 #define MOLE_KERNEL_RING 1   /* persistent blocks, rows and router chunks streamed through a shared-memory ring: any shape */
 #define MOLE_KERNEL_DECODE 2 /* one block per token, rows held in registers, built for decode batches: bf16, N of 4, 8, \
                                 16 or 32, d a multiple of 128 up to 2048 (1024 for N = 32), d_split 0 */
+
+/* storage of a table (mole_args.lut_format): plain elements of `dtype`, or the quantised records of Sec. 4.5 / Table 8 */
+#define MOLE_LUT_PLAIN 0
+#define MOLE_LUT_NF4 1 /* 4-bit NormalFloat codes, one float32 absmax scale per block (paper: block 768 -> 25.3 % of FP16) */
+#define MOLE_LUT_NF3 2 /* 3-bit NormalFloat codes, one float16 absmax scale per block (paper: block 128 -> 19.5 % of FP16) */
 
 /* mole_decode_step_ex mode: how the L layers of a step are launched */
 #define MOLE_STEP_AUTO 0    /* fused unless the batch is large (then chained) */
@@ -143,6 +149,12 @@ typedef struct mole_args {
                               App. A.2 listing, whose router input is the normalised state and whose residual is
                               not.  The normalisation happens in shared memory inside the same kernel. */
     float norm_eps;        /* >= 0; read only with norm_weight */
+    int32_t lut_format;    /* MOLE_LUT_*.  NF4 / NF3: `lut` points to V packed records of mole_quant_record_bytes() bytes
+                              each (written by mole_quantize_lut) instead of [V][N][d] elements; the layer gathers a
+                              token's record and de-quantises inside the weighted sum: out = res + sum_j g_j *
+                              (codebook[code] * scale).  bf16 activations, N of 4, 8, 16 or 32, d a multiple of 128 up
+                              to 2048, d_split 0; MOLE_ERR_UNSUPPORTED_SHAPE otherwise. */
+    int32_t lut_block;     /* elements per quantisation block (a multiple of 32 that divides d); read only with NF4 / NF3 */
     int32_t reserved2;     /* must be 0 */
 } mole_args;
 
@@ -214,6 +226,8 @@ typedef struct mole_step_args {
     int32_t kernel;        /* as mole_args.kernel, for the single-layer launches of CHAINED mode; a FUSED step of
                               several layers always runs on the ring kernel */
     float norm_eps;        /* >= 0; read only with norm_weight_base */
+    int32_t lut_format;    /* as mole_args.lut_format; quantised tables run as CHAINED steps (AUTO picks that) */
+    int32_t lut_block;     /* as mole_args.lut_block */
     int32_t reserved;      /* must be 0 */
     void *stream;          /* cudaStream_t */
 } mole_step_args;
@@ -233,6 +247,32 @@ MOLE_API int mole_decode_step_host(const void *hidden_host, const int32_t *ids_h
                           int64_t lut_layer_stride_bytes, const void *w_router_base,
                           int64_t wr_layer_stride_bytes, uint32_t *status, int L, int B, int T, int N, int d,
                           int V, int dtype, void *stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Quantised tables (Sec. 4.5, Table 8): post-training quantisation of a 16-bit table to the NF4 / NF3
+ * NormalFloat types of the QLoRA paper, block-wise absmax scaling.  Per block: scale = max |x| (stored as
+ * float32 for NF4, as the float16 rounding of min(max, 65504) for NF3); every element takes the code of the
+ * codebook value nearest to x / scale (decided in float32, a value on a midpoint takes the lower code);
+ * de-quantised value = codebook[code] * scale.  A block never straddles two (id, expert) rows.
+ * Record of one id, the unit that is gathered (zero padded to a multiple of 16 bytes):
+ *   NF4: N rows of d/2 bytes (byte i: code 2i in the low, code 2i+1 in the high nibble), then N*d/block float32 scales;
+ *   NF3: N rows of d/4 bytes with the codes' two low bits (byte i: codes 4i..4i+3, code 4i+k at bits 2k, 2k+1), N rows
+ *        of d/8 bytes with their high bits (byte i: codes 8i..8i+7, code 8i+k at bit k), then N*d/block float16 scales.
+ * ------------------------------------------------------------------------------------- */
+
+/* the 16 (NF4) or 8 (NF3) codebook values in ascending order: quantiles of N(0,1) at evenly spaced
+ * probabilities, one more on the positive side so that zero is exact, scaled to [-1, 1].  Host arithmetic. */
+MOLE_API int mole_nf_codebook(int lut_format, float *values);
+
+/* bytes of one id's record; N 1..64, d a multiple of 32, block a multiple of 32 that divides d */
+MOLE_API int mole_quant_record_bytes(int N, int d, int lut_format, int block, int64_t *bytes);
+
+/* mole_quantize_lut -- quantise a bf16 table on the device.
+ *   lut    device bf16 [V][N][d]           packed device, V * record_bytes bytes (16-byte aligned; padding bytes of a
+ *                                           record are not written: zero the buffer once if records are compared)
+ * Asynchronous on `stream`. */
+MOLE_API int mole_quantize_lut(const void *lut, void *packed, int64_t V, int N, int d, int lut_format, int block,
+                      void *stream);
 
 /* ---------------------------------------------------------------------------------------
  * Offload mode: the table lives off the accelerator, in pinned host memory, and only the
@@ -304,7 +344,28 @@ MOLE_API int mole_host_free(void *ptr);
 typedef struct mole_offload_ctx mole_offload_ctx;
 
 MOLE_API int mole_offload_create(mole_offload_ctx **ctx, int max_tokens, int N, int d, int V, int dtype, int n_buffers);
+/* ... for a quantised host table (lut_format MOLE_LUT_NF4 / NF3, lut_block as in mole_args): the host
+ * table holds V packed records per layer, only the distinct ids' records cross the host link (25.3 % /
+ * 19.5 % of the 16-bit bytes with the paper's blocks), and the layers de-quantise from the staging area.
+ * MOLE_LUT_PLAIN gives mole_offload_create. */
+MOLE_API int mole_offload_create_ex(mole_offload_ctx **ctx, int max_tokens, int N, int d, int V, int dtype, int n_buffers,
+                           int lut_format, int lut_block);
 MOLE_API int mole_offload_destroy(mole_offload_ctx *ctx);
+
+/*
+ * mole_offload_set_hot_rows -- a cache of hot rows in device memory in front of the host link.  Token ids
+ * follow a heavy-tailed distribution, so a few ids account for most look-ups: the rows of the n_hot ids
+ * listed (distinct, in [0, V), HOST array) are copied once, for all L layers of the host tables at
+ * lut_host_base + l*lut_layer_stride_bytes, into n_hot*L*row_bytes bytes of device memory (plus a V-entry
+ * index); every later fetch from one of those tables takes a listed id's row from there instead of across
+ * the link.  Results do not change by a bit.  Synchronous (it waits for the device); replaces an earlier
+ * set; n_hot == 0 frees it.  The host tables must not change while they are mirrored.
+ * mole_offload_hot_hits reads (and optionally resets) the number of (row, layer) fetches the cache served;
+ * it waits for the device's queued work.
+ */
+MOLE_API int mole_offload_set_hot_rows(mole_offload_ctx *ctx, const int32_t *hot_ids_host, int n_hot,
+                              const void *lut_host_base, int64_t lut_layer_stride_bytes, int L);
+MOLE_API int mole_offload_hot_hits(mole_offload_ctx *ctx, uint64_t *hits, int reset);
 
 /*
  * mole_offload_prefetch -- on side_stream: wait until buffer `buf`'s previous consumer has
@@ -356,6 +417,32 @@ MOLE_API int mole_offload_decode_step(mole_offload_ctx *ctx, const void *hidden_
 MOLE_API int mole_offload_buffers(mole_offload_ctx *ctx, int buf, const int32_t **uniq, const int32_t **slot,
                          const int32_t **count, const void **staging);
 
+/* ---------------------------------------------------------------------------------------
+ * Table files: the tables of all L layers on a storage device below host memory (Sec. 3.3: the tables stay
+ * offloaded; Sec. 4.2: lower-tier storage).  Layout: a 4096-byte header (magic "MOLELUT1", version, shapes,
+ * element type, table format, bytes per row), then layer after layer, V rows of row_bytes each -- plain
+ * [N][d] elements or the packed records of a quantised table.  Host calls, no CUDA; MOLE_ERR_IO on any
+ * file error (missing, short, not a table file).
+ * ------------------------------------------------------------------------------------- */
+typedef struct mole_table_info {
+    int64_t L, V;
+    int32_t N, d;
+    int32_t dtype;      /* MOLE_DTYPE_* of plain elements (and of the activations a quantised table serves) */
+    int32_t lut_format; /* MOLE_LUT_* */
+    int32_t lut_block;  /* quantisation block, 0 for plain tables */
+    int32_t reserved;
+    int64_t row_bytes;  /* bytes of one id's row: N*d elements, or one packed record */
+} mole_table_info;
+
+/* write L tables from host memory (layer l at tables_host + l*layer_stride_bytes, V rows each) */
+MOLE_API int mole_table_file_write(const char *path, const void *tables_host, int64_t layer_stride_bytes, int L, int V,
+                          int N, int d, int dtype, int lut_format, int lut_block);
+MOLE_API int mole_table_file_info(const char *path, mole_table_info *info);
+/* read layers layer0 .. layer0 + n_layers - 1 into host memory (e.g. from mole_host_alloc), dst_layer_stride_bytes apart */
+MOLE_API int mole_table_file_read(const char *path, void *dst_host, int64_t dst_layer_stride_bytes, int layer0, int n_layers);
+/* read the rows of n ids of one layer, densely, into dst_host (n * row_bytes): a tier that leaves the file on disk */
+MOLE_API int mole_table_file_read_rows(const char *path, int layer, const int32_t *ids_host, int n, void *dst_host);
+
 /* --------------------------------------------------------------------------------------- */
 
 MOLE_API const char *mole_status_string(int code);
@@ -384,12 +471,13 @@ MOLE_API int mole_reload_debug_env(void);
 MOLE_API int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads,
               int *out_smem_bytes, int *out_stages, int *out_blocks_per_sm);
 
-/* Name of the kernel instantiation a launch of this shape runs ("decode<N,NORM>" or
- * "step<storage,N,P,MODE,SHAPE,DIRECT,NORM>"), with its block size and dynamic shared memory: lets a
- * test list which instantiations a workload reaches.  norm != 0: with a normalised router; kernel as
- * mole_args.kernel.  name receives at most name_bytes - 1 characters and a terminator.  Launches nothing. */
-MOLE_API int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, char *name,
-                 int name_bytes, int *out_threads, int *out_smem_bytes);
+/* Name of the kernel instantiation a launch of this shape runs ("decode<N,NORM>", "fstep<N,DB,NORM>",
+ * "qdecode<N,nfB,NORM>" or "step<storage,N,P,MODE,SHAPE,DIRECT,NORM>"), with its block size and dynamic
+ * shared memory: lets a test list which instantiations a workload reaches.  norm != 0: with a normalised
+ * router; kernel as mole_args.kernel; lut_format / lut_block as mole_args (a quantised table: L must be 1).
+ * name receives at most name_bytes - 1 characters and a terminator.  Launches nothing. */
+MOLE_API int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, int lut_format,
+                 int lut_block, char *name, int name_bytes, int *out_threads, int *out_smem_bytes);
 
 #ifdef __cplusplus
 }

@@ -16,12 +16,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmole_b200.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, ERR_NOMEM, ERR_TOO_LARGE = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, ERR_NOMEM, ERR_TOO_LARGE, ERR_IO = range(7)
 STATUS_BAD_ID, STATUS_TIMEOUT = 1, 2
 DTYPE_BF16, DTYPE_F32 = 0, 1
 FLAG_IDS_INT64, FLAG_CHAIN = 1, 2
 STEP_AUTO, STEP_FUSED, STEP_CHAINED = 0, 1, 2
 KERNEL_AUTO, KERNEL_RING, KERNEL_DECODE = 0, 1, 2
+LUT_PLAIN, LUT_NF4, LUT_NF3 = 0, 1, 2
 
 # every symbol include/mole.h declares
 EXPORTS = (
@@ -30,7 +31,8 @@ EXPORTS = (
     "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_decode_step",
     "mole_offload_buffers",
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan", "mole_variant", "mole_reload_debug_env",
-    "mole_decode_step_args",
+    "mole_table_file_write", "mole_table_file_info", "mole_table_file_read", "mole_table_file_read_rows",
+    "mole_decode_step_args", "mole_offload_create_ex", "mole_offload_set_hot_rows", "mole_offload_hot_hits", "mole_nf_codebook", "mole_quant_record_bytes", "mole_quantize_lut",
 )
 
 
@@ -42,7 +44,8 @@ class MoleArgs(ctypes.Structure):
         ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
         ("dtype", c_int32), ("kernel", c_int32), ("d_split", c_int32),
         ("stream", c_void_p),
-        ("norm_weight", c_void_p), ("norm_eps", ctypes.c_float), ("reserved2", c_int32),
+        ("norm_weight", c_void_p), ("norm_eps", ctypes.c_float), ("lut_format", c_int32), ("lut_block", c_int32),
+        ("reserved2", c_int32),
     ]
 
 
@@ -55,9 +58,14 @@ class MoleStepArgs(ctypes.Structure):
         ("out", c_void_p), ("tmp", c_void_p), ("status", c_void_p),
         ("L", c_int32), ("B", c_int32), ("T", c_int32), ("N", c_int32), ("d", c_int32), ("V", c_int32),
         ("dtype", c_int32), ("mode", c_int32), ("d_split", c_int32), ("kernel", c_int32),
-        ("norm_eps", ctypes.c_float), ("reserved", c_int32),
+        ("norm_eps", ctypes.c_float), ("lut_format", c_int32), ("lut_block", c_int32), ("reserved", c_int32),
         ("stream", c_void_p),
     ]
+
+
+class MoleTableInfo(ctypes.Structure):
+    _fields_ = [("L", c_int64), ("V", c_int64), ("N", c_int32), ("d", c_int32), ("dtype", c_int32), ("lut_format", c_int32),
+                ("lut_block", c_int32), ("reserved", c_int32), ("row_bytes", c_int64)]
 
 
 class MoleError(RuntimeError):
@@ -96,6 +104,13 @@ def lib() -> ctypes.CDLL:
         L.mole_host_alloc.argtypes = [POINTER(c_void_p), c_size_t]
         L.mole_host_free.argtypes = [vp]
         L.mole_offload_create.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_int]
+        L.mole_offload_create_ex.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int]
+        L.mole_table_file_write.argtypes = [c_char_p, vp, c_int64, c_int, c_int, c_int, c_int, c_int, c_int, c_int]
+        L.mole_table_file_info.argtypes = [c_char_p, POINTER(MoleTableInfo)]
+        L.mole_table_file_read.argtypes = [c_char_p, vp, c_int64, c_int, c_int]
+        L.mole_table_file_read_rows.argtypes = [c_char_p, c_int, vp, c_int, vp]
+        L.mole_offload_set_hot_rows.argtypes = [vp, vp, c_int, vp, c_int64, c_int]
+        L.mole_offload_hot_hits.argtypes = [vp, POINTER(ctypes.c_uint64), c_int]
         L.mole_offload_destroy.argtypes = [vp]
         L.mole_offload_prefetch.argtypes = [vp, c_int, ip, c_int, vp, vp]
         L.mole_layer_forward_offload.argtypes = [vp, c_int, vp, vp, vp, vp, c_int, c_int, vp]
@@ -109,10 +124,13 @@ def lib() -> ctypes.CDLL:
         L.mole_version.argtypes = []
         L.mole_plan.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
                                 POINTER(c_int), POINTER(c_int), POINTER(c_int)]
-        L.mole_variant.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, ctypes.c_char_p, c_int,
-                                   POINTER(c_int), POINTER(c_int)]
+        L.mole_variant.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, ctypes.c_char_p,
+                                   c_int, POINTER(c_int), POINTER(c_int)]
         L.mole_reload_debug_env.argtypes = []
         L.mole_decode_step_args.argtypes = [POINTER(MoleStepArgs)]
+        L.mole_nf_codebook.argtypes = [c_int, POINTER(ctypes.c_float)]
+        L.mole_quant_record_bytes.argtypes = [c_int, c_int, c_int, c_int, POINTER(c_int64)]
+        L.mole_quantize_lut.argtypes = [vp, vp, c_int64, c_int, c_int, c_int, c_int, vp]
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is not c_char_p:
@@ -151,20 +169,73 @@ def _dev(t: torch.Tensor, name: str):
         raise ValueError(f"{name} must be a contiguous CUDA tensor")
 
 
+class QuantTable:
+    """A table quantised to NF4 / NF3 (Sec. 4.5 of the paper): `packed` is a uint8 device (or pinned host)
+    tensor [V][record_bytes] -- or [L][V][record_bytes] for the tables of L layers -- of the records
+    mole_quantize_lut writes."""
+
+    def __init__(self, packed, N: int, d: int, fmt: int, block: int):
+        self.packed, self.N, self.d, self.fmt, self.block = packed, N, d, fmt, block
+        self.record_bytes = quant_record_bytes(N, d, fmt, block)
+        if packed.dtype != torch.uint8 or packed.shape[-1] != self.record_bytes:
+            raise ValueError("packed must be uint8 [..., V, record_bytes]")
+        self.V = packed.shape[-2]
+
+    def layer(self, l: int) -> "QuantTable":
+        return QuantTable(self.packed[l], self.N, self.d, self.fmt, self.block)
+
+    @staticmethod
+    def quantize(lut, fmt: int, block: int, out=None, stream=None) -> "QuantTable":
+        """mole_quantize_lut: lut bf16 [V][N][d] (or [L][V][N][d]) on the device."""
+        _dev(lut, "lut")
+        if lut.dtype != torch.bfloat16:
+            raise TypeError("mole_quantize_lut takes a bf16 table")
+        N, d = lut.shape[-2], lut.shape[-1]
+        rb = quant_record_bytes(N, d, fmt, block)
+        lead = tuple(lut.shape[:-2])
+        if out is None:
+            out = torch.zeros(lead + (rb,), dtype=torch.uint8, device=lut.device)
+        rows = 1
+        for n in lead:
+            rows *= n
+        _check(lib().mole_quantize_lut(_ptr(lut), _ptr(out), rows, N, d, fmt, block, _stream(stream)), "mole_quantize_lut")
+        return QuantTable(out, N, d, fmt, block)
+
+
+def nf_codebook(fmt: int):
+    """mole_nf_codebook: the codebook values (16 for NF4, 8 for NF3) as Python floats (exact float32 values)."""
+    buf = (ctypes.c_float * 16)()
+    _check(lib().mole_nf_codebook(fmt, buf), "mole_nf_codebook")
+    return [float(buf[i]) for i in range(16 if fmt == LUT_NF4 else 8)]
+
+
+def quant_record_bytes(N: int, d: int, fmt: int, block: int) -> int:
+    b = c_int64()
+    _check(lib().mole_quant_record_bytes(N, d, fmt, block, ctypes.byref(b)), "mole_quant_record_bytes")
+    return b.value
+
+
 def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_out=None, status=None,
                   d_split: int = 0, chain: bool = False, stream=None, B=None, T=None, norm_weight=None,
                   norm_eps: float = 1e-6, kernel: int = KERNEL_AUTO):
-    """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d],
-    w_router [d][N]; returns out (allocated like hidden if not given).  norm_weight [d]: the router
-    reads RMSNorm(hidden) with that scale and norm_eps, the residual stays un-normalised."""
-    for name, t in (("hidden", hidden), ("ids", ids), ("lut", lut), ("w_router", w_router)):
+    """mole_layer_forward_ex.  hidden [M][d] (or [B][T][d]), ids [M] int32/int64, lut [V][N][d] or a
+    QuantTable, w_router [d][N]; returns out (allocated like hidden if not given).  norm_weight [d]: the
+    router reads RMSNorm(hidden) with that scale and norm_eps, the residual stays un-normalised."""
+    quant = lut if isinstance(lut, QuantTable) else None
+    lut_t = quant.packed if quant else lut
+    for name, t in (("hidden", hidden), ("ids", ids), ("lut", lut_t), ("w_router", w_router)):
         _dev(t, name)
-    V, N, d = lut.shape
+    if quant:
+        V, N, d = quant.V, quant.N, quant.d
+        if quant.packed.dim() != 2:
+            raise ValueError("a single layer takes one table: use QuantTable.layer(l)")
+    else:
+        V, N, d = lut.shape
     M = hidden.numel() // d if d else 0
     if hidden.shape[-1] != d or tuple(w_router.shape) != (d, N) or ids.numel() != M:
         raise ValueError("shape mismatch between hidden, ids, lut and w_router")
     tag = _dtype_tag(hidden)
-    if not (lut.dtype == w_router.dtype == hidden.dtype):
+    if not ((quant or lut.dtype == hidden.dtype) and w_router.dtype == hidden.dtype):
         raise TypeError("hidden, lut and w_router must share one element type")
     if out is None:
         out = torch.empty_like(hidden)
@@ -181,7 +252,7 @@ def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_
     a = MoleArgs()
     a.struct_size = ctypes.sizeof(MoleArgs)
     a.flags = flags
-    a.hidden, a.ids, a.lut, a.w_router, a.out = _ptr(hidden), _ptr(ids), _ptr(lut), _ptr(w_router), _ptr(out)
+    a.hidden, a.ids, a.lut, a.w_router, a.out = _ptr(hidden), _ptr(ids), _ptr(lut_t), _ptr(w_router), _ptr(out)
     a.residual, a.gates_out, a.status = _ptr(residual), _ptr(gates_out), _ptr(status)
     a.B, a.T, a.N, a.d, a.V = B, T, N, d, V
     a.dtype, a.kernel, a.d_split = tag, kernel, d_split
@@ -191,6 +262,7 @@ def layer_forward(hidden, ids, lut, w_router, out=None, *, residual=None, gates_
         if norm_weight.dtype != hidden.dtype or norm_weight.numel() != d:
             raise ValueError("norm_weight must be [d] of the element type of hidden")
     a.norm_weight, a.norm_eps, a.reserved2 = _ptr(norm_weight), float(norm_eps), 0
+    a.lut_format, a.lut_block = (quant.fmt, quant.block) if quant else (LUT_PLAIN, 0)
     _check(lib().mole_layer_forward_ex(ctypes.byref(a)), "mole_layer_forward_ex")
     return out
 
@@ -221,14 +293,20 @@ def decode_step(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, str
 def decode_step_args(hidden_in, ids, luts, w_routers, out, tmp=None, status=None, stream=None, mode: int = STEP_AUTO,
                      d_split: int = 0, norm_weights=None, norm_eps: float = 1e-6, kernel: int = KERNEL_AUTO,
                      chain_first: bool = False):
-    """mole_decode_step_args: decode_step with every option; norm_weights [L][d] puts RMSNorm(hidden) in
-    front of every layer's router."""
-    L, V, N, d = luts.shape
+    """mole_decode_step_args: decode_step with every option; luts [L][V][N][d] or a QuantTable with packed
+    [L][V][record_bytes]; norm_weights [L][d] puts RMSNorm(hidden) in front of every layer's router."""
+    quant = luts if isinstance(luts, QuantTable) else None
+    if quant:
+        lut_t = quant.packed
+        L, V, N, d = lut_t.shape[0], quant.V, quant.N, quant.d
+    else:
+        lut_t = luts
+        L, V, N, d = luts.shape
     a = MoleStepArgs()
     a.struct_size = ctypes.sizeof(MoleStepArgs)
     a.flags = FLAG_CHAIN if chain_first else 0
-    a.hidden_in, a.ids, a.lut_base = _ptr(hidden_in), _ptr(ids), _ptr(luts)
-    a.lut_layer_stride_bytes = luts.stride(0) * luts.element_size()
+    a.hidden_in, a.ids, a.lut_base = _ptr(hidden_in), _ptr(ids), _ptr(lut_t)
+    a.lut_layer_stride_bytes = lut_t.stride(0) * lut_t.element_size()
     a.w_router_base, a.wr_layer_stride_bytes = _ptr(w_routers), w_routers.stride(0) * w_routers.element_size()
     if norm_weights is not None:
         _dev(norm_weights, "norm_weights")
@@ -239,6 +317,7 @@ def decode_step_args(hidden_in, ids, luts, w_routers, out, tmp=None, status=None
     a.L, a.B, a.T, a.N, a.d, a.V = L, ids.numel(), 1, N, d, V
     a.dtype, a.mode, a.d_split, a.kernel = _dtype_tag(hidden_in), mode, d_split, kernel
     a.norm_eps, a.reserved = float(norm_eps), 0
+    a.lut_format, a.lut_block = (quant.fmt, quant.block) if quant else (LUT_PLAIN, 0)
     a.stream = _stream(stream)
     _check(lib().mole_decode_step_args(ctypes.byref(a)), "mole_decode_step_args")
     return out
@@ -330,11 +409,13 @@ class HostTable:
 class OffloadContext:
     """mole_offload_create / prefetch / forward / destroy."""
 
-    def __init__(self, max_tokens: int, N: int, d: int, V: int, dtype=torch.bfloat16, n_buffers: int = 2):
+    def __init__(self, max_tokens: int, N: int, d: int, V: int, dtype=torch.bfloat16, n_buffers: int = 2,
+                 lut_format: int = LUT_PLAIN, lut_block: int = 0):
         self.max_tokens, self.N, self.d, self.V, self.dtype, self.n_buffers = max_tokens, N, d, V, dtype, n_buffers
         tag = DTYPE_BF16 if dtype == torch.bfloat16 else DTYPE_F32
         h = c_void_p()
-        _check(lib().mole_offload_create(ctypes.byref(h), max_tokens, N, d, V, tag, n_buffers), "mole_offload_create")
+        _check(lib().mole_offload_create_ex(ctypes.byref(h), max_tokens, N, d, V, tag, n_buffers, lut_format, lut_block),
+               "mole_offload_create_ex")
         self.handle = h.value
 
     def prefetch(self, buf: int, ids, lut_host_layer, side_stream=None):
@@ -357,6 +438,19 @@ class OffloadContext:
                                               _ptr(status), L, M, 1, _stream(stream), _stream(side_stream)),
                "mole_offload_decode_step")
         return out
+
+    def set_hot_rows(self, hot_ids, luts_host):
+        """mole_offload_set_hot_rows: keep the rows of hot_ids (host int32 tensor / array, distinct) of every layer of
+        luts_host ([L][V][...] pinned host tensor) in device memory; an empty list frees the cache."""
+        ids = torch.as_tensor(hot_ids, dtype=torch.int32).contiguous().cpu()
+        L = luts_host.shape[0]
+        _check(lib().mole_offload_set_hot_rows(self.handle, _ptr(ids) if ids.numel() else None, ids.numel(), _ptr(luts_host),
+                                               luts_host.stride(0) * luts_host.element_size(), L), "mole_offload_set_hot_rows")
+
+    def hot_hits(self, reset: bool = False) -> int:
+        h = ctypes.c_uint64()
+        _check(lib().mole_offload_hot_hits(self.handle, ctypes.byref(h), int(reset)), "mole_offload_hot_hits")
+        return h.value
 
     def buffers(self, buf: int):
         """(uniq, slot, count, staging) device pointers of a buffer, as ints."""
@@ -396,12 +490,12 @@ def plan(M: int, N: int, d: int, dtype: int = DTYPE_BF16, d_split: int = 0, L: i
 
 
 def variant(M: int, N: int, d: int, dtype: int = DTYPE_BF16, d_split: int = 0, L: int = 1, norm: bool = False,
-            kernel: int = KERNEL_AUTO):
+            kernel: int = KERNEL_AUTO, lut_format: int = LUT_PLAIN, lut_block: int = 0):
     """mole_variant: (name, threads, smem_bytes) of the kernel instantiation a launch of this shape runs."""
     buf = ctypes.create_string_buffer(96)
     th, sm = c_int(), c_int()
-    _check(lib().mole_variant(M, L, N, d, dtype, d_split, int(norm), kernel, buf, len(buf), ctypes.byref(th),
-                              ctypes.byref(sm)), "mole_variant")
+    _check(lib().mole_variant(M, L, N, d, dtype, d_split, int(norm), kernel, lut_format, lut_block, buf, len(buf),
+                              ctypes.byref(th), ctypes.byref(sm)), "mole_variant")
     return buf.value.decode(), th.value, sm.value
 
 
@@ -427,6 +521,33 @@ class debug_env:
             else:
                 os.environ[k] = old
         _check(lib().mole_reload_debug_env(), "mole_reload_debug_env")
+
+
+def table_file_write(path: str, tables, N: int, d: int, lut_format: int = LUT_PLAIN, lut_block: int = 0):
+    """mole_table_file_write: tables is a CPU tensor [L][V][N][d] (plain) or uint8 [L][V][record_bytes] (quantised)."""
+    t = tables.contiguous()
+    dtype = DTYPE_BF16 if lut_format != LUT_PLAIN else _dtype_tag(t)
+    _check(lib().mole_table_file_write(path.encode(), _ptr(t), t.stride(0) * t.element_size(), t.shape[0], t.shape[1], N, d, dtype,
+                                       lut_format, lut_block), "mole_table_file_write")
+
+
+def table_file_info(path: str) -> MoleTableInfo:
+    info = MoleTableInfo()
+    _check(lib().mole_table_file_info(path.encode(), ctypes.byref(info)), "mole_table_file_info")
+    return info
+
+
+def table_file_read(path: str, dst, layer0: int = 0, n_layers: int = None):
+    """mole_table_file_read into a CPU (ideally pinned) tensor whose first axis is the layer."""
+    n = dst.shape[0] if n_layers is None else n_layers
+    _check(lib().mole_table_file_read(path.encode(), _ptr(dst), dst.stride(0) * dst.element_size(), layer0, n), "mole_table_file_read")
+    return dst
+
+
+def table_file_read_rows(path: str, layer: int, ids, dst):
+    ids = torch.as_tensor(ids, dtype=torch.int32).contiguous().cpu()
+    _check(lib().mole_table_file_read_rows(path.encode(), layer, _ptr(ids), ids.numel(), _ptr(dst)), "mole_table_file_read_rows")
+    return dst
 
 
 def version() -> int:

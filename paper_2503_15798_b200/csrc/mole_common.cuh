@@ -71,6 +71,16 @@ struct StepLaunch {
 };
 int launch_step(const StepLaunch &a);
 
+// kernels that need more than 48 KB of dynamic shared memory opt in once per device
+int ensure_smem_opt_in(const void *fn, int smem);
+// poll limit of the bounded device-side waits (the default unless a debugging variable shortens it)
+uint32_t current_wait_polls();
+
+// the fused layer over a quantised table (mole_quant.cu): single layer, bf16 activations
+bool quant_layer_shape_ok(int N, int d, int format, int block);
+const char *quant_variant_name(int N, int format, bool norm);
+int launch_quant_layer(const StepLaunch &a, int format, int block, uint32_t wait_polls);
+
 #ifdef __CUDACC__
 // ---- device side ---------------------------------------------------------------------------
 

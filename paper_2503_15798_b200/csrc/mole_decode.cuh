@@ -78,6 +78,27 @@ __device__ __forceinline__ unsigned short float_to_bf16_bits(float f)
     return *reinterpret_cast<const unsigned short *>(&b);
 }
 
+// Softmax numerator of expert `lane` (Eq. 4; lanes >= N get 0) from the per-warp partial logits
+// partial[w * N + j]: independent loads, one chain of adds in warp order, exp(z - m) with the maximum m
+// taken only when some logit is large enough for exp to leave the comfortable range (any shift gives
+// the same gates).  Every warp of a block calls it and gets the same values.
+template <int N>
+__device__ __forceinline__ float softmax_numerator(const float *partial, int nwarps, int lane)
+{
+    float z = 0.f;
+    if (lane < N) {
+        float v[kDecodeMaxWarps];
+#pragma unroll
+        for (int w = 0; w < kDecodeMaxWarps; ++w) v[w] = w < nwarps ? partial[w * N + lane] : 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecodeMaxWarps; ++w) z += v[w];
+    }
+    const bool big = lane < N && !(fabsf(z) < 80.f);
+    float zmax = 0.f;
+    if (__any_sync(0xffffffffu, big)) zmax = warp_max(lane < N ? z : -INFINITY);
+    return lane < N ? expf(z - zmax) : 0.f;
+}
+
 // N: experts (4, 8, 16 or 32).  NORM: the router reads RMSNorm(hidden) rounded to bf16 (App. A.2 listing).
 // Launch: one block per token, blockDim.x == d / 4 (a multiple of 32), dynamic shared memory
 // decode_smem_bytes(N, d).
@@ -204,13 +225,7 @@ __global__ void __launch_bounds__(decode_max_threads(N)) mole_decode_kernel(cons
     __syncthreads();
 
     // ---- every warp: logits, softmax numerators (Eq. 4), lane j <-> expert j ----
-    float z = 0.f;
-    if (lane < N)
-        for (int w = 0; w < nwarps; ++w) z += partial[w * N + lane];
-    const bool big = lane < N && !(fabsf(z) < 80.f);
-    float zmax = 0.f;
-    if (__any_sync(0xffffffffu, big)) zmax = warp_max(lane < N ? z : -INFINITY);  // any shift gives the same gates
-    const float e = lane < N ? expf(z - zmax) : 0.f;
+    const float e = softmax_numerator<N>(partial, nwarps, lane);
 
     // ---- weighted sum of the rows (Eq. 8), residual, store ----
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;

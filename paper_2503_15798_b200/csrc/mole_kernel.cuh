@@ -143,7 +143,7 @@ __device__ __forceinline__ float warp_sum(float v)
 // gives up first; everyone else then stops waiting at once.
 // `patient`: sleep after every failed poll (the producer, which runs several items ahead and
 // must not take issue slots from the warps that compute).
-__device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
+static __device__ __noinline__ bool wait_or_give_up(uint64_t *bar, uint32_t parity, volatile int *dead, uint32_t polls,
                                              bool patient = false)
 {
 #pragma unroll 1
@@ -532,18 +532,18 @@ __device__ __forceinline__ void rmsnorm_to_shared(uint32_t src, uint32_t dst, co
 }
 
 // Cold paths, kept out of the consumers' loop body (its size shows in instruction-fetch stalls).
-__device__ __noinline__ void report_timeout(volatile int *dead, uint32_t *status)
+static __device__ __noinline__ void report_timeout(volatile int *dead, uint32_t *status)
 {
     if (!*dead && status) atomicOr(status, MOLE_STATUS_TIMEOUT);
     *dead = 1;
 }
-__device__ __noinline__ void write_gates(float *gates_out, long long t, int N, int lane, float e0, float e1)
+static __device__ __noinline__ void write_gates(float *gates_out, long long t, int N, int lane, float e0, float e1)
 {
     const float esum = warp_sum(e0 + e1);
     if (lane < N) gates_out[t * N + lane] = e0 / esum;
     if (lane + 32 < N) gates_out[t * N + lane + 32] = e1 / esum;
 }
-__device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
+static __device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
 {
     return warp_max(fmaxf(lane < N ? z0 : -INFINITY, lane + 32 < N ? z1 : -INFINITY));
 }
@@ -552,7 +552,7 @@ __device__ __noinline__ float logit_max(float z0, float z1, int N, int lane)
 // that is still computing (returns whether the data arrived; reports the timeout otherwise), or --
 // for a warp that has given up -- a short wait that lets copies already issued land, so that none
 // is in flight when the block exits.
-__device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volatile int *dead, bool alive, bool issued,
+static __device__ __noinline__ bool acquire_slow(uint64_t *bar, uint32_t parity, volatile int *dead, bool alive, bool issued,
                                           uint32_t *status, int lane, uint32_t polls)
 {
     if (alive) {

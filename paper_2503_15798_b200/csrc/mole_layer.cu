@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include "mole_decode.cuh"
+#include "mole_fstep.cuh"
 #include "mole_kernel.cuh"
 
 namespace mole {
@@ -71,6 +72,8 @@ static uint32_t wait_polls_from(const DebugEnv &e)
     if (e.wait_limit > 0) return e.wait_limit > 0x7fffffffLL ? 0x7fffffffu : static_cast<uint32_t>(e.wait_limit);
     return kWaitPolls;
 }
+
+uint32_t current_wait_polls() { return wait_polls_from(debug_env()); }
 
 // Lanes per 16-byte column group in the combine (1, 2 or 4).
 static int lanes_per_group(int dcc, int vec, const DebugEnv &env)
@@ -328,8 +331,88 @@ static DecodeVariant pick_decode(int N, bool norm)
     }
 }
 
+// The fused step with the decode arithmetic (mole_fstep.cuh): bf16, N of 4, 8, 16 or 32, d a multiple of
+// 128 with d / 4 <= 512 compute threads, router matrix in 1, 2 or 4 column chunks of at most 32 KB, rows in
+// chunks of whole experts of at most 32 KB.
+typedef void (*FStepKernel)(const FStepParams);
+struct FStepVariant {
+    FStepKernel fn;
+    const char *name;
+};
+struct FStepPlan {
+    int db, kw, kr, rexp, stages, blocks_per_sm, threads, smem;
+};
+static bool plan_fstep(long long M, int L, int N, int d, int dtype, bool norm, int sms, FStepPlan *f)
+{
+    if (dtype != MOLE_DTYPE_BF16 || d % 128 != 0 || d / 4 > kDecodeMaxThreads) return false;
+    if (N != 4 && N != 8 && N != 16 && N != 32) return false;
+    // the cut of an item into ring slots follows the width class (FStepCut): column chunks of the router
+    // matrix, chunks of whole experts' rows, neither above 32 KB
+    const int db = d <= 512 ? 0 : (d <= 1024 ? 1 : 2);
+    const int dmax = db == 0 ? 512 : (db == 1 ? 1024 : 2048);
+    int kw = N * dmax * 2 / static_cast<int>(kFStepSlotBytes);
+    if (kw < 1) kw = 1;
+    int rexp = static_cast<int>(kFStepSlotBytes) / (2 * dmax);
+    if (rexp > 16) rexp = 16;
+    if (rexp > N) rexp = N;
+    if (N / 2 / kw < 1 || rexp < 4) return false;
+    // blocks per SM aimed at: one per token while tokens are few (the deepest ring that fits), two or three
+    // token chains per SM when there are more tokens than SMs
+    int want = static_cast<int>((M + sms - 1) / sms);
+    want = want < 1 ? 1 : (want > 3 ? 3 : want);
+    const DebugEnv env = debug_env();
+    if (env.target_blocks > 0) want = env.target_blocks;
+    int stages = 0;
+    for (; want >= 1 && stages < 2; --want) {
+        const long long budget = kSmemPerSM / want - 1024;
+        stages = 0;
+        for (int s = kMaxStages; s >= 2; --s)
+            if (fstep_smem(N, d, s, norm ? 1 : 0).total <= budget && fstep_smem(N, d, s, norm ? 1 : 0).total <= static_cast<uint32_t>(kSmemPerBlockMax)) {
+                stages = s;
+                break;
+            }
+        if (stages >= 2) break;
+    }
+    if (stages < 2) return false;
+    if (env.stages >= 2 && env.stages <= kMaxStages && fstep_smem(N, d, env.stages, norm ? 1 : 0).total <= static_cast<uint32_t>(kSmemPerBlockMax))
+        stages = env.stages;
+    const long long chunks = ((M + static_cast<long long>(sms) * 3 - 1) / (static_cast<long long>(sms) * 3)) * L * (kw + N / rexp);
+    (void)chunks;
+    f->db = db;
+    f->kw = kw;
+    f->rexp = rexp;
+    f->kr = N / rexp;
+    f->stages = stages;
+    f->threads = d / 4 + 32;
+    f->smem = static_cast<int>(fstep_smem(N, d, stages, norm ? 1 : 0).total);
+    int per_sm = kSmemPerSM / (f->smem + 1024);
+    if (per_sm > 2048 / f->threads) per_sm = 2048 / f->threads;
+    f->blocks_per_sm = per_sm < 1 ? 1 : per_sm;
+    return true;
+}
+#define MOLE_FV(N, DB, NORM) FStepVariant { mole_fstep_kernel<N, DB, NORM>, "fstep<" #N "," #DB "," #NORM ">" }
+#define MOLE_FV_N(N)                                                          \
+    switch (db * 2 + (norm ? 1 : 0)) {                                        \
+        case 0: return MOLE_FV(N, 0, 0);                                      \
+        case 1: return MOLE_FV(N, 0, 1);                                      \
+        case 2: return MOLE_FV(N, 1, 0);                                      \
+        case 3: return MOLE_FV(N, 1, 1);                                      \
+        case 4: return MOLE_FV(N, 2, 0);                                      \
+        default: return MOLE_FV(N, 2, 1);                                     \
+    }
+static FStepVariant pick_fstep(int N, int db, bool norm)
+{
+    switch (N) {
+        case 4: MOLE_FV_N(4)
+        case 8: MOLE_FV_N(8)
+        case 16: MOLE_FV_N(16)
+        case 32: MOLE_FV_N(32)
+        default: return FStepVariant{nullptr, "none"};
+    }
+}
+
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
-static int ensure_smem(const void *fn, int smem)
+int ensure_smem_opt_in(const void *fn, int smem)
 {
     if (smem <= 48 * 1024) return MOLE_OK;
     struct Slot {
@@ -390,6 +473,9 @@ struct ShapeKey {
 };
 struct LaunchChoice {
     bool decode;        // the one-block-per-token kernel; otherwise the ring kernel with `plan`
+    bool fstep;         // the fused step with the decode arithmetic, with `fplan`
+    FStepPlan fplan;
+    FStepKernel fstep_fn;
     StepPlan plan;
     StepKernel step_fn;
     DecodeKernel decode_fn;
@@ -412,7 +498,34 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     int rc = plan_step(M, L, N, d, dtype, d_split, &plan, false, sms, norm);  // also validates the shape
     if (rc != MOLE_OK) return rc;
     const bool decode_ok = L == 1 && d_split == 0 && decode_shape_ok(dtype, N, d);
-    if (kernel == MOLE_KERNEL_DECODE && !decode_ok) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    c->decode = c->fstep = false;
+    FStepPlan fplan;
+    const bool fstep_ok = L > 1 && d_split == 0 && plan_fstep(M, L, N, d, dtype, norm, sms, &fplan);
+    if (kernel == MOLE_KERNEL_DECODE && !(decode_ok || fstep_ok)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    if (fstep_ok && kernel != MOLE_KERNEL_RING) {
+        const FStepVariant v = pick_fstep(N, fplan.db, norm);
+        if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        c->fstep = true;
+        c->fplan = fplan;
+        c->fstep_fn = v.fn;
+        c->plan = plan;
+        c->step_fn = nullptr;
+        c->decode_fn = nullptr;
+        c->name = v.name;
+        c->threads = fplan.threads;
+        c->smem = fplan.smem;
+        int per_sm = fplan.blocks_per_sm;
+        if (prepare) {
+            rc = ensure_smem_opt_in(reinterpret_cast<const void *>(v.fn), fplan.smem);
+            if (rc != MOLE_OK) return rc;
+            MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, v.fn, fplan.threads, fplan.smem));
+        }
+        if (per_sm < 1) per_sm = 1;
+        if (env.blocks_per_sm >= 1 && env.blocks_per_sm < per_sm) per_sm = env.blocks_per_sm;
+        c->grid = static_cast<long long>(per_sm) * sms;
+        if (c->grid > M) c->grid = M;
+        return MOLE_OK;
+    }
     if (decode_ok && (kernel == MOLE_KERNEL_DECODE || (kernel == MOLE_KERNEL_AUTO && M <= kDecodeKernelMaxTokens))) {
         const DecodeVariant v = pick_decode(N, norm);
         if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
@@ -424,7 +537,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
         c->threads = d / 4;
         c->smem = static_cast<int>(decode_smem_bytes(N, d));
         c->grid = M;
-        if (prepare) return ensure_smem(reinterpret_cast<const void *>(v.fn), c->smem);
+        if (prepare) return ensure_smem_opt_in(reinterpret_cast<const void *>(v.fn), c->smem);
         return MOLE_OK;
     }
     const bool direct = M >= 128 && M <= 4LL * sms;  // see pick_kernel
@@ -450,7 +563,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     c->smem = plan.smem;
     int per_sm = plan.blocks_per_sm;
     if (prepare) {
-        rc = ensure_smem(reinterpret_cast<const void *>(v.fn), plan.smem);
+        rc = ensure_smem_opt_in(reinterpret_cast<const void *>(v.fn), plan.smem);
         if (rc != MOLE_OK) return rc;
         // a persistent grid: as many blocks as fit at once, never more than the tokens
         MOLE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, v.fn, plan.threads, plan.smem));
@@ -520,6 +633,31 @@ int launch_step(const StepLaunch &a)
     cfg.attrs = attrs;
     cfg.numAttrs = na;
 
+    if (c->fstep) {
+        FStepParams p;
+        p.hidden = a.hidden;
+        p.row_index = a.row_index;
+        p.lut = a.lut;
+        p.w_router = a.w_router;
+        p.norm_weight = a.norm_weight;
+        p.out = a.out;
+        p.status = a.status;
+        p.lut_stride = a.lut_stride;
+        p.wr_stride = a.wr_stride;
+        p.norm_stride = a.norm_stride;
+        p.M = a.M;
+        p.rows = a.rows;
+        p.d = a.d;
+        p.L = a.L;
+        p.stages = c->fplan.stages;
+        p.kr = c->fplan.kr;
+        p.rexp = c->fplan.rexp;
+        p.norm_eps = a.norm_eps;
+        p.flags = a.flags;
+        p.wait_polls = c->wait_polls;
+        MOLE_CUDA_TRY(cudaLaunchKernelEx(&cfg, c->fstep_fn, p));
+        return MOLE_OK;
+    }
     if (c->decode) {
         DecodeParams p;
         p.hidden = a.hidden;
@@ -596,6 +734,7 @@ int mole_layer_forward_ex(const mole_args *a)
     if (!a || a->struct_size != sizeof(mole_args)) return MOLE_ERR_INVALID_ARG;
     if (a->flags & ~(MOLE_FLAG_IDS_INT64 | MOLE_FLAG_CHAIN)) return MOLE_ERR_INVALID_ARG;
     if (a->reserved2 != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->lut_format != MOLE_LUT_PLAIN && a->lut_format != MOLE_LUT_NF4 && a->lut_format != MOLE_LUT_NF3) return MOLE_ERR_INVALID_ARG;
     if (a->kernel != MOLE_KERNEL_AUTO && a->kernel != MOLE_KERNEL_RING && a->kernel != MOLE_KERNEL_DECODE) return MOLE_ERR_INVALID_ARG;
     if (a->norm_weight && (!aligned16(a->norm_weight) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f)) return MOLE_ERR_INVALID_ARG;
     int rc = check_common(a->hidden, a->ids, a->lut, a->w_router, a->out, a->residual, a->B, a->T, a->N, a->d, a->V,
@@ -627,6 +766,12 @@ int mole_layer_forward_ex(const mole_args *a)
     s.norm_weight = a->norm_weight;
     s.norm_eps = a->norm_eps;
     s.kernel = a->kernel;
+    if (a->lut_format != MOLE_LUT_PLAIN) {
+        // a quantised table: the one-block-per-token kernel that de-quantises inside the weighted sum
+        if (a->dtype != MOLE_DTYPE_BF16 || a->d_split != 0 || a->kernel == MOLE_KERNEL_RING) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        if (!quant_layer_shape_ok(a->N, a->d, a->lut_format, a->lut_block)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        return launch_quant_layer(s, a->lut_format, a->lut_block, current_wait_polls());
+    }
     return launch_step(s);
 }
 
@@ -655,6 +800,8 @@ int mole_decode_step_args(const mole_step_args *a)
 {
     if (!a || a->struct_size != sizeof(mole_step_args)) return MOLE_ERR_INVALID_ARG;
     if ((a->flags & ~MOLE_FLAG_CHAIN) || a->reserved != 0) return MOLE_ERR_INVALID_ARG;
+    if (a->lut_format != MOLE_LUT_PLAIN && a->lut_format != MOLE_LUT_NF4 && a->lut_format != MOLE_LUT_NF3) return MOLE_ERR_INVALID_ARG;
+    const bool quant = a->lut_format != MOLE_LUT_PLAIN;
     const int L = a->L;
     int mode = a->mode;
     if (L < 1 || mode < MOLE_STEP_AUTO || mode > MOLE_STEP_CHAINED) return MOLE_ERR_INVALID_ARG;
@@ -668,7 +815,14 @@ int mole_decode_step_args(const mole_step_args *a)
     if (a->norm_weight_base &&
         (!aligned16(a->norm_weight_base) || (a->norm_layer_stride_bytes & 15) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f))
         return MOLE_ERR_INVALID_ARG;
-    if (mode == MOLE_STEP_AUTO) mode = (L > 1 && M > kFusedMaxTokens) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
+    if (mode == MOLE_STEP_AUTO) mode = (quant || (L > 1 && M > kFusedMaxTokens)) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
+    if (quant) {
+        // quantised tables run layer by layer (one block per token de-quantising inside the weighted sum)
+        if (mode == MOLE_STEP_FUSED && L > 1) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        mode = MOLE_STEP_CHAINED;
+        if (a->dtype != MOLE_DTYPE_BF16 || a->d_split != 0 || a->kernel == MOLE_KERNEL_RING) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        if (!quant_layer_shape_ok(a->N, a->d, a->lut_format, a->lut_block)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    }
 
     StepLaunch s;
     s.residual = nullptr;
@@ -696,7 +850,6 @@ int mole_decode_step_args(const mole_step_args *a)
         s.out = a->out;
         s.L = L;
         s.flags = a->flags & MOLE_FLAG_CHAIN;
-        if (L > 1 && s.kernel == MOLE_KERNEL_DECODE) return MOLE_ERR_UNSUPPORTED_SHAPE;
         return launch_step(s);
     }
     if (L > 1 && (!a->tmp || !aligned16(a->tmp) || a->out == a->hidden_in || a->tmp == a->hidden_in || a->tmp == a->out))
@@ -717,7 +870,7 @@ int mole_decode_step_args(const mole_step_args *a)
         s.out = dst;
         s.L = 1;
         s.flags = l > 0 ? MOLE_FLAG_CHAIN : (a->flags & MOLE_FLAG_CHAIN);
-        rc = launch_step(s);
+        rc = quant ? launch_quant_layer(s, a->lut_format, a->lut_block, current_wait_polls()) : launch_step(s);
         if (rc != MOLE_OK) return rc;
         src = dst;
     }
@@ -819,10 +972,20 @@ int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_spl
     return MOLE_OK;
 }
 
-int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, char *name, int name_bytes, int *out_threads,
-                 int *out_smem_bytes)
+int mole_variant(int M, int L, int N, int d, int dtype, int d_split, int norm, int kernel, int lut_format, int lut_block, char *name,
+                 int name_bytes, int *out_threads, int *out_smem_bytes)
 {
     if (M < 1 || !name || name_bytes < 1) return MOLE_ERR_INVALID_ARG;
+    if (lut_format != MOLE_LUT_PLAIN) {
+        if (lut_format != MOLE_LUT_NF4 && lut_format != MOLE_LUT_NF3) return MOLE_ERR_INVALID_ARG;
+        if (L != 1 || dtype != MOLE_DTYPE_BF16 || d_split != 0 || kernel == MOLE_KERNEL_RING ||
+            !quant_layer_shape_ok(N, d, lut_format, lut_block))
+            return MOLE_ERR_UNSUPPORTED_SHAPE;
+        snprintf(name, static_cast<size_t>(name_bytes), "%s", quant_variant_name(N, lut_format, norm != 0));
+        if (out_threads) *out_threads = d / 4;
+        if (out_smem_bytes) *out_smem_bytes = 0;
+        return MOLE_OK;
+    }
     LaunchChoice c;
     int rc = choose_launch(M, L, N, d, dtype, d_split, norm != 0, kernel, sms_or_nominal(), false, &c);
     if (rc != MOLE_OK) return rc;
@@ -848,6 +1011,7 @@ const char *mole_status_string(int code)
         case MOLE_ERR_CUDA: return "CUDA runtime error";
         case MOLE_ERR_NOMEM: return "out of memory";
         case MOLE_ERR_TOO_LARGE: return "size beyond the stated maximum";
+        case MOLE_ERR_IO: return "table file error";
         default: return "unknown status";
     }
 }

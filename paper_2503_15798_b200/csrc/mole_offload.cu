@@ -97,18 +97,36 @@ __global__ void __launch_bounds__(kDedupThreads) mole_dedup_kernel(const int32_t
 // of the row, blockIdx.z = z, one of several layers' tables (table_stride bytes apart on the host,
 // staging_stride bytes apart in the staging area) fetched for the same ids in one launch.  All of
 // a thread's loads are issued before its first store so that many reads are in flight on the host link.
+// Hot rows: ids with hot_slot[id] >= 0 have their rows of every layer cached in device memory
+// (hot_base[(hot_layer0 + z) * hot_rows + hot_slot[id]]); those are copied from there and never touch
+// the host link.
+struct HotRows {
+    const int32_t *slot;        // [V] position in the cache or -1; NULL: no cache
+    const unsigned char *base;  // [layers][rows][row_bytes]
+    long long rows;
+    int layer0;                 // cache layer of this launch's z = 0
+    unsigned long long *hits;   // rows served from the cache (one count per row and layer), or NULL
+};
 __global__ void __launch_bounds__(kFetchThreads) mole_fetch_kernel(const unsigned char *__restrict__ table_host,
                                                                    const int32_t *__restrict__ uniq,
                                                                    const int32_t *__restrict__ count, long long row_bytes,
                                                                    unsigned char *__restrict__ staging, long long table_stride,
-                                                                   long long staging_stride)
+                                                                   long long staging_stride, const HotRows hot)
 {
     const int u = blockIdx.y;
     if (u >= *count) return;
     const long long row = uniq[u];
     const long long chunk0 = static_cast<long long>(blockIdx.x) * kFetchChunk;
     const long long z = blockIdx.z;
-    const uint4 *src = reinterpret_cast<const uint4 *>(table_host + z * table_stride + row * row_bytes + chunk0);
+    const unsigned char *from = table_host + z * table_stride + row * row_bytes;
+    if (hot.slot) {
+        const int hs = hot.slot[row];
+        if (hs >= 0) {
+            from = hot.base + ((hot.layer0 + z) * hot.rows + hs) * row_bytes;
+            if (hot.hits && blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(hot.hits, 1ull);
+        }
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(from + chunk0);
     uint4 *dst = reinterpret_cast<uint4 *>(staging + z * staging_stride + static_cast<long long>(u) * row_bytes + chunk0);
     const long long nvec = min(static_cast<long long>(kFetchChunk), row_bytes - chunk0) / 16;
     uint4 v[kFetchVecPerThread];
@@ -132,17 +150,43 @@ static int launch_dedup(const int32_t *ids, int M, int V, int32_t *scratch, int3
     return MOLE_OK;
 }
 
+// Device alias of a pinned host allocation; the last answer is remembered per thread (a decoding loop asks
+// for the same table again and again).
+static int device_alias(const void *host, const unsigned char **out)
+{
+    thread_local const void *last_host = nullptr;
+    thread_local const unsigned char *last_dev = nullptr;
+    thread_local int last_device = -1;
+    int dev = 0;
+    MOLE_CUDA_TRY(cudaGetDevice(&dev));
+    if (host == last_host && dev == last_device && last_dev) {
+        *out = last_dev;
+        return MOLE_OK;
+    }
+    void *alias = nullptr;
+    MOLE_CUDA_TRY(cudaHostGetDevicePointer(&alias, const_cast<void *>(host), 0));
+    last_host = host;
+    last_dev = static_cast<const unsigned char *>(alias);
+    last_device = dev;
+    *out = last_dev;
+    return MOLE_OK;
+}
+
 // `layers` tables, table_stride bytes apart from lut_host on (one pinned allocation), into staging areas
 // staging_stride bytes apart
 static int launch_fetch(const void *lut_host, const int32_t *uniq, const int32_t *count, int max_rows, long long row_bytes,
-                        void *staging, cudaStream_t st, int layers = 1, long long table_stride = 0, long long staging_stride = 0)
+                        void *staging, cudaStream_t st, int layers = 1, long long table_stride = 0, long long staging_stride = 0,
+                        const HotRows *hot = nullptr)
 {
-    void *dev_alias = nullptr;
-    MOLE_CUDA_TRY(cudaHostGetDevicePointer(&dev_alias, const_cast<void *>(lut_host), 0));
+    const unsigned char *dev_alias = nullptr;
+    int rc = device_alias(lut_host, &dev_alias);
+    if (rc != MOLE_OK) return rc;
     dim3 grid(static_cast<unsigned>((row_bytes + kFetchChunk - 1) / kFetchChunk), static_cast<unsigned>(max_rows),
               static_cast<unsigned>(layers));
-    mole_fetch_kernel<<<grid, kFetchThreads, 0, st>>>(static_cast<const unsigned char *>(dev_alias), uniq, count, row_bytes,
-                                                      static_cast<unsigned char *>(staging), table_stride, staging_stride);
+    HotRows none;
+    memset(&none, 0, sizeof none);
+    mole_fetch_kernel<<<grid, kFetchThreads, 0, st>>>(dev_alias, uniq, count, row_bytes, static_cast<unsigned char *>(staging),
+                                                      table_stride, staging_stride, hot ? *hot : none);
     MOLE_CUDA_TRY(cudaGetLastError());
     return MOLE_OK;
 }
@@ -153,8 +197,17 @@ using namespace mole;
 
 struct mole_offload_ctx {
     int max_tokens, N, d, V, dtype, n_buffers;
+    int lut_format, lut_block;  // MOLE_LUT_*: rows are plain elements, or the packed records of a quantised table
     long long row_bytes;
     int32_t *table;  // [V] dedup scratch, kept all zero between kernels
+    // hot rows: the rows of hot_rows ids of hot_layers layers kept in device memory
+    int32_t *hot_slot;        // [V]: position in the cache or -1
+    unsigned char *hot_base;  // [hot_layers][hot_rows][row_bytes]
+    long long hot_rows;
+    int hot_layers;
+    const unsigned char *hot_host_base;  // the host tables the cache mirrors: layer l at + l * hot_host_stride
+    long long hot_host_stride;
+    unsigned long long *hot_hits;  // device counter
     cudaEvent_t step_begin;  // orders the side stream after the main stream at the start of a whole step
     struct Buffer {
         unsigned char *staging;  // [max_tokens][N][d]
@@ -221,6 +274,9 @@ int mole_offload_destroy(mole_offload_ctx *c)
         delete[] c->buf;
     }
     if (c->table) cudaFree(c->table);
+    if (c->hot_slot) cudaFree(c->hot_slot);
+    if (c->hot_base) cudaFree(c->hot_base);
+    if (c->hot_hits) cudaFree(c->hot_hits);
     if (c->step_begin) cudaEventDestroy(c->step_begin);
     delete c;
     (void)cudaGetLastError();
@@ -229,15 +285,28 @@ int mole_offload_destroy(mole_offload_ctx *c)
 
 int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, int V, int dtype, int n_buffers)
 {
+    return mole_offload_create_ex(out, max_tokens, N, d, V, dtype, n_buffers, MOLE_LUT_PLAIN, 0);
+}
+
+int mole_offload_create_ex(mole_offload_ctx **out, int max_tokens, int N, int d, int V, int dtype, int n_buffers, int lut_format,
+                           int lut_block)
+{
     if (!out) return MOLE_ERR_INVALID_ARG;
     *out = nullptr;
     if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
+    if (lut_format != MOLE_LUT_PLAIN && lut_format != MOLE_LUT_NF4 && lut_format != MOLE_LUT_NF3) return MOLE_ERR_INVALID_ARG;
     if (max_tokens < 1 || n_buffers < 1 || n_buffers > 16) return MOLE_ERR_INVALID_ARG;
     if (max_tokens > 65535) return MOLE_ERR_TOO_LARGE;
     StepPlan plan;
     int rc = plan_step(max_tokens, 1, N, d, dtype, 0, &plan);
     if (rc != MOLE_OK) return rc;
     if (V < 1) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    int64_t rec_bytes = 0;
+    if (lut_format != MOLE_LUT_PLAIN) {
+        if (dtype != MOLE_DTYPE_BF16 || !quant_layer_shape_ok(N, d, lut_format, lut_block)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        rc = mole_quant_record_bytes(N, d, lut_format, lut_block, &rec_bytes);
+        if (rc != MOLE_OK) return rc;
+    }
     mole_offload_ctx *c = new (std::nothrow) mole_offload_ctx;
     if (!c) return MOLE_ERR_NOMEM;
     memset(c, 0, sizeof *c);
@@ -247,7 +316,9 @@ int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, in
     c->V = V;
     c->dtype = dtype;
     c->n_buffers = n_buffers;
-    c->row_bytes = static_cast<long long>(N) * d * elem_bytes(dtype);
+    c->lut_format = lut_format;
+    c->lut_block = lut_block;
+    c->row_bytes = lut_format != MOLE_LUT_PLAIN ? rec_bytes : static_cast<long long>(N) * d * elem_bytes(dtype);
     c->buf = new (std::nothrow) mole_offload_ctx::Buffer[n_buffers];
     if (!c->buf) {
         delete c;
@@ -276,6 +347,99 @@ int mole_offload_create(mole_offload_ctx **out, int max_tokens, int N, int d, in
     return MOLE_OK;
 }
 
+// The cache as the fetch kernel sees it for tables starting at `lut_host` (layer 0 of the launch): only if
+// that address is one of the mirrored host tables.
+static bool hot_for(const mole_offload_ctx *c, const void *lut_host, long long table_stride, int layers, HotRows *h)
+{
+    if (!c->hot_slot || !c->hot_base || c->hot_rows == 0) return false;
+    const long long off = static_cast<const unsigned char *>(lut_host) - c->hot_host_base;
+    if (off < 0) return false;
+    long long layer0 = 0;
+    if (c->hot_layers > 1) {
+        if (c->hot_host_stride <= 0 || off % c->hot_host_stride != 0) return false;
+        layer0 = off / c->hot_host_stride;
+        if (layers > 1 && table_stride != c->hot_host_stride) return false;
+    } else if (off != 0) {
+        return false;
+    }
+    if (layer0 + layers > c->hot_layers) return false;
+    h->slot = c->hot_slot;
+    h->base = c->hot_base;
+    h->rows = c->hot_rows;
+    h->layer0 = static_cast<int>(layer0);
+    h->hits = c->hot_hits;
+    return true;
+}
+
+int mole_offload_set_hot_rows(mole_offload_ctx *c, const int32_t *hot_ids_host, int n_hot, const void *lut_host_base,
+                              int64_t lut_layer_stride_bytes, int L)
+{
+    if (!c || n_hot < 0 || L < 1) return MOLE_ERR_INVALID_ARG;
+    MOLE_CUDA_TRY(cudaDeviceSynchronize());  // nothing of this context may be in flight while the cache changes
+    if (c->hot_slot) cudaFree(c->hot_slot);
+    if (c->hot_base) cudaFree(c->hot_base);
+    if (c->hot_hits) cudaFree(c->hot_hits);
+    c->hot_slot = nullptr;
+    c->hot_base = nullptr;
+    c->hot_hits = nullptr;
+    c->hot_rows = 0;
+    c->hot_layers = 0;
+    if (n_hot == 0) return MOLE_OK;
+    if (!hot_ids_host || !lut_host_base || !aligned16(lut_host_base) || (lut_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    if (n_hot > c->V) return MOLE_ERR_TOO_LARGE;
+    int32_t *slot_host = new (std::nothrow) int32_t[c->V];
+    if (!slot_host) return MOLE_ERR_NOMEM;
+    for (int i = 0; i < c->V; ++i) slot_host[i] = -1;
+    for (int i = 0; i < n_hot; ++i) {
+        const int id = hot_ids_host[i];
+        if (id < 0 || id >= c->V || slot_host[id] != -1) {  // outside the table, or listed twice
+            delete[] slot_host;
+            return MOLE_ERR_INVALID_ARG;
+        }
+        slot_host[id] = i;
+    }
+    cudaError_t e = cudaMalloc(&c->hot_slot, sizeof(int32_t) * static_cast<size_t>(c->V));
+    if (e == cudaSuccess) e = cudaMalloc(&c->hot_base, static_cast<size_t>(L) * n_hot * c->row_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&c->hot_hits, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(c->hot_hits, 0, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemcpy(c->hot_slot, slot_host, sizeof(int32_t) * static_cast<size_t>(c->V), cudaMemcpyHostToDevice);
+    for (int l = 0; l < L && e == cudaSuccess; ++l)
+        for (int i = 0; i < n_hot && e == cudaSuccess; ++i)
+            e = cudaMemcpyAsync(c->hot_base + (static_cast<size_t>(l) * n_hot + i) * c->row_bytes,
+                                static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l) * lut_layer_stride_bytes +
+                                    static_cast<int64_t>(hot_ids_host[i]) * c->row_bytes,
+                                static_cast<size_t>(c->row_bytes), cudaMemcpyHostToDevice, nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    delete[] slot_host;
+    if (e != cudaSuccess) {
+        set_cuda_error(e);
+        if (c->hot_slot) cudaFree(c->hot_slot);
+        if (c->hot_base) cudaFree(c->hot_base);
+        if (c->hot_hits) cudaFree(c->hot_hits);
+        c->hot_slot = nullptr;
+        c->hot_base = nullptr;
+        c->hot_hits = nullptr;
+        return e == cudaErrorMemoryAllocation ? MOLE_ERR_NOMEM : MOLE_ERR_CUDA;
+    }
+    c->hot_rows = n_hot;
+    c->hot_layers = L;
+    c->hot_host_base = static_cast<const unsigned char *>(lut_host_base);
+    c->hot_host_stride = lut_layer_stride_bytes;
+    return MOLE_OK;
+}
+
+int mole_offload_hot_hits(mole_offload_ctx *c, uint64_t *hits, int reset)
+{
+    if (!c || !hits) return MOLE_ERR_INVALID_ARG;
+    *hits = 0;
+    if (!c->hot_hits) return MOLE_OK;
+    unsigned long long v = 0;
+    MOLE_CUDA_TRY(cudaMemcpy(&v, c->hot_hits, sizeof v, cudaMemcpyDeviceToHost));  // waits for the device's work queued so far
+    *hits = v;
+    if (reset) MOLE_CUDA_TRY(cudaMemset(c->hot_hits, 0, sizeof v));
+    return MOLE_OK;
+}
+
 int mole_offload_prefetch(mole_offload_ctx *c, int b, const int32_t *ids, int M, const void *lut_host_layer,
                           void *side_stream)
 {
@@ -290,7 +454,9 @@ int mole_offload_prefetch(mole_offload_ctx *c, int b, const int32_t *ids, int M,
     MOLE_CUDA_TRY(cudaStreamWaitEvent(st, B.consumed, 0));
     int rc = launch_dedup(ids, M, c->V, c->table, B.uniq, B.slot, B.count, nullptr, st);
     if (rc != MOLE_OK) return rc;
-    rc = launch_fetch(lut_host_layer, B.uniq, B.count, M, c->row_bytes, B.staging, st);
+    HotRows hot;
+    const bool use_hot = hot_for(c, lut_host_layer, 0, 1, &hot);
+    rc = launch_fetch(lut_host_layer, B.uniq, B.count, M, c->row_bytes, B.staging, st, 1, 0, 0, use_hot ? &hot : nullptr);
     if (rc != MOLE_OK) return rc;
     MOLE_CUDA_TRY(cudaEventRecord(B.ready, st));
     return MOLE_OK;
@@ -328,7 +494,7 @@ int mole_layer_forward_offload(mole_offload_ctx *c, int b, const void *hidden, c
     a.flags = 0;
     a.d_split = 0;
     a.stream = st;
-    int rc = launch_step(a);
+    int rc = c->lut_format != MOLE_LUT_PLAIN ? launch_quant_layer(a, c->lut_format, c->lut_block, current_wait_polls()) : launch_step(a);
     if (rc != MOLE_OK) return rc;
     MOLE_CUDA_TRY(cudaEventRecord(B.consumed, st));
     return MOLE_OK;
@@ -384,9 +550,11 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
         mole_offload_ctx::Buffer &Bk = c->buf[k & 1];
         const int l0 = k * g, n = (l0 + g <= L) ? g : L - l0;
         if (k >= 2) MOLE_CUDA_TRY(cudaStreamWaitEvent(side, Bk.consumed, 0));
-        int r = launch_fetch(static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l0) * lut_layer_stride_bytes,
-                             B0.uniq, B0.count, static_cast<int>(M), c->row_bytes, Bk.staging, side, n, lut_layer_stride_bytes,
-                             area);
+        const unsigned char *tables = static_cast<const unsigned char *>(lut_host_base) + static_cast<int64_t>(l0) * lut_layer_stride_bytes;
+        HotRows hot;
+        const bool use_hot = hot_for(c, tables, lut_layer_stride_bytes, n, &hot);
+        int r = launch_fetch(tables, B0.uniq, B0.count, static_cast<int>(M), c->row_bytes, Bk.staging, side, n, lut_layer_stride_bytes,
+                             area, use_hot ? &hot : nullptr);
         if (r != MOLE_OK) return r;
         MOLE_CUDA_TRY(cudaEventRecord(Bk.ready, side));
         return MOLE_OK;
@@ -398,33 +566,52 @@ int mole_offload_decode_step(mole_offload_ctx *c, const void *hidden_in, const i
         mole_offload_ctx::Buffer &Bk = c->buf[k & 1];
         MOLE_CUDA_TRY(cudaStreamWaitEvent(st, Bk.ready, 0));
         const int l0 = k * g, n = (l0 + g <= L) ? g : L - l0;
-        // the group's layers in ONE launch: their rows lie `area` bytes apart in the staging area, which is
-        // all the fused step kernel needs (a token's chain through the n layers stays on chip)
-        void *dst = (groups - 1 - k) % 2 == 0 ? out : tmp;
         StepLaunch a;
-        a.hidden = src;
         a.residual = nullptr;
         a.row_index = B0.slot;  // gather from staging[slot[t]]; slot is -1 for an id outside [0, V)
-        a.lut = Bk.staging;
-        a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l0) * wr_layer_stride_bytes;
-        a.out = dst;
         a.gates_out = nullptr;
         a.status = status;
         a.lut_stride = area;
         a.wr_stride = wr_layer_stride_bytes;
         a.M = M;
-        a.L = n;
         a.N = c->N;
         a.d = c->d;
         a.rows = M;  // a slot never exceeds the number of distinct ids
         a.dtype = c->dtype;
-        a.flags = 0;
         a.d_split = 0;
-        a.kernel = MOLE_KERNEL_RING;  // every group on one kernel family: the step's bits do not depend on how it is grouped
         a.stream = st;
-        rc = launch_step(a);
-        if (rc != MOLE_OK) return rc;
-        src = dst;
+        if (c->lut_format != MOLE_LUT_PLAIN) {
+            // quantised records: layer by layer from the staging area (the layers of a group chained to one
+            // another with programmatic dependent launch), ping-pong so that the last layer writes `out`
+            for (int i = 0; i < n; ++i) {
+                const int l = l0 + i;
+                void *dst = ((L - 1 - l) % 2 == 0) ? out : tmp;
+                a.hidden = src;
+                a.lut = Bk.staging + static_cast<long long>(i) * area;
+                a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l) * wr_layer_stride_bytes;
+                a.out = dst;
+                a.L = 1;
+                a.flags = i > 0 ? MOLE_FLAG_CHAIN : 0;
+                rc = launch_quant_layer(a, c->lut_format, c->lut_block, current_wait_polls());
+                if (rc != MOLE_OK) return rc;
+                src = dst;
+            }
+        } else {
+            // the group's layers in ONE launch: their rows lie `area` bytes apart in the staging area, which is
+            // all the fused step kernel needs (a token's chain through the n layers stays on chip).  The last
+            // group writes `out`, the groups before it alternate between tmp and out.
+            void *dst = (groups - 1 - k) % 2 == 0 ? out : tmp;
+            a.hidden = src;
+            a.lut = Bk.staging;
+            a.w_router = static_cast<const unsigned char *>(w_router_base) + static_cast<int64_t>(l0) * wr_layer_stride_bytes;
+            a.out = dst;
+            a.L = n;
+            a.flags = 0;
+            a.kernel = MOLE_KERNEL_RING;  // every group on one kernel family: the step's bits do not depend on how it is grouped
+            rc = launch_step(a);
+            if (rc != MOLE_OK) return rc;
+            src = dst;
+        }
         MOLE_CUDA_TRY(cudaEventRecord(Bk.consumed, st));
     }
     return MOLE_OK;

@@ -91,6 +91,14 @@ def zipf_ids(M: int, V: int, s: float = 1.1, seed: int = 0, permute: bool = True
     return ranks.astype(np.int32)
 
 
+def zipf_hot_ids(V: int, K: int, permute: bool = True) -> np.ndarray:
+    """The ids of the K most probable ranks of zipf_ids' distribution (what a cache of hot rows holds)."""
+    K = min(K, V)
+    if permute:
+        return np.random.default_rng(0x5EED + V).permutation(V)[:K].astype(np.int32)
+    return np.arange(K, dtype=np.int32)
+
+
 def uniform_ids(M: int, V: int, seed: int = 0) -> np.ndarray:
     return np.random.default_rng(seed).integers(0, V, size=M, dtype=np.int64).astype(np.int32)
 

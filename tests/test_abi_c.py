@@ -29,7 +29,8 @@ int main(void)
     FIELD(mole_args, lut); FIELD(mole_args, w_router); FIELD(mole_args, out); FIELD(mole_args, residual);
     FIELD(mole_args, gates_out); FIELD(mole_args, status); FIELD(mole_args, B); FIELD(mole_args, T); FIELD(mole_args, N);
     FIELD(mole_args, d); FIELD(mole_args, V); FIELD(mole_args, dtype); FIELD(mole_args, kernel); FIELD(mole_args, d_split);
-    FIELD(mole_args, stream); FIELD(mole_args, norm_weight); FIELD(mole_args, norm_eps); FIELD(mole_args, reserved2);
+    FIELD(mole_args, stream); FIELD(mole_args, norm_weight); FIELD(mole_args, norm_eps); FIELD(mole_args, lut_format);
+    FIELD(mole_args, lut_block); FIELD(mole_args, reserved2);
     printf("sizeof.mole_step_args %zu\n", sizeof(mole_step_args));
     FIELD(mole_step_args, struct_size); FIELD(mole_step_args, flags); FIELD(mole_step_args, hidden_in); FIELD(mole_step_args, ids);
     FIELD(mole_step_args, lut_base); FIELD(mole_step_args, lut_layer_stride_bytes); FIELD(mole_step_args, w_router_base);
@@ -38,6 +39,7 @@ int main(void)
     FIELD(mole_step_args, status); FIELD(mole_step_args, L); FIELD(mole_step_args, B); FIELD(mole_step_args, T);
     FIELD(mole_step_args, N); FIELD(mole_step_args, d); FIELD(mole_step_args, V); FIELD(mole_step_args, dtype);
     FIELD(mole_step_args, mode); FIELD(mole_step_args, d_split); FIELD(mole_step_args, kernel); FIELD(mole_step_args, norm_eps);
+    FIELD(mole_step_args, lut_format); FIELD(mole_step_args, lut_block);
     FIELD(mole_step_args, reserved); FIELD(mole_step_args, stream);
     return 0;
 }

@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert lib.mole_version() == 300
-    seen = {lib.mole_status_string(c).decode() for c in range(6)}
-    assert len(seen) == 6 and "ok" in seen
+    seen = {lib.mole_status_string(c).decode() for c in range(7)}
+    assert len(seen) == 7 and "ok" in seen
     assert lib.mole_status_string(99).decode() == "unknown status"
 
 
@@ -47,10 +47,11 @@ def test_variant_names_and_kernel_choice(lib):
     # beyond 2048 tokens, with an explicit chunk count, for several layers, or on request: the ring kernel
     assert V(16384, 16, 1024)[0] == "step<bf16,16,1,2,2,0,0>"
     assert V(256, 16, 768, d_split=1)[0] == "step<bf16,16,1,2,1,1,0>"
-    assert V(256, 16, 768, L=12)[0] == "step<bf16,16,1,1,1,0,0>"
+    assert V(256, 16, 768, L=12)[0] == "fstep<16,1,0>" and V(256, 16, 768, L=12, kernel=binding.KERNEL_RING)[0] == "step<bf16,16,1,1,1,0,0>"
     assert V(256, 16, 768, kernel=binding.KERNEL_RING)[0] == "step<bf16,16,1,2,1,1,0>"
     # the 1B width (512 column groups of 8 bytes, N = 32) is outside the decode kernel: ring kernel, rows cut by experts
-    assert V(256, 32, 2048)[0] == "step<bf16,32,2,3,3,0,0>" and V(64, 32, 2048, L=16)[0] == "step<bf16,32,2,3,4,0,0>"
+    assert V(256, 32, 2048)[0] == "step<bf16,32,2,3,3,0,0>" and V(64, 32, 2048, L=16)[0] == "fstep<32,2,0>"
+    assert V(64, 32, 2048, L=16, kernel=binding.KERNEL_RING)[0] == "step<bf16,32,2,3,4,0,0>"
     with pytest.raises(binding.MoleError) as e:
         V(256, 32, 2048, kernel=binding.KERNEL_DECODE)
     assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE

@@ -318,3 +318,84 @@ def test_offload_decode_step_at_the_benchmarked_shape(M):
     finally:
         ctx.destroy()
         host.free()
+
+
+@pytest.mark.parametrize("M,cap", [(48, 64), (5, 64), (64, 64)])
+def test_hot_rows_cache_serves_the_listed_ids_and_changes_no_bit(M, cap):
+    """A cache of hot rows in device memory in front of the host link: ids on the list are served from it
+    (shown by overwriting their rows in the host table after they were cached -- the output must not notice),
+    the hit counter counts exactly the (distinct id, layer) pairs on the list, and dropping the cache goes
+    back to the host rows."""
+    N, d, V, L = 16, 1024, 700, 4
+    g = torch.Generator().manual_seed(9)
+    host = mole.HostTable((L, V, N, d), torch.bfloat16)
+    ctx = mole.OffloadContext(max_tokens=cap, N=N, d=d, V=V, n_buffers=2)
+    side = torch.cuda.Stream()
+    try:
+        host.tensor.copy_(torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16))
+        wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
+        hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
+        ids_np = inputs.zipf_ids(M, V, seed=3)
+        ids = torch.from_numpy(ids_np).to(DEV)
+        out, tmp = torch.empty_like(hidden), torch.empty_like(hidden)
+        want = ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, side_stream=side).clone()
+        torch.cuda.synchronize()
+        hot = inputs.zipf_hot_ids(V, 40)
+        assert len(set(hot.tolist()) & set(ids_np.tolist())) >= 1
+        ctx.set_hot_rows(hot, host.tensor)
+        assert ctx.hot_hits(reset=True) == 0
+        keep = host.tensor[:, torch.from_numpy(hot).long()].clone()
+        host.tensor[:, torch.from_numpy(hot).long()] = 7.0   # the host copies of the cached rows are never read again
+        got = ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, side_stream=side)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+        assert ctx.hot_hits() == len(set(hot.tolist()) & set(ids_np.tolist())) * L
+        # the single-layer path finds the cache through the layer's host address
+        one = torch.empty_like(hidden)
+        ctx.prefetch(0, ids, host.tensor[2], side_stream=side)
+        ctx.forward(0, hidden, wrs[2], one)
+        torch.cuda.synchronize()
+        host.tensor[:, torch.from_numpy(hot).long()] = keep
+        plain = torch.empty_like(hidden)
+        ctx.set_hot_rows([], host.tensor)
+        ctx.prefetch(0, ids, host.tensor[2], side_stream=side)
+        ctx.forward(0, hidden, wrs[2], plain)
+        assert torch.equal(ctx.decode_step(hidden, ids, host.tensor, wrs, out, tmp, side_stream=side), want)
+        torch.cuda.synchronize()
+        assert torch.equal(one, plain)
+        with pytest.raises(mole.MoleError):  # an id listed twice
+            ctx.set_hot_rows([1, 2, 1], host.tensor)
+        with pytest.raises(mole.MoleError):
+            ctx.set_hot_rows([V], host.tensor)
+    finally:
+        ctx.destroy()
+        host.free()
+
+
+def test_tables_from_a_file_feed_the_offload_mode(tmp_path):
+    """Disk -> pinned host memory -> offload step: tables written to a table file, read back into a pinned
+    host allocation, served by the offload step; equal to the step over the tables they were written from."""
+    N, d, V, L, M = 16, 768, 300, 3, 20
+    g = torch.Generator().manual_seed(4)
+    tables = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16)
+    path = str(tmp_path / "tables.mole")
+    mole.table_file_write(path, tables, N, d)
+    host = mole.HostTable((L, V, N, d), torch.bfloat16)
+    ctx = mole.OffloadContext(max_tokens=32, N=N, d=d, V=V, n_buffers=2)
+    side = torch.cuda.Stream()
+    try:
+        mole.table_file_read(path, host.tensor)
+        assert torch.equal(host.tensor.view(torch.int16), tables.view(torch.int16))
+        wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
+        hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
+        ids = torch.from_numpy(inputs.zipf_ids(M, V, seed=1)).to(DEV)
+        out = ctx.decode_step(hidden, ids, host.tensor, wrs, torch.empty_like(hidden), torch.empty_like(hidden), side_stream=side)
+        h = hidden
+        dev_tables = tables.to(DEV)
+        for l in range(L):
+            h = mole.layer_forward(h, ids, dev_tables[l], wrs[l], kernel=mole.KERNEL_RING)
+        torch.cuda.synchronize()
+        assert torch.equal(out, h)
+    finally:
+        ctx.destroy()
+        host.free()

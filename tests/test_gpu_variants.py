@@ -34,24 +34,39 @@ CASES = {
     "step<bf16,16,1,2,1,0,1>": [(700, 16, 768, 1, True, RING)],
     "step<bf16,16,1,2,2,1,1>": [(256, 16, 1024, 1, True, RING)],
     "step<bf16,16,1,2,2,0,1>": [(2500, 16, 1024, 1, True, AUTO)],
-    "step<bf16,32,2,3,3,0,0>": [(256, 32, 2048, 1, False, AUTO), (256, 32, 2048, 3, False, AUTO)],
-    "step<bf16,32,2,3,4,0,0>": [(64, 32, 2048, 1, False, AUTO), (64, 32, 2048, 3, False, AUTO), (148, 32, 2048, 2, False, AUTO)],
     "step<bf16,32,2,3,3,0,1>": [(256, 32, 2048, 1, True, AUTO)],
-    "step<bf16,32,1,0,0,0,1>": [(16, 32, 2048, 1, True, AUTO), (16, 32, 2048, 2, True, AUTO)],
-    "step<bf16,32,2,0,0,0,1>": [(256, 32, 2048, 2, True, AUTO)],
-    # fused steps
-    "step<bf16,16,1,1,1,0,0>": [(256, 16, 768, 3, False, AUTO), (64, 16, 768, 12, False, AUTO)],
-    "step<bf16,16,1,1,2,0,0>": [(256, 16, 1024, 3, False, AUTO), (64, 16, 1024, 4, False, AUTO), (8, 16, 1024, 8, False, AUTO)],
-    "step<bf16,16,1,0,0,0,1>": [(256, 16, 768, 3, True, AUTO), (64, 16, 1024, 2, True, AUTO)],
+    # fused steps: the decode arithmetic with a ring (default) ...
+    "fstep<16,1,0>": [(256, 16, 768, 3, False, AUTO), (64, 16, 768, 12, False, AUTO), (256, 16, 1024, 3, False, AUTO),
+                      (8, 16, 1024, 8, False, AUTO), (1, 16, 768, 12, False, AUTO), (700, 16, 768, 2, False, AUTO)],
+    "fstep<16,1,1>": [(256, 16, 768, 3, True, AUTO), (64, 16, 1024, 2, True, AUTO)],
+    "fstep<32,2,0>": [(256, 32, 2048, 3, False, AUTO), (64, 32, 2048, 3, False, AUTO), (16, 32, 2048, 2, False, AUTO)],
+    "fstep<32,2,1>": [(256, 32, 2048, 2, True, AUTO), (16, 32, 2048, 2, True, AUTO)],
+    "fstep<32,1,0>": [(40, 32, 1024, 2, False, AUTO)],
+    "fstep<32,0,1>": [(40, 32, 512, 3, True, AUTO)],
+    "fstep<16,2,0>": [(40, 16, 2048, 2, False, AUTO)],
+    "fstep<8,0,0>": [(33, 8, 256, 5, False, AUTO)],
+    "fstep<4,0,1>": [(33, 4, 128, 3, True, AUTO)],
+    # ... and the ring kernel's own fused form (on request; the offload step's groups)
+    "step<bf16,16,1,1,1,0,0>": [(256, 16, 768, 3, False, RING), (64, 16, 768, 12, False, RING)],
+    "step<bf16,16,1,1,2,0,0>": [(256, 16, 1024, 3, False, RING), (64, 16, 1024, 4, False, RING), (8, 16, 1024, 8, False, RING)],
+    "step<bf16,16,1,0,0,0,1>": [(256, 16, 768, 3, True, RING), (64, 16, 1024, 2, True, RING)],
+    "step<bf16,32,2,3,3,0,0>": [(256, 32, 2048, 1, False, AUTO), (256, 32, 2048, 3, False, RING)],
+    "step<bf16,32,2,3,4,0,0>": [(64, 32, 2048, 1, False, AUTO), (64, 32, 2048, 3, False, RING), (148, 32, 2048, 2, False, RING)],
+    "step<bf16,32,1,0,0,0,1>": [(16, 32, 2048, 1, True, AUTO), (16, 32, 2048, 2, True, RING)],
+    "step<bf16,32,2,0,0,0,1>": [(256, 32, 2048, 2, True, RING)],
 }
 FLAT = [(name,) + c for name, cs in CASES.items() for c in cs]
 
 
 def test_every_launch_shape_the_bench_times_has_a_parity_case():
+    import test_gpu_quant
+
+    covered = set(CASES) | test_gpu_quant.covered_variants()
     missing = {}
     for sh in bench.timed_launch_shapes():
-        name = mole.variant(sh["M"], sh["N"], sh["d"], L=sh["L"], norm=sh["norm"], kernel=sh["kernel"])[0]
-        if name not in CASES:
+        name = mole.variant(sh["M"], sh["N"], sh["d"], L=sh["L"], norm=sh["norm"], kernel=sh["kernel"],
+                            lut_format=sh["lut_format"], lut_block=sh["lut_block"])[0]
+        if name not in covered:
             missing.setdefault(name, []).append(sh["what"])
     assert not missing, missing
 
@@ -118,5 +133,8 @@ def test_variant_against_the_oracle(name, M, N, d, L, norm, kernel):
         assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref)) + slack).all(), (mode, float(err.max()))
         outs.append(out)
     if not norm:
-        # the two ways of launching a step differ only in the order of fp32 sums
+        # the two ways of launching a step differ at most in the order of fp32 sums
         assert (np.abs(as_f64(outs[0]) - as_f64(outs[1])) <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))).all()
+    if name.startswith("fstep") and mole.variant(M, N, d, norm=norm)[0].startswith("decode"):
+        # the fused step adds in the order of the one-block-per-token kernel: the bits of L chained launches of it
+        assert torch.equal(outs[0], outs[1])
