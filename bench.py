@@ -69,6 +69,17 @@ def offload_groups(L: int, M: int, row_bytes: int) -> int:
     return -(-L // g)
 
 
+def decode_family_covers(M, sh, L) -> bool:
+    """Whether the one-block-per-token family (MOLE_KERNEL_DECODE) has a kernel for this launch."""
+    from paper_2503_15798_b200 import binding as mole
+
+    try:
+        mole.variant(M, sh.N, sh.d, L=L, kernel=mole.KERNEL_DECODE)
+        return True
+    except mole.MoleError:
+        return False
+
+
 def timed_launch_shapes():
     """Every launch shape a timed region of this file issues, as dicts (what, M, N, d, L, norm, kernel,
     lut_format, lut_block): the parity tests walk this list and require a parity case for the kernel
@@ -89,9 +100,9 @@ def timed_launch_shapes():
                 add(f"{name} batch {M} chained{tag}", M, sh, 1, norm)
                 if M <= 4096:
                     add(f"{name} batch {M} fused{tag}", M, sh, sh.L, norm)
-            add(f"{name} batch {M} chained, ring kernel", M, sh, 1, kernel=1)
-            if M <= 4096:
-                add(f"{name} batch {M} fused, ring kernel", M, sh, sh.L, kernel=1)
+            for L in (1, sh.L):
+                if (L == 1 or M <= 4096) and decode_family_covers(M, sh, L):
+                    add(f"{name} batch {M} {'chained' if L == 1 else 'fused'}, one block per token", M, sh, L, kernel=2)
             for fmt, tag in ((1, "nf4"), (2, "nf3")):
                 add(f"{name} batch {M} chained, {tag} table", M, sh, 1, fmt=fmt, block=QUANT_BLOCKS[name][tag])
     sh = inputs.SHAPES["410m"]
@@ -442,10 +453,13 @@ def config_rows(torch, mole, inputs, sh, L, luts, wrs, batches, steps, warmup, p
         bl = [inputs.make_ids(m, sh.V, seed=4000 + b + 7 * m, device=dev) for b in range(N_BATCHES_EXTRA)]
         k = max(10, min(steps, int(2e6 // max(m * L, 64))))
         row = {"batch": m, "steps": k}
-        modes = [("chained", mole.STEP_CHAINED, mole.KERNEL_AUTO, None),
-                 ("chained_ring_kernel", mole.STEP_CHAINED, mole.KERNEL_RING, None)]
+        modes = [("chained", mole.STEP_CHAINED, mole.KERNEL_AUTO, None)]
+        if decode_family_covers(m, sh, 1):
+            modes.append(("chained_one_block_per_token", mole.STEP_CHAINED, mole.KERNEL_DECODE, None))
         if m <= 4096:
-            modes += [("fused", mole.STEP_FUSED, mole.KERNEL_AUTO, None), ("fused_ring_kernel", mole.STEP_FUSED, mole.KERNEL_RING, None)]
+            modes.append(("fused", mole.STEP_FUSED, mole.KERNEL_AUTO, None))
+            if decode_family_covers(m, sh, L):
+                modes.append(("fused_one_block_per_token", mole.STEP_FUSED, mole.KERNEL_DECODE, None))
         for tag in qtables:
             modes.append(("chained_" + tag, mole.STEP_CHAINED, mole.KERNEL_AUTO, qtables[tag]))
         for name, mode, kernel, qt in modes:

@@ -83,8 +83,9 @@ extern "C" {
 /* which kernel family runs a single-layer launch (mole_args.kernel, mole_step_args.kernel) */
 #define MOLE_KERNEL_AUTO 0   /* the library's choice */
 #define MOLE_KERNEL_RING 1   /* persistent blocks, rows and router chunks streamed through a shared-memory ring: any shape */
-#define MOLE_KERNEL_DECODE 2 /* one block per token, rows held in registers, built for decode batches: bf16, N of 4, 8, \
-                                16 or 32, d a multiple of 128 up to 2048 (1024 for N = 32), d_split 0 */
+#define MOLE_KERNEL_DECODE 2 /* one block per token (single layer: rows held in registers; fused step: rows through a ring, \
+                                router matrix through registers): bf16, N of 4, 8, 16 or 32, d a multiple of 128 up to   \
+                                2048 (single layer with N = 32: up to 1024), d_split 0 */
 
 /* storage of a table (mole_args.lut_format): plain elements of `dtype`, or the quantised records of Sec. 4.5 / Table 8 */
 #define MOLE_LUT_PLAIN 0
@@ -130,11 +131,11 @@ typedef struct mole_args {
     uint32_t *status;      /* device status word (MOLE_STATUS_* bits OR-ed in), or NULL */
     int32_t B, T, N, d, V;
     int32_t dtype;         /* MOLE_DTYPE_* */
-    int32_t kernel;        /* MOLE_KERNEL_*; AUTO takes the decode kernel for up to 2048 tokens where it exists and
-                              d_split is 0, the ring kernel otherwise.  The two families add the same fp32 terms in a
-                              different order, so their outputs may differ in a rounding decision; within one family
-                              and launch shape a token's result is the same bits whatever batch it is in.
-                              MOLE_ERR_UNSUPPORTED_SHAPE if DECODE is asked for a shape it does not cover. */
+    int32_t kernel;        /* MOLE_KERNEL_*; AUTO is the ring kernel (measured at least as fast at every batch size on
+                              B200).  The two families add the same fp32 terms in a different order, so their outputs may
+                              differ in a rounding decision; within one family and launch shape a token's result is the
+                              same bits whatever batch it is in.  MOLE_ERR_UNSUPPORTED_SHAPE if DECODE is asked for a
+                              shape it does not cover. */
     int32_t d_split;       /* chunks a token's router matrix and rows are streamed in (1, 2, 4, 8 or 16; d/d_split must
                               stay a multiple of the vector width); 0 = auto: the fewest chunks of at most 32 KB.
                               The router matrix is cut by columns.  The rows are cut by experts (whole rows of
@@ -223,8 +224,8 @@ typedef struct mole_step_args {
     int32_t dtype;         /* MOLE_DTYPE_* */
     int32_t mode;          /* MOLE_STEP_* */
     int32_t d_split;       /* as mole_args.d_split */
-    int32_t kernel;        /* as mole_args.kernel, for the single-layer launches of CHAINED mode; a FUSED step of
-                              several layers always runs on the ring kernel */
+    int32_t kernel;        /* as mole_args.kernel: the family of the single-layer launches of CHAINED mode and of the
+                              one launch of FUSED mode */
     float norm_eps;        /* >= 0; read only with norm_weight_base */
     int32_t lut_format;    /* as mole_args.lut_format; quantised tables run as CHAINED steps (AUTO picks that) */
     int32_t lut_block;     /* as mole_args.lut_block */
@@ -416,6 +417,23 @@ MOLE_API int mole_offload_decode_step(mole_offload_ctx *ctx, const void *hidden_
 /* device pointers of a buffer's arrays, for inspection: uniq [max_tokens], slot [max_tokens], count [1], staging */
 MOLE_API int mole_offload_buffers(mole_offload_ctx *ctx, int buf, const int32_t **uniq, const int32_t **slot,
                          const int32_t **count, const void **staging);
+
+/* ---------------------------------------------------------------------------------------
+ * Re-parameterisation (Sec. 3.3, Eq. 6-7): build a layer's table from its routed experts,
+ *     LUT[i][j][:] = FFN_j(x_i),   FFN_j(x) = W2_j . gelu(W1_j . x)   (two matrices, no bias, exact erf GELU),
+ *     x_i = Embedding(i), or RMSNorm(Embedding(i)) * norm_weight when norm_weight is given (the
+ *     expert_layernorm of the training listing in App. A.1, folded into the table),
+ * as one forward pass over the whole embedding matrix: two bf16 tensor-core GEMMs with fp32 accumulation;
+ * the hidden activations gelu(W1 x) and the normalised rows are materialised in bf16.
+ *   embedding  device bf16 [V][d]          w1 device bf16 [N][D][d]          w2 device bf16 [N][d][D]
+ *   norm_weight device bf16 [d] or NULL    lut device bf16 [V][N][d] (written)
+ *   scratch    device, mole_build_lut_scratch_bytes() bytes (V*N*D bf16, plus V*d with a norm), 16-byte aligned
+ * d and D multiples of 8.  Asynchronous on `stream`; status as elsewhere (MOLE_STATUS_TIMEOUT if a bounded
+ * wait inside the kernel ran out: the table is then undefined).
+ * ------------------------------------------------------------------------------------- */
+MOLE_API int mole_build_lut_scratch_bytes(int V, int N, int d, int D, int with_norm, int64_t *bytes);
+MOLE_API int mole_build_lut(const void *embedding, const void *w1, const void *w2, const void *norm_weight, float norm_eps,
+                   void *lut, void *scratch, int V, int N, int d, int D, uint32_t *status, void *stream);
 
 /* ---------------------------------------------------------------------------------------
  * Table files: the tables of all L layers on a storage device below host memory (Sec. 3.3: the tables stay

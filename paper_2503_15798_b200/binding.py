@@ -31,7 +31,7 @@ EXPORTS = (
     "mole_offload_destroy", "mole_offload_prefetch", "mole_layer_forward_offload", "mole_offload_decode_step",
     "mole_offload_buffers",
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan", "mole_variant", "mole_reload_debug_env",
-    "mole_table_file_write", "mole_table_file_info", "mole_table_file_read", "mole_table_file_read_rows",
+    "mole_build_lut", "mole_build_lut_scratch_bytes", "mole_table_file_write", "mole_table_file_info", "mole_table_file_read", "mole_table_file_read_rows",
     "mole_decode_step_args", "mole_offload_create_ex", "mole_offload_set_hot_rows", "mole_offload_hot_hits", "mole_nf_codebook", "mole_quant_record_bytes", "mole_quantize_lut",
 )
 
@@ -105,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.mole_host_free.argtypes = [vp]
         L.mole_offload_create.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_int]
         L.mole_offload_create_ex.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int]
+        L.mole_build_lut_scratch_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int, POINTER(c_int64)]
+        L.mole_build_lut.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, c_int, c_int, c_int, c_int, vp, vp]
         L.mole_table_file_write.argtypes = [c_char_p, vp, c_int64, c_int, c_int, c_int, c_int, c_int, c_int, c_int]
         L.mole_table_file_info.argtypes = [c_char_p, POINTER(MoleTableInfo)]
         L.mole_table_file_read.argtypes = [c_char_p, vp, c_int64, c_int, c_int]
@@ -521,6 +523,28 @@ class debug_env:
             else:
                 os.environ[k] = old
         _check(lib().mole_reload_debug_env(), "mole_reload_debug_env")
+
+
+def build_lut(embedding, w1, w2, norm_weight=None, norm_eps: float = 1e-6, out=None, status=None, stream=None):
+    """mole_build_lut (Eq. 6-7 on the tensor cores): embedding [V][d], w1 [N][D][d], w2 [N][d][D], all bf16 on the
+    device; returns the table [V][N][d] bf16.  The scratch buffer is allocated here (torch) and freed on return."""
+    for name, t in (("embedding", embedding), ("w1", w1), ("w2", w2)):
+        _dev(t, name)
+        if t.dtype != torch.bfloat16:
+            raise TypeError("mole_build_lut takes bf16 inputs")
+    V, d = embedding.shape
+    N, D, d1 = w1.shape
+    if d1 != d or tuple(w2.shape) != (N, d, D):
+        raise ValueError("shape mismatch between embedding, w1 and w2")
+    if out is None:
+        out = torch.empty((V, N, d), dtype=torch.bfloat16, device=embedding.device)
+    b = c_int64()
+    _check(lib().mole_build_lut_scratch_bytes(V, N, d, D, int(norm_weight is not None), ctypes.byref(b)), "mole_build_lut_scratch_bytes")
+    scratch = torch.empty(b.value, dtype=torch.uint8, device=embedding.device)
+    _check(lib().mole_build_lut(_ptr(embedding), _ptr(w1), _ptr(w2), _ptr(norm_weight), float(norm_eps), _ptr(out), _ptr(scratch),
+                                V, N, d, D, _ptr(status), _stream(stream)), "mole_build_lut")
+    torch.cuda.current_stream().synchronize() if stream is None else None  # the scratch buffer dies with this frame
+    return out
 
 
 def table_file_write(path: str, tables, N: int, d: int, lut_format: int = LUT_PLAIN, lut_block: int = 0):

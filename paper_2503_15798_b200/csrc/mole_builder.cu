@@ -1,0 +1,355 @@
+// Re-parameterisation on the GPU (Sec. 3.3, Eq. 6-7 of arXiv 2503.15798): the table of a layer is the
+// output of every routed expert on every embedding row, LUT[i][j] = FFN_j(Embedding(i)) -- "a single
+// forward pass with the embedding matrix as the input".  This is the one dense contraction of the method,
+// so it runs on the 5th-generation tensor cores: two bf16 GEMMs with fp32 accumulation in tensor memory,
+//     H = gelu(X . W1^T)      X [V][d] (the embedding rows, optionally RMS-normalised as in the training
+//                             listing's expert_layernorm), W1 all experts stacked [N*D][d], H [V][N*D] bf16
+//     LUT[:, j, :] = H[:, jD:(j+1)D] . W2_j^T      per expert j, W2_j [d][D], written straight into [V][N][d]
+// each a launch of one kernel: C[z][m][n] = epilogue(sum_k A[z][m][k] * B[z][n][k]), both operands K-major.
+//
+// Kernel: one 128 x 128 output tile per block.  Warp 0 (one thread) streams 128 x 64 tiles of A and B
+// through a ring of shared-memory stages with tiled bulk tensor copies (128-byte swizzle, each into this
+// block's own shared memory); warp 1 (one thread) issues tcgen05.mma 128 x 128 x 16 on the staged tiles,
+// accumulating in 128 columns of tensor memory, and hands stages back with tcgen05.commit; warps 2-5 read
+// the accumulator back with tcgen05.ld, apply the epilogue (exact erf GELU for the first GEMM) and store
+// bf16.  Every wait is bounded; a wait that runs out sets MOLE_STATUS_TIMEOUT and the block winds down
+// (tensor memory is freed on every path).
+#include <cuda.h>
+#include <math.h>
+#include <mutex>
+#include <string.h>
+
+#include "mole_kernel.cuh"
+
+namespace mole {
+
+constexpr int kBM = 128, kBN = 128, kBK = 64;          // tile; kBK bf16 = one 128-byte swizzle span
+constexpr int kGemmStages = 6;
+constexpr int kTileBytes = kBM * kBK * 2;              // 16 KB, A and B tiles alike
+constexpr int kGemmThreads = 192;                      // producer warp, MMA warp, four epilogue warps
+constexpr uint32_t kGemmSmem = kGemmStages * 2 * kTileBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint32_t kGemmWaitPolls = 1u << 22;
+
+struct GemmParams {
+    void *c;                // bf16 output
+    long long c_row_stride; // elements between rows of C
+    long long c_z_stride;   // elements between the z slices of C
+    int M, N, K;            // per z slice
+    int gelu;               // epilogue: 1 = exact erf GELU
+    uint32_t *status;
+};
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *dead)
+{
+    for (uint32_t i = 0; i < kGemmWaitPolls; ++i) {
+        if (bar_try_wait(bar, parity)) return true;
+        if (i > 32) {
+            __nanosleep(40);
+            if ((i & 255u) == 0 && *dead) return false;
+        }
+    }
+    return false;
+}
+// shared-memory operand descriptor of tcgen05.mma: a K-major tile of rows x 64 bf16, rows 128 bytes apart,
+// 128-byte swizzle (as the tensor copy wrote it), 1024 bytes between groups of eight rows
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                      // leading-dimension offset (unused with a swizzled K-major tile)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;              // stride between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                      // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                      // 128-byte swizzle
+    return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = kBN
+__device__ __forceinline__ uint32_t umma_idesc()
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+
+__global__ void __launch_bounds__(kGemmThreads) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                    const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
+    unsigned char *ctl = smem_raw + (tiles - raw) + kGemmStages * 2 * kTileBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);  // full[stages], empty[stages], accumulator ready
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + (2 * kGemmStages + 1) * 8);
+    volatile int *dead = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + kGemmStages * 8, accum_bar = full0 + 2 * kGemmStages * 8;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN, z = blockIdx.z;
+    const int ktiles = (p.K + kBK - 1) / kBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2 * kGemmStages + 1; ++s) mbar_init(bars + s, 1);
+        *dead = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) {  // tensor memory: kBN columns for the 128 x kBN fp32 accumulator
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kBN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {  // ---- producer: tiles of A and B, kGemmStages ahead ----
+            for (int kt = 0; kt < ktiles; ++kt) {
+                const int s = kt % kGemmStages;
+                const uint32_t par = ((kt / kGemmStages) & 1) ^ 1;  // first pass: the stage has never been used
+                if (!bar_wait_bounded(empty0 + s * 8, par, dead)) {
+                    if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                    *dead = 1;
+                    break;
+                }
+                const uint32_t a_dst = tiles + s * 2 * kTileBytes, b_dst = a_dst + kTileBytes;
+                mbar_expect_tx(bars + s, 2 * kTileBytes);
+                tma_load_3d(a_dst, &map_a, kt * kBK, m0, z, full0 + s * 8);
+                tma_load_3d(b_dst, &map_b, kt * kBK, n0, z, full0 + s * 8);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {  // ---- tensor-core issue ----
+            const uint32_t idesc = umma_idesc();
+            bool ok = true;
+            for (int kt = 0; kt < ktiles && ok; ++kt) {
+                const int s = kt % kGemmStages;
+                ok = bar_wait_bounded(full0 + s * 8, (kt / kGemmStages) & 1, dead);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_src = tiles + s * 2 * kTileBytes, b_src = a_src + kTileBytes;
+                const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+#pragma unroll
+                for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes along K inside the swizzle span: +2 in 16-byte units
+                    umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty0 + s * 8);  // the stage is free once these have read it
+            }
+            if (ok) {
+                umma_commit(accum_bar);
+            } else {
+                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                *dead = 1;
+            }
+        }
+    } else {
+        // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread ----
+        const bool ok = bar_wait_bounded(accum_bar, 0, dead);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const int quarter = warp & 3;
+            const int row = m0 + quarter * 32 + lane;
+            __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(p.c) + static_cast<long long>(z) * p.c_z_stride +
+                                  static_cast<long long>(row) * p.c_row_stride + n0;
+#pragma unroll 1
+            for (int c = 0; c < kBN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(c * 32), r);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row < p.M) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0 = __uint_as_float(r[i]), x1 = __uint_as_float(r[i + 1]);
+                        if (p.gelu) {
+                            x0 = 0.5f * x0 * (1.0f + erff(x0 * 0.70710678118654752440f));
+                            x1 = 0.5f * x1 * (1.0f + erff(x1 * 0.70710678118654752440f));
+                        }
+                        const int col = n0 + c * 32 + i;
+                        if (col + 1 < p.N) {
+                            *reinterpret_cast<__nv_bfloat162 *>(crow + c * 32 + i) = __floats2bfloat162_rn(x0, x1);
+                        } else if (col < p.N) {
+                            crow[c * 32 + i] = __float2bfloat16_rn(x0);
+                        }
+                    }
+                }
+            }
+        } else if (lane == 0 && !*dead && p.status) {
+            atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kBN) : "memory");
+    }
+}
+
+// y = (x / sqrt(mean(x^2) + eps)) * w, rounded once to bf16: the embedding rows as the routed experts of the
+// training listing see them.  One warp per row.
+__global__ void mole_rmsnorm_rows_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w,
+                                         __nv_bfloat16 *__restrict__ y, long long rows, int d, float eps)
+{
+    const long long row = static_cast<long long>(blockIdx.x) * (blockDim.x / 32) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const __nv_bfloat16 *xr = x + row * d;
+    float ss = 0.f;
+    for (int c = lane; c < d; c += 32) {
+        const float v = __bfloat162float(xr[c]);
+        ss = fmaf(v, v, ss);
+    }
+    ss = warp_sum(ss);
+    const float r = 1.0f / sqrtf(ss / static_cast<float>(d) + eps);
+    for (int c = lane; c < d; c += 32) y[row * d + c] = __float2bfloat16_rn((__bfloat162float(xr[c]) * r) * __bfloat162float(w[c]));
+}
+
+#endif  // __CUDACC__
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    });
+    return fn;
+}
+
+// K-major bf16 operand [z][rows][k]: rows row_stride elements apart, z slices z_stride elements apart
+static int make_operand_map(CUtensorMap *map, const void *base, long long k, long long rows, long long zs, long long row_stride,
+                            long long z_stride)
+{
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return MOLE_ERR_CUDA;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(k), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(zs)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(row_stride) * 2, static_cast<cuuint64_t>(z_stride) * 2};
+    const cuuint32_t box[3] = {kBK, kBM, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MOLE_OK : MOLE_ERR_CUDA;
+}
+
+// C[z][m][n] = epilogue(sum_k A[z][m][k] B[z][n][k])
+static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stride, const void *b, long long b_row_stride,
+                       long long b_z_stride, void *c, long long c_row_stride, long long c_z_stride, int M, int N, int K, int Z, int gelu,
+                       uint32_t *status, cudaStream_t st)
+{
+    CUtensorMap map_a, map_b;
+    int rc = make_operand_map(&map_a, a, K, M, Z, a_row_stride, a_z_stride);
+    if (rc != MOLE_OK) return rc;
+    rc = make_operand_map(&map_b, b, K, N, Z, b_row_stride, b_z_stride);
+    if (rc != MOLE_OK) return rc;
+    rc = ensure_smem_opt_in(reinterpret_cast<const void *>(mole_gemm_tn_kernel), static_cast<int>(kGemmSmem));
+    if (rc != MOLE_OK) return rc;
+    GemmParams p;
+    p.c = c;
+    p.c_row_stride = c_row_stride;
+    p.c_z_stride = c_z_stride;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.gelu = gelu;
+    p.status = status;
+    dim3 grid(static_cast<unsigned>((M + kBM - 1) / kBM), static_cast<unsigned>((N + kBN - 1) / kBN), static_cast<unsigned>(Z));
+    mole_gemm_tn_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
+    MOLE_CUDA_TRY(cudaGetLastError());
+    return MOLE_OK;
+}
+
+}  // namespace mole
+
+using namespace mole;
+
+extern "C" {
+
+int mole_build_lut_scratch_bytes(int V, int N, int d, int D, int with_norm, int64_t *bytes)
+{
+    if (!bytes || V < 1 || N < 1 || N > 64 || d < 8 || D < 8 || (d & 7) || (D & 7)) return MOLE_ERR_INVALID_ARG;
+    int64_t b = static_cast<int64_t>(V) * N * D * 2;
+    if (with_norm) b += (static_cast<int64_t>(V) * d * 2 + 255) / 256 * 256;
+    *bytes = b;
+    return MOLE_OK;
+}
+
+int mole_build_lut(const void *embedding, const void *w1, const void *w2, const void *norm_weight, float norm_eps, void *lut,
+                   void *scratch, int V, int N, int d, int D, uint32_t *status, void *stream)
+{
+    if (V < 1 || N < 1 || N > 64 || d < 8 || D < 8 || (d & 7) || (D & 7)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    if (static_cast<long long>(N) * D > 0x7fffffffLL / 2 || V > 0x7fffffff / 2) return MOLE_ERR_TOO_LARGE;
+    if (!embedding || !w1 || !w2 || !lut || !scratch) return MOLE_ERR_INVALID_ARG;
+    if (!aligned16(embedding) || !aligned16(w1) || !aligned16(w2) || !aligned16(lut) || !aligned16(scratch)) return MOLE_ERR_INVALID_ARG;
+    if (norm_weight && (!aligned16(norm_weight) || !(norm_eps >= 0.f) || norm_eps > 3.0e38f)) return MOLE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *hbuf = static_cast<unsigned char *>(scratch);
+    const void *x = embedding;
+    if (norm_weight) {
+        __nv_bfloat16 *xn = reinterpret_cast<__nv_bfloat16 *>(hbuf);
+        hbuf += (static_cast<int64_t>(V) * d * 2 + 255) / 256 * 256;
+        const int warps = 8;
+        mole_rmsnorm_rows_kernel<<<static_cast<unsigned>((V + warps - 1) / warps), warps * 32, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(embedding), static_cast<const __nv_bfloat16 *>(norm_weight), xn, V, d, norm_eps);
+        MOLE_CUDA_TRY(cudaGetLastError());
+        x = xn;
+    }
+    const long long ND = static_cast<long long>(N) * D;
+    // H = gelu(X . W1^T): one GEMM over all experts' first matrices stacked [N*D][d]
+    int rc = launch_gemm(x, d, static_cast<long long>(V) * d, w1, d, ND * d, hbuf, ND, static_cast<long long>(V) * ND, V, static_cast<int>(ND), d,
+                         1, 1, status, st);
+    if (rc != MOLE_OK) return rc;
+    // LUT[:, j, :] = H[:, jD:(j+1)D] . W2_j^T: z = expert; A's z slices are D columns apart, C's are d columns apart
+    return launch_gemm(hbuf, ND, D, w2, D, static_cast<long long>(d) * D, lut, static_cast<long long>(N) * d, d, V, d, D, N, 0, status, st);
+}
+
+}  // extern "C"

@@ -8,10 +8,11 @@
 //   - d / 4 compute threads: thread i owns columns 4i .. 4i+3 of the hidden state (in registers, fp32
 //     arithmetic, rounded to bf16 after every layer as a layer-by-layer execution would) and of every
 //     expert's row;
-//   - one producer warp streams, `stages` chunks ahead through a ring of 32 KB shared-memory slots, first
-//     the KW column chunks of the layer's router matrix, then the chunks of the token's rows (whole rows
-//     of N / kr experts, one contiguous bulk copy each); rows depend only on the id, so they run ahead of
-//     the arithmetic by several layers;
+//   - one producer warp streams, `stages` chunks ahead through a ring of 32 KB shared-memory slots, the
+//     chunks of the token's rows (whole rows of N / kr experts, one contiguous bulk copy each); rows depend
+//     only on the id, so they run ahead of the arithmetic by several layers.  The layer's router matrix
+//     comes from L2 straight into the compute threads' registers one item ahead (up to 16 experts), or
+//     through the same ring in column chunks in front of the rows (32 experts);
 //   - two block barriers per item: partial logits written / new hidden state written.  Every warp forms
 //     the softmax numerators itself from the per-warp partial logits (lane j <-> expert j) and hands them
 //     round by shuffles inside the weighted sum.
@@ -73,7 +74,7 @@ struct FStepCut {
 // N: experts (4, 8, 16, 32).  DB: width class (see FStepCut).  NORM: routers read RMSNorm(hidden) rounded
 // to bf16.  Launch: blockDim.x == d / 4 + 32, p.kr == KR, p.rexp == REXP.
 template <int N, int DB, int NORM>
-__global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(const FStepParams p)
+__global__ void __launch_bounds__(FStepCut<N, DB>::dmax / 4 + 32) mole_fstep_kernel(const FStepParams p)
 {
     constexpr int KW = FStepCut<N, DB>::KW, REXP = FStepCut<N, DB>::REXP, KR = FStepCut<N, DB>::KR;
     using E = Elem<__nv_bfloat16>;
@@ -83,6 +84,13 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
     constexpr int CPV = N >= VEC ? 1 : VEC / N;
     constexpr int RQ = N / 2 / KW;  // sweep vectors per thread and router chunk
     static_assert(RQ >= 1 && RQ * KW * 2 == N, "chunk count must divide N / 2");
+    // Up to 16 experts the router matrix does not travel through the ring at all: every compute thread loads
+    // its N / 2 vectors of the NEXT item's matrix straight from global memory (L2: all blocks share it) into
+    // registers as soon as the current sweep has used them up.  The ring then carries rows only -- half the
+    // bytes per item, twice the items in flight -- which is what a block's copy pipeline can keep up with.
+    constexpr bool WREG = N <= 16;
+    constexpr int KWR = WREG ? 0 : KW;  // router chunks per item in the ring
+    constexpr int RW = N / 2;           // vectors of a whole matrix per thread
     extern __shared__ __align__(128) unsigned char smem[];
 
     pdl_launch_dependents();
@@ -91,7 +99,7 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
     const long long G = gridDim.x, b0 = blockIdx.x;
     const int ntok = b0 < p.M ? static_cast<int>((p.M - b0 + G - 1) / G) : 0;
-    constexpr int kr = KR, rexp = REXP, cpi = KW + KR;  // chunks per item
+    constexpr int kr = KR, rexp = REXP, cpi = KWR + KR;  // chunks per item
     const FStepSmem m = fstep_smem(N, d, stages, NORM);
     const uint32_t wchunk_bytes = static_cast<uint32_t>(d) * N * 2 / KW, rchunk_bytes = static_cast<uint32_t>(rexp) * d * 2;
 
@@ -146,7 +154,7 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
             const bool valid = row >= 0 && row < p.rows;
             unsigned char *slot = smem + static_cast<size_t>(pst) * kFStepSlotBytes;
             if (lane == 0) {
-                if (q < KW) {
+                if (q < KWR) {
                     mbar_expect_tx(full + pst, wchunk_bytes);
                     bulk_g2s(slot,
                              static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(l) * p.wr_stride +
@@ -156,11 +164,11 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
                     // whole rows of experts (q - KW) * rexp ..: contiguous.  An id outside the table gathers
                     // row 0 (always present); its routed term is dropped by the consumers.
                     meta[pst] = valid ? 1 : 0;
-                    if (!valid && l == 0 && q == KW && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
+                    if (!valid && l == 0 && q == KWR && p.status) atomicOr(p.status, MOLE_STATUS_BAD_ID);
                     mbar_expect_tx(full + pst, rchunk_bytes);
                     bulk_g2s(slot,
                              static_cast<const unsigned char *>(p.lut) + static_cast<size_t>(l) * p.lut_stride +
-                                 (static_cast<size_t>(valid ? row : 0) * N + static_cast<size_t>(q - KW) * rexp) * d * 2,
+                                 (static_cast<size_t>(valid ? row : 0) * N + static_cast<size_t>(q - KWR) * rexp) * d * 2,
                              rchunk_bytes, full + pst);
                 }
                 *issued = static_cast<int>(ci + 1 < 0x7fffffff ? ci + 1 : 0x7fffffff);
@@ -205,6 +213,16 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
         }
     };
 
+    uint4 wreg[WREG ? RW : 1];
+    auto load_router = [&](int l) {  // this thread's vectors of layer l's matrix: u = tid + r * T, 16 bytes per lane, coalesced
+        const uint4 *w = reinterpret_cast<const uint4 *>(static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(l) * p.wr_stride);
+#pragma unroll
+        for (int r = 0; r < RW; ++r) wreg[r] = ldg_nc_v4(w + tid + r * T);
+    };
+    if constexpr (WREG) {
+        if (ntok > 0) load_router(0);
+    }
+
 #pragma unroll 1
     for (int k = 0; k < ntok; ++k) {
         const long long t = b0 + static_cast<long long>(k) * G;
@@ -240,24 +258,42 @@ __global__ void __launch_bounds__(kDecodeMaxThreads + 32) mole_fstep_kernel(cons
             float acc[NV];
 #pragma unroll
             for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+            if constexpr (WREG) {
+                unsigned short hs[RW * CPV];
 #pragma unroll
-            for (int q = 0; q < KW; ++q) {
-                acquire();
-                const uint32_t wbase = smem_base + static_cast<uint32_t>(st) * kFStepSlotBytes;
-                uint4 wv[RQ];
-                unsigned short hs[RQ * CPV];
-#pragma unroll
-                for (int r = 0; r < RQ; ++r) {
-                    wv[r] = lds128(wbase + 16u * static_cast<uint32_t>(tid + r * T));
-                    const int u = tid + (q * RQ + r) * T;  // vector index in the whole matrix
+                for (int r = 0; r < RW; ++r) {
+                    const int u = tid + r * T;
 #pragma unroll
                     for (int cc = 0; cc < CPV; ++cc) hs[r * CPV + cc] = static_cast<unsigned short>(lds16(rd_s + 2u * (N >= VEC ? u / QL : u * CPV + cc)));
                 }
-                release();  // the chunk is in registers
 #pragma unroll
-                for (int r = 0; r < RQ; ++r)
+                for (int r = 0; r < RW; ++r)
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) E::fma_elem(acc[e % NV], wv[r], e, hs[r * CPV + e / NV]);
+                    for (int e = 0; e < VEC; ++e) E::fma_elem(acc[e % NV], wreg[r], e, hs[r * CPV + e / NV]);
+                // the registers are free again: request the next item's matrix (the next layer's, or layer 0's for
+                // the block's next token); it lands while this item's softmax and weighted sum run
+                if (l + 1 < L) load_router(l + 1);
+                else if (k + 1 < ntok) load_router(0);
+            } else {
+#pragma unroll
+                for (int q = 0; q < KW; ++q) {
+                    acquire();
+                    const uint32_t wbase = smem_base + static_cast<uint32_t>(st) * kFStepSlotBytes;
+                    uint4 wv[RQ];
+                    unsigned short hs[RQ * CPV];
+#pragma unroll
+                    for (int r = 0; r < RQ; ++r) {
+                        wv[r] = lds128(wbase + 16u * static_cast<uint32_t>(tid + r * T));
+                        const int u = tid + (q * RQ + r) * T;  // vector index in the whole matrix
+#pragma unroll
+                        for (int cc = 0; cc < CPV; ++cc) hs[r * CPV + cc] = static_cast<unsigned short>(lds16(rd_s + 2u * (N >= VEC ? u / QL : u * CPV + cc)));
+                    }
+                    release();  // the chunk is in registers
+#pragma unroll
+                    for (int r = 0; r < RQ; ++r)
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) E::fma_elem(acc[e % NV], wv[r], e, hs[r * CPV + e / NV]);
+                }
             }
             int base = 0;
             lane_reduce_scatter<NV, NV, 16, QL>(acc, lane, base);

@@ -29,7 +29,6 @@ constexpr int kNumSMs = 148;                  // B200; used when no device can b
 constexpr int kSmemPerBlockMax = 227 * 1024;  // opt-in limit per block
 constexpr int kSmemPerSM = 228 * 1024;        // per SM, of which every resident block reserves 1 KB
 constexpr long long kFusedMaxTokens = 4096;   // above this a step runs as L chained launches
-constexpr long long kDecodeKernelMaxTokens = 2048;  // single-layer launches up to here take the one-block-per-token kernel
 
 // ---- debugging aids: the MOLE_FORCE_* / MOLE_DEBUG_* variables, read once ---------------------------
 struct DebugEnv {
@@ -502,7 +501,11 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     FStepPlan fplan;
     const bool fstep_ok = L > 1 && d_split == 0 && plan_fstep(M, L, N, d, dtype, norm, sms, &fplan);
     if (kernel == MOLE_KERNEL_DECODE && !(decode_ok || fstep_ok)) return MOLE_ERR_UNSUPPORTED_SHAPE;
-    if (fstep_ok && kernel != MOLE_KERNEL_RING) {
+    // MOLE_KERNEL_AUTO takes the ring kernel for plain tables: measured on B200, neither the one-block-per-token
+    // kernel (chained steps) nor the fused step built on it beats it -- a decode batch is bound by the latency of one
+    // token's dependent instruction stream, which the two families execute at about the same length.  They run on
+    // request (MOLE_KERNEL_DECODE), and their structure carries the quantised tables.
+    if (fstep_ok && kernel == MOLE_KERNEL_DECODE) {
         const FStepVariant v = pick_fstep(N, fplan.db, norm);
         if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
         c->fstep = true;
@@ -526,7 +529,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
         if (c->grid > M) c->grid = M;
         return MOLE_OK;
     }
-    if (decode_ok && (kernel == MOLE_KERNEL_DECODE || (kernel == MOLE_KERNEL_AUTO && M <= kDecodeKernelMaxTokens))) {
+    if (decode_ok && kernel == MOLE_KERNEL_DECODE) {
         const DecodeVariant v = pick_decode(N, norm);
         if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
         c->decode = true;

@@ -41,22 +41,22 @@ def test_version_and_status_strings(lib):
 
 def test_variant_names_and_kernel_choice(lib):
     V = binding.variant
-    # decode batches of the paper's 160M / 410M widths: the one-block-per-token kernel, d / 4 threads
-    assert V(256, 16, 768) == ("decode<16,0>", 192, V(256, 16, 768)[2]) and V(64, 16, 1024)[:2] == ("decode<16,0>", 256)
-    assert V(256, 16, 768, norm=True)[0] == "decode<16,1>"
-    # beyond 2048 tokens, with an explicit chunk count, for several layers, or on request: the ring kernel
-    assert V(16384, 16, 1024)[0] == "step<bf16,16,1,2,2,0,0>"
-    assert V(256, 16, 768, d_split=1)[0] == "step<bf16,16,1,2,1,1,0>"
-    assert V(256, 16, 768, L=12)[0] == "fstep<16,1,0>" and V(256, 16, 768, L=12, kernel=binding.KERNEL_RING)[0] == "step<bf16,16,1,1,1,0,0>"
-    assert V(256, 16, 768, kernel=binding.KERNEL_RING)[0] == "step<bf16,16,1,2,1,1,0>"
-    # the 1B width (512 column groups of 8 bytes, N = 32) is outside the decode kernel: ring kernel, rows cut by experts
-    assert V(256, 32, 2048)[0] == "step<bf16,32,2,3,3,0,0>" and V(64, 32, 2048, L=16)[0] == "fstep<32,2,0>"
-    assert V(64, 32, 2048, L=16, kernel=binding.KERNEL_RING)[0] == "step<bf16,32,2,3,4,0,0>"
-    with pytest.raises(binding.MoleError) as e:
-        V(256, 32, 2048, kernel=binding.KERNEL_DECODE)
-    assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
-    assert V(64, 32, 1024)[0] == "decode<32,0>" and V(64, 5, 768)[0].startswith("step<bf16,0,")
-    assert V(64, 4, 64, binding.DTYPE_F32)[0].startswith("step<f32,4,")
+    D, R = binding.KERNEL_DECODE, binding.KERNEL_RING
+    # the library's own choice: the ring kernel, single layers and fused steps alike
+    assert V(256, 16, 768)[0] == "step<bf16,16,1,2,1,1,0>" == V(256, 16, 768, kernel=R)[0]
+    assert V(16384, 16, 1024)[0] == "step<bf16,16,1,2,2,0,0>" and V(256, 16, 768, L=12)[0] == "step<bf16,16,1,1,1,0,0>"
+    assert V(256, 32, 2048)[0] == "step<bf16,32,2,3,3,0,0>" and V(64, 32, 2048, L=16)[0] == "step<bf16,32,2,3,4,0,0>"
+    # on request: one block per token (d / 4 threads), and the fused step built on it
+    assert V(256, 16, 768, kernel=D) == ("decode<16,0>", 192, V(256, 16, 768, kernel=D)[2]) and V(64, 16, 1024, kernel=D)[:2] == ("decode<16,0>", 256)
+    assert V(256, 16, 768, norm=True, kernel=D)[0] == "decode<16,1>" and V(64, 32, 1024, kernel=D)[0] == "decode<32,0>"
+    assert V(256, 16, 768, L=12, kernel=D)[0] == "fstep<16,1,0>" and V(64, 32, 2048, L=16, kernel=D)[0] == "fstep<32,2,0>"
+    for args, kw in (((256, 32, 2048), {}), ((64, 5, 768), {}), ((64, 16, 768), {"d_split": 2}), ((64, 4, 64, binding.DTYPE_F32), {})):
+        with pytest.raises(binding.MoleError) as e:  # shapes the family does not cover
+            V(*args, kernel=D, **kw)
+        assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    assert V(64, 5, 768)[0].startswith("step<bf16,0,") and V(64, 4, 64, binding.DTYPE_F32)[0].startswith("step<f32,4,")
+    # quantised tables
+    assert V(256, 16, 768, lut_format=binding.LUT_NF4, lut_block=768)[0] == "qdecode<16,nf4,0>"
 
 
 def test_plan_shapes():

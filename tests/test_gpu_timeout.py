@@ -50,7 +50,7 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_stream_stays_usable(kernel
     assert (buf[:GUARD] == 12345.0).all() and (buf[GUARD + M:] == 12345.0).all()
 
 
-@pytest.mark.parametrize("kernel", [mole.KERNEL_AUTO, mole.KERNEL_RING])
+@pytest.mark.parametrize("kernel", [mole.KERNEL_DECODE, mole.KERNEL_RING])
 def test_the_producer_of_the_ring_gives_up_when_no_slot_comes_back(kernel):
     """More chunks per block than ring slots: with a limit of zero polls the producer's first wait for a free
     slot runs out, it stops issuing, and the consumers, told so, stop waiting too."""
@@ -63,7 +63,7 @@ def test_the_producer_of_the_ring_gives_up_when_no_slot_comes_back(kernel):
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     buf, out = _padded_out(M, d)
     assert mole.plan(M, N, d, mole.DTYPE_BF16, 0, L)[3] < 2 * L
-    assert mole.variant(M, N, d, L=L, kernel=kernel)[0].startswith("fstep" if kernel == mole.KERNEL_AUTO else "step")
+    assert mole.variant(M, N, d, L=L, kernel=kernel)[0].startswith("fstep" if kernel == mole.KERNEL_DECODE else "step")
     with mole.debug_env(MOLE_DEBUG_WAIT_LIMIT=-1):
         mole.decode_step_args(hidden, ids, luts, wrs, out, None, status=status, mode=mole.STEP_FUSED, kernel=kernel)
         torch.cuda.synchronize()
