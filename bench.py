@@ -50,12 +50,16 @@ N_BATCHES_EXTRA = 16    # ... and the rows beside it
 MIN_SPAN_S = 0.25       # the timed region is repeated until the repeats span this long
 OFFLOAD_CONTEXT_TOKENS = 256  # offload mode: the context (staging areas) is sized for this many tokens
 OFFLOAD_BATCHES = (1, 8, 64)
+OFFLOAD_HOT_ROWS = 1024       # ids whose rows (all layers) the offload rows "with a hot-row cache" keep in HBM
 FALLBACK_HBM_GBS = 6650.0
 QUANT_BLOCKS = {"160m": {"nf4": 768, "nf3": 128}, "410m": {"nf4": 1024, "nf3": 128}, "1b": {"nf4": 1024, "nf3": 128}}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ ((config, batch, layers) -> bytes); None until one is taken
 # of the kernel as it stands
-TRAFFIC = {}
+TRAFFIC = {
+    # profiles/mole_step_kernel_single_layer_160m_batch256.md: mean of three captured launches (one layer each)
+    ("160m", 256, 12): 4.29e6,
+}
 FUSED_TRAFFIC = {}
 
 
@@ -133,6 +137,10 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override L (debugging; the line then says so)")
     ap.add_argument("--vocab", type=int, default=0,
                     help="override V, the number of table rows (small profiler captures; the line then says so)")
+    ap.add_argument("--min-span-s", type=float, default=MIN_SPAN_S,
+                    help="repeat every timed region until the repeats span this long (0: three repeats; profiler captures)")
+    ap.add_argument("--builder", action="store_true",
+                    help="the table builder alone (Eq. 6-7 on the tensor cores), one 160M-shaped layer; --vocab shrinks it")
     ap.add_argument("--offload", action="store_true",
                     help="offload mode alone: table in pinned host memory, per-step dedup + row fetch overlapped with "
                          "the previous layers' combine; roofline = measured host-link GB/s")
@@ -240,9 +248,10 @@ def reference_arm_runs_here(rank: int) -> bool:
     return rank == 0
 
 
-def repeats_for(ms_one: float, min_span_s: float = MIN_SPAN_S) -> int:
+def repeats_for(ms_one: float, min_span_s: float = None) -> int:
     """How often a timed region of ms_one milliseconds is repeated to span min_span_s (at least 3, at most 4000)."""
-    return max(3, min(4000, int(math.ceil(min_span_s * 1e3 / max(ms_one, 1e-6)))))
+    span = MIN_SPAN_S if min_span_s is None else min_span_s
+    return max(3, min(4000, int(math.ceil(span * 1e3 / max(ms_one, 1e-6)))))
 
 
 # ------------------------------------------------------------------------------------------------------
@@ -533,6 +542,45 @@ def isolated_rows(torch, mole, inputs, sh, luts, wrs, batches, peak, dev):
     return rows
 
 
+def measured_tensor_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst: the builder is timed alone)"
+    except Exception:
+        return 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+
+
+def builder_row(torch, mole, inputs, dev, vocab=0):
+    """The re-parameterisation of one 160M-shaped layer (Eq. 6-7): V = 50304 embedding rows through N = 16 experts
+    of width D = 4 d = 3072 (Table 2), two tensor-core GEMMs; TFLOP/s against the measured bf16 GEMM rate."""
+    sh = inputs.SHAPES["160m"]
+    if vocab > 0:
+        sh = dataclasses.replace(sh, V=vocab)
+    D = 4 * sh.d
+    g = torch.Generator(device=dev)
+    g.manual_seed(77)
+    E = torch.empty((sh.V, sh.d), dtype=torch.bfloat16, device=dev).normal_(0, 1, generator=g)
+    W1 = torch.empty((sh.N, D, sh.d), dtype=torch.bfloat16, device=dev).normal_(0, sh.d ** -0.5, generator=g)
+    W2 = torch.empty((sh.N, sh.d, D), dtype=torch.bfloat16, device=dev).normal_(0, D ** -0.5, generator=g)
+    lut = torch.empty((sh.V, sh.N, sh.d), dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    mole.build_lut(E, W1, W2, out=lut, status=status)  # allocates its scratch buffer through torch; synchronises
+    times = []
+    for _ in range(3):
+        torch.cuda.synchronize()
+        times.append(event_ms(torch, lambda: mole.build_lut(E, W1, W2, out=lut, status=status)))
+    assert int(status.item()) == 0
+    ms = statistics.median(times)
+    flops = 2 * 2.0 * sh.V * sh.d * D * sh.N
+    peak, src = measured_tensor_peak()
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"V": sh.V, "d": sh.d, "D": D, "N": sh.N, "ms_per_layer": ms, "flops_per_layer": flops, "TFLOPps": tf,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
+                         "kernel": "mole_gemm_tn_kernel", "peak_source": src},
+            "table_rows_per_s": sh.V / (ms * 1e-3)}
+
+
 def run_mole(args):
     import numpy as np
     import torch
@@ -612,6 +660,20 @@ def run_mole(args):
                      "algorithmic_bytes_per_launch": launch_bytes, "us_per_launch": ms * 1e3 / launches},
         "clocks": clocks.summary(),
     }
+    if extras:
+        # the same chained step issued from the host every step (no CUDA graph): what the library's launch path costs
+        ids_all, out_h, tmp_h, st_h = graphs.id_batches, graphs.out, graphs.tmp, graphs.status
+        step_fn = plain_step(mole.STEP_CHAINED)
+
+        def host_run(k0, k1):
+            for k in range(k0, k1):
+                step_fn(ids_all[k % N_BATCHES], out_h, tmp_h, st_h)
+
+        ms_h, _ = timed_steps(torch, host_run, args.steps, args.warmup)
+        line["chained_step_host_issued"] = {"what": "the headline's step without a CUDA graph: one mole_decode_step_args call per step, "
+                                                    "L launches issued by the library from the host",
+                                            "us_per_step": ms_h * 1e3 / args.steps, "value": M * args.steps / (ms_h * 1e-3), "unit": UNIT,
+                                            "ratio_to_graph_replay": ms_h / ms}
     del graphs
 
     # ---- extra, never the headline: the same step as ONE launch that keeps a token's chain through all L
@@ -752,6 +814,11 @@ def run_mole(args):
             except Exception as e:  # e.g. not enough device memory for the 105 GB table on a smaller part
                 configs[name] = {"error": f"{type(e).__name__}: {e}"}
             torch.cuda.empty_cache()
+        try:
+            configs["builder_160m_layer"] = builder_row(torch, mole, inputs, dev)
+        except Exception as e:
+            configs["builder_160m_layer"] = {"error": f"{type(e).__name__}: {e}"}
+        torch.cuda.empty_cache()
         if not args.no_offload:
             try:
                 configs["410m_offload"] = offload_rows(args, torch, mole, inputs, dev)
@@ -823,11 +890,14 @@ def offload_rows(args, torch, mole, inputs, dev, formats=("bf16", "nf4", "nf3"))
                                    "of the pinned table")
             del big
         rows = []
-        for M in OFFLOAD_BATCHES:
+        hot_ids = inputs.zipf_hot_ids(sh.V, OFFLOAD_HOT_ROWS)
+        for M, hot in [(m, False) for m in OFFLOAD_BATCHES] + ([(m, True) for m in OFFLOAD_BATCHES] if fmt == mole.LUT_PLAIN else []):
             # one context sized for a server's largest batch (256 tokens: two staging areas): at the batches timed
             # here a staging area has room for several layers' rows, fetched in one launch
             ctx = mole.OffloadContext(OFFLOAD_CONTEXT_TOKENS, sh.N, sh.d, sh.V, torch.bfloat16, n_buffers=2, lut_format=fmt,
                                       lut_block=block)
+            if hot:  # the rows of the most probable ids of all layers kept in HBM: they never cross the link again
+                ctx.set_hot_rows(hot_ids, host.tensor)
             hidden = inputs.make_hidden(M, sh.d, seed=3000, device=dev)
             bufs = [torch.empty_like(hidden), torch.empty_like(hidden)]
             id_batches = [inputs.make_ids(M, sh.V, seed=4000 + b + 7 * M, device=dev) for b in range(N_BATCHES)]
@@ -858,13 +928,20 @@ def offload_rows(args, torch, mole, inputs, dev, formats=("bf16", "nf4", "nf3"))
 
             ms, spread = timed_steps(torch, run, steps, 5)
             assert int(status.item()) == 0
-            del graphs
             us_step = ms * 1e3 / steps
             link_bytes = uniq_rows * row_bytes * L  # distinct rows only cross the link
-            rows.append({"batch": M, "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
+            hits_per_step = None
+            if hot:  # ... and of those, not the ones the hot-row cache serves (counted by the fetch kernel)
+                ctx.hot_hits(reset=True)
+                run(0, N_BATCHES)
+                hits_per_step = ctx.hot_hits() / N_BATCHES
+                link_bytes -= hits_per_step * row_bytes
+            rows.append({"batch": M, "hot_rows_cached": OFFLOAD_HOT_ROWS if hot else 0, "rows_from_cache_per_step": hits_per_step,
+                         "us_per_step": us_step, "tokens_per_s": M / (us_step * 1e-6),
                          "mean_distinct_ids": uniq_rows, "link_bytes_per_step": link_bytes,
                          "link_GBps": link_bytes / us_step / 1e3, "frac_of_link": link_bytes / us_step / 1e3 / link["peak_GBps"],
                          "us_per_step_without_graph": us_calls, "repeats": spread["repeats"]})
+            del graphs
             ctx.destroy()
         result[tag] = {"row_bytes": row_bytes, "host_table_GB": row_bytes * sh.V * L / 1e9, "rows": rows}
         host.free()
@@ -885,7 +962,7 @@ def run_offload(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     res = offload_rows(args, torch, mole, inputs, dev)
-    top = res["bf16"]["rows"][-1]
+    top = [r for r in res["bf16"]["rows"] if r["batch"] == OFFLOAD_BATCHES[-1] and not r["hot_rows_cached"]][0]
     steps = max(20, min(args.steps, 200))
     line = {
         "metric": "MoLE offload-mode tokens/s (L-layer decode step) and achieved host-link GB/s", "value": top["tokens_per_s"],
@@ -905,8 +982,31 @@ def run_offload(args):
     print(json.dumps(line), flush=True)
 
 
+def run_builder(args):
+    """--builder: the table builder alone, one JSON line of its own."""
+    import torch
+
+    from paper_2503_15798_b200 import binding as mole
+    from paper_2503_15798_b200 import build as lib_build
+    from paper_2503_15798_b200 import inputs
+
+    lib_build.build()
+    torch.cuda.set_device(0)
+    row = builder_row(torch, mole, inputs, torch.device("cuda", 0), args.vocab)
+    line = {"metric": "MoLE table builder (Eq. 6-7) TFLOP/s, one 160M-shaped layer", "value": row["TFLOPps"], "unit": "TFLOP/s",
+            "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": row["ms_per_layer"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"re-parameterisation of one layer: V={row['V']}, d={row['d']}, D={row['D']}, N={row['N']}"},
+            "gpu_launches": 6, "roofline": row["roofline"], "builder": row}
+    print(json.dumps(line), flush=True)
+
+
 def main():
+    global MIN_SPAN_S
     args = parse_args()
+    MIN_SPAN_S = args.min_span_s
+    if args.builder:
+        return run_builder(args)
     if args.offload:
         return run_offload(args)
     if args.impl == "reference":

@@ -10,9 +10,11 @@
 // Kernel: one 128 x 128 output tile per block.  Warp 0 (one thread) streams 128 x 64 tiles of A and B
 // through a ring of shared-memory stages with tiled bulk tensor copies (128-byte swizzle, each into this
 // block's own shared memory); warp 1 (one thread) issues tcgen05.mma 128 x 128 x 16 on the staged tiles,
-// accumulating in 128 columns of tensor memory, and hands stages back with tcgen05.commit; warps 2-5 read
+// accumulating in 128 columns of tensor memory, and hands stages back with tcgen05.commit; warps 2-9 read
 // the accumulator back with tcgen05.ld, apply the epilogue (exact erf GELU for the first GEMM) and store
-// bf16.  Every wait is bounded; a wait that runs out sets MOLE_STATUS_TIMEOUT and the block winds down
+// bf16.  Two blocks fit an SM (96 KB of tiles, 128 of the 512 tensor-memory columns each), so that one
+// block's epilogue -- for the first GEMM, with erf, as long as its main loop -- runs under the other's
+// tensor-core work.  Every wait is bounded; a wait that runs out sets MOLE_STATUS_TIMEOUT and the block winds down
 // (tensor memory is freed on every path).
 #include <cuda.h>
 #include <math.h>
@@ -24,9 +26,9 @@
 namespace mole {
 
 constexpr int kBM = 128, kBN = 128, kBK = 64;          // tile; kBK bf16 = one 128-byte swizzle span
-constexpr int kGemmStages = 6;
+constexpr int kGemmStages = 3;                         // 96 KB of tiles: two blocks per SM, one's epilogue under the other's main loop
 constexpr int kTileBytes = kBM * kBK * 2;              // 16 KB, A and B tiles alike
-constexpr int kGemmThreads = 192;                      // producer warp, MMA warp, four epilogue warps
+constexpr int kGemmThreads = 320;                      // producer warp, MMA warp, eight epilogue warps
 constexpr uint32_t kGemmSmem = kGemmStages * 2 * kTileBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr uint32_t kGemmWaitPolls = 1u << 22;
 
@@ -113,7 +115,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr));
 }
 
-__global__ void __launch_bounds__(kGemmThreads) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
+__global__ void __launch_bounds__(kGemmThreads, 2) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                     const __grid_constant__ CUtensorMap map_b, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -183,7 +185,8 @@ __global__ void __launch_bounds__(kGemmThreads) mole_gemm_tn_kernel(const __grid
             }
         }
     } else {
-        // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread ----
+        // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread; the two warps
+        // that share a lane quarter take half of the columns each ----
         const bool ok = bar_wait_bounded(accum_bar, 0, dead);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
@@ -191,12 +194,15 @@ __global__ void __launch_bounds__(kGemmThreads) mole_gemm_tn_kernel(const __grid
             const int row = m0 + quarter * 32 + lane;
             __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(p.c) + static_cast<long long>(z) * p.c_z_stride +
                                   static_cast<long long>(row) * p.c_row_stride + n0;
+            const int c_begin = (warp - 2) < 4 ? 0 : kBN / 64, c_end = c_begin + kBN / 64;
 #pragma unroll 1
-            for (int c = 0; c < kBN / 32; ++c) {
+            for (int c = c_begin; c < c_end; ++c) {
                 uint32_t r[32];
                 tmem_ld32(tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(c * 32), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (row < p.M) {
+                    // 32 consecutive columns of this thread's row: round in pairs, store 16 bytes (8 columns) at a time
+                    uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
                         float x0 = __uint_as_float(r[i]), x1 = __uint_as_float(r[i + 1]);
@@ -204,12 +210,20 @@ __global__ void __launch_bounds__(kGemmThreads) mole_gemm_tn_kernel(const __grid
                             x0 = 0.5f * x0 * (1.0f + erff(x0 * 0.70710678118654752440f));
                             x1 = 0.5f * x1 * (1.0f + erff(x1 * 0.70710678118654752440f));
                         }
-                        const int col = n0 + c * 32 + i;
-                        if (col + 1 < p.N) {
-                            *reinterpret_cast<__nv_bfloat162 *>(crow + c * 32 + i) = __floats2bfloat162_rn(x0, x1);
-                        } else if (col < p.N) {
-                            crow[c * 32 + i] = __float2bfloat16_rn(x0);
-                        }
+                        const __nv_bfloat162 b = __floats2bfloat162_rn(x0, x1);
+                        packed[i / 2] = *reinterpret_cast<const uint32_t *>(&b);
+                    }
+                    const int col0 = n0 + c * 32;
+                    if (col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            *reinterpret_cast<uint4 *>(crow + c * 32 + v * 8) =
+                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < p.N)
+                                crow[c * 32 + i] = __ushort_as_bfloat16(static_cast<unsigned short>((i & 1) ? (packed[i / 2] >> 16) : (packed[i / 2] & 0xffffu)));
                     }
                 }
             }
