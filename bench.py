@@ -60,7 +60,10 @@ TRAFFIC = {
     # profiles/mole_step_kernel_single_layer_160m_batch256.md: mean of three captured launches (one layer each)
     ("160m", 256, 12): 4.29e6,
 }
-FUSED_TRAFFIC = {}
+FUSED_TRAFFIC = {
+    # profiles/mole_step_kernel_fused_160m_batch256.md: 8.1 MB per 2-layer launch, x6 for the 12 layers of a full launch
+    ("160m", 256, 12): 48.6e6,
+}
 
 
 def offload_groups(L: int, M: int, row_bytes: int) -> int:
