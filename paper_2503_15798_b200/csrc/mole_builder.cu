@@ -7,15 +7,15 @@
 //     LUT[:, j, :] = H[:, jD:(j+1)D] . W2_j^T      per expert j, W2_j [d][D], written straight into [V][N][d]
 // each a launch of one kernel: C[z][m][n] = epilogue(sum_k A[z][m][k] * B[z][n][k]), both operands K-major.
 //
-// Kernel: one 128 x 128 output tile per block.  Warp 0 (one thread) streams 128 x 64 tiles of A and B
-// through a ring of shared-memory stages with tiled bulk tensor copies (128-byte swizzle, each into this
-// block's own shared memory); warp 1 (one thread) issues tcgen05.mma 128 x 128 x 16 on the staged tiles,
-// accumulating in 128 columns of tensor memory, and hands stages back with tcgen05.commit; warps 2-9 read
-// the accumulator back with tcgen05.ld, apply the epilogue (exact erf GELU for the first GEMM) and store
-// bf16.  Two blocks fit an SM (96 KB of tiles, 128 of the 512 tensor-memory columns each), so that one
-// block's epilogue -- for the first GEMM, with erf, as long as its main loop -- runs under the other's
-// tensor-core work.  Every wait is bounded; a wait that runs out sets MOLE_STATUS_TIMEOUT and the block winds down
-// (tensor memory is freed on every path).
+// Kernel: persistent, one block per SM, each walking 128 x 256 output tiles (raster: eight tile rows by all
+// tile columns at a time, so that the blocks in flight share operand tiles in L2).  Warp 0 (one thread)
+// streams 128 x 64 tiles of A and 256 x 64 tiles of B through a four-stage ring of shared memory with tiled
+// bulk tensor copies (128-byte swizzle, each into this block's own shared memory); warp 1 (one thread) issues
+// tcgen05.mma 128 x 256 x 16 on the staged tiles and hands stages back with tcgen05.commit; the accumulator
+// is double-buffered in tensor memory (2 x 256 of the 512 columns), so that warps 2-9 read tile i back with
+// tcgen05.ld, apply the epilogue (GELU for the first GEMM) and store bf16 while the tensor cores already
+// work on tile i + 1.  Every wait is bounded; a wait that runs out sets MOLE_STATUS_TIMEOUT and the block
+// winds down: copies and MMAs in flight are waited for (again bounded) and tensor memory is freed on every path.
 #include <cuda.h>
 #include <math.h>
 #include <mutex>
@@ -25,19 +25,28 @@
 
 namespace mole {
 
-constexpr int kBM = 128, kBN = 128, kBK = 64;          // tile; kBK bf16 = one 128-byte swizzle span
-constexpr int kGemmStages = 3;                         // 96 KB of tiles: two blocks per SM, one's epilogue under the other's main loop
-constexpr int kTileBytes = kBM * kBK * 2;              // 16 KB, A and B tiles alike
-constexpr int kGemmThreads = 320;                      // producer warp, MMA warp, eight epilogue warps
-constexpr uint32_t kGemmSmem = kGemmStages * 2 * kTileBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kBM = 128, kBN = 256, kBK = 64;          // tile; kBK bf16 = one 128-byte swizzle span
+constexpr int kGemmStages = 4;                         // 192 KB of operand tiles in flight per SM
+constexpr int kTileBytesA = kBM * kBK * 2;             // 16 KB
+constexpr int kTileBytesB = kBN * kBK * 2;             // 32 KB
+constexpr int kStageBytes = kTileBytesA + kTileBytesB;
+constexpr int kAccBuffers = 2;                         // accumulators in tensor memory: 2 x kBN of the 512 columns
+constexpr int kTmemCols = kAccBuffers * kBN;
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = (2 + kEpiWarps) * 32;     // producer warp, MMA warp, eight epilogue warps
+constexpr int kRasterRows = 8;                         // tile rows walked together
+constexpr int kGemmBarriers = 2 * kGemmStages + 2 * kAccBuffers + 1;
+constexpr uint32_t kGemmSmem = kGemmStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr uint32_t kGemmWaitPolls = 1u << 22;
+static_assert(kTmemCols == 512 && kGemmBarriers * 8 <= 128, "tensor-memory columns are a power of two; barriers fit their block");
 
 struct GemmParams {
     void *c;                // bf16 output
     long long c_row_stride; // elements between rows of C
     long long c_z_stride;   // elements between the z slices of C
     int M, N, K;            // per z slice
-    int gelu;               // epilogue: 1 = exact erf GELU
+    int m_tiles, n_tiles;   // per z slice
+    int total_tiles;        // over all z slices
     uint32_t *status;
 };
 
@@ -61,9 +70,9 @@ __device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *dead)
+__device__ __forceinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *dead, uint32_t polls = kGemmWaitPolls)
 {
-    for (uint32_t i = 0; i < kGemmWaitPolls; ++i) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (bar_try_wait(bar, parity)) return true;
         if (i > 32) {
             __nanosleep(40);
@@ -71,6 +80,10 @@ __device__ __forceinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity, 
         }
     }
     return false;
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // shared-memory operand descriptor of tcgen05.mma: a K-major tile of rows x 64 bf16, rows 128 bytes apart,
 // 128-byte swizzle (as the tensor copy wrote it), 1024 bytes between groups of eight rows
@@ -84,7 +97,7 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
     d |= static_cast<uint64_t>(2) << 61;                      // 128-byte swizzle
     return d;
 }
-// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = kBN
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = kBM, N = kBN
 __device__ __forceinline__ uint32_t umma_idesc()
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
@@ -115,29 +128,70 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr));
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 2) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
+// GELU(x) = x Phi(x) with Phi through erfc(|x| / sqrt 2) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-x^2 / 2),
+// t = 1 / (1 + p |x| / sqrt 2) (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7 on erf): within 3.5e-7 of the exact
+// GELU everywhere, a fraction of the bf16 rounding that follows, at about half the instructions of erff().
+__device__ __forceinline__ float gelu_erf(float x)
+{
+    const float au = fabsf(x) * 0.70710678118654752440f;
+    const float t = __fdividef(1.0f, fmaf(0.3275911f, au, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"((x * x) * -0.72134752044448170368f));  // exp(-x^2 / 2)
+    const float erfc_au = poly * t * e;
+    return fmaxf(x, 0.0f) - fabsf(0.5f * x * erfc_au);  // x >= 0: x - x erfc / 2;  x < 0: x erfc / 2
+}
+
+struct TileCoord {
+    int m0, n0, z;
+};
+// tiles in the order the blocks walk them: z slice by z slice, kRasterRows tile rows at a time, down the rows first
+__device__ __forceinline__ TileCoord tile_coord(int tile, const GemmParams &p)
+{
+    const int per_z = p.m_tiles * p.n_tiles;
+    const int z = tile / per_z, r = tile - z * per_z;
+    const int band = r / (kRasterRows * p.n_tiles);
+    const int first = band * kRasterRows;
+    const int rows = min(kRasterRows, p.m_tiles - first);
+    const int w = r - band * kRasterRows * p.n_tiles;
+    TileCoord t;
+    t.m0 = (first + w % rows) * kBM;
+    t.n0 = (w / rows) * kBN;
+    t.z = z;
+    return t;
+}
+
+template <int GELU>
+__global__ void __launch_bounds__(kGemmThreads, 1) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                     const __grid_constant__ CUtensorMap map_b, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
-    unsigned char *ctl = smem_raw + (tiles - raw) + kGemmStages * 2 * kTileBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);  // full[stages], empty[stages], accumulator ready
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + (2 * kGemmStages + 1) * 8);
+    unsigned char *ctl = smem_raw + (tiles - raw) + kGemmStages * kStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);  // full[stages], empty[stages], acc_full[2], acc_empty[2], drain
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 128);
     volatile int *dead = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + kGemmStages * 8, accum_bar = full0 + 2 * kGemmStages * 8;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + kGemmStages * 8, acc_full0 = empty0 + kGemmStages * 8,
+                   acc_empty0 = acc_full0 + kAccBuffers * 8, drain_bar = acc_empty0 + kAccBuffers * 8;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN, z = blockIdx.z;
     const int ktiles = (p.K + kBK - 1) / kBK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 2 * kGemmStages + 1; ++s) mbar_init(bars + s, 1);
-        *dead = 0;
+        for (int s = 0; s < kGemmBarriers; ++s) {
+            const bool acc_empty = s >= 2 * kGemmStages + kAccBuffers && s < 2 * kGemmStages + 2 * kAccBuffers;
+            mbar_init(bars + s, acc_empty ? kEpiWarps : 1);  // every epilogue warp hands an accumulator back
+        }
+        dead[0] = 0;
+        dead[1] = 0;  // stays 0: the flag the draining waits look at
         mbar_init_fence();
     }
-    if (warp == 1) {  // tensor memory: kBN columns for the 128 x kBN fp32 accumulator
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kBN) : "memory");
+    if (warp == 1) {  // all of this SM's tensor memory: two 128 x kBN fp32 accumulators (one block per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -146,74 +200,112 @@ __global__ void __launch_bounds__(kGemmThreads, 2) mole_gemm_tn_kernel(const __g
     const uint32_t tmem_acc = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {  // ---- producer: tiles of A and B, kGemmStages ahead ----
-            for (int kt = 0; kt < ktiles; ++kt) {
-                const int s = kt % kGemmStages;
-                const uint32_t par = ((kt / kGemmStages) & 1) ^ 1;  // first pass: the stage has never been used
-                if (!bar_wait_bounded(empty0 + s * 8, par, dead)) {
-                    if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
-                    *dead = 1;
-                    break;
+        if (lane == 0) {  // ---- producer: tiles of A and B, kGemmStages ahead, across output tiles ----
+            uint32_t it = 0;  // k-tiles issued by this block so far
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                const TileCoord tc = tile_coord(tile, p);
+                for (int kt = 0; kt < ktiles; ++kt, ++it) {
+                    const uint32_t s = it % kGemmStages;
+                    const uint32_t par = ((it / kGemmStages) & 1u) ^ 1u;  // first pass: the stage has never been used
+                    if (!bar_wait_bounded(empty0 + s * 8, par, dead)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a_dst = tiles + s * kStageBytes, b_dst = a_dst + kTileBytesA;
+                    mbar_expect_tx(bars + s, kStageBytes);
+                    tma_load_3d(a_dst, &map_a, kt * kBK, tc.m0, tc.z, full0 + s * 8);
+                    tma_load_3d(b_dst, &map_b, kt * kBK, tc.n0, tc.z, full0 + s * 8);
                 }
-                const uint32_t a_dst = tiles + s * 2 * kTileBytes, b_dst = a_dst + kTileBytes;
-                mbar_expect_tx(bars + s, 2 * kTileBytes);
-                tma_load_3d(a_dst, &map_a, kt * kBK, m0, z, full0 + s * 8);
-                tma_load_3d(b_dst, &map_b, kt * kBK, n0, z, full0 + s * 8);
+            }
+            if (!ok) {
+                if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+                *dead = 1;
+                // the copies already issued land in this block's shared memory: let them, before the block can exit
+                const uint32_t first = it > static_cast<uint32_t>(kGemmStages) ? it - kGemmStages : 0u;
+                for (uint32_t j = first; j < it; ++j)
+                    (void)bar_wait_bounded(full0 + (j % kGemmStages) * 8, (j / kGemmStages) & 1u, dead + 1, kDrainPolls);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {  // ---- tensor-core issue ----
             const uint32_t idesc = umma_idesc();
+            uint32_t it = 0, t = 0;  // k-tiles and output tiles consumed by this block so far
             bool ok = true;
-            for (int kt = 0; kt < ktiles && ok; ++kt) {
-                const int s = kt % kGemmStages;
-                ok = bar_wait_bounded(full0 + s * 8, (kt / kGemmStages) & 1, dead);
+            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++t) {
+                const uint32_t b = t & 1u;
+                // the epilogue warps have read this accumulator's previous tile out
+                ok = bar_wait_bounded(acc_empty0 + b * 8, ((t >> 1) & 1u) ^ 1u, dead);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_src = tiles + s * 2 * kTileBytes, b_src = a_src + kTileBytes;
-                const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+                const uint32_t acc = tmem_acc + b * kBN;
+                for (int kt = 0; kt < ktiles; ++kt, ++it) {
+                    const uint32_t s = it % kGemmStages;
+                    ok = bar_wait_bounded(full0 + s * 8, (it / kGemmStages) & 1u, dead);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_src = tiles + s * kStageBytes, b_src = a_src + kTileBytesA;
+                    const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes along K inside the swizzle span: +2 in 16-byte units
-                    umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
-                umma_commit(empty0 + s * 8);  // the stage is free once these have read it
+                    for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes along K inside the swizzle span: +2 in 16-byte units
+                        umma_bf16(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(empty0 + s * 8);  // the stage is free once these have read it
+                }
+                if (ok) umma_commit(acc_full0 + b * 8);
             }
-            if (ok) {
-                umma_commit(accum_bar);
-            } else {
+            if (!ok) {
                 if (!*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
                 *dead = 1;
+                umma_commit(drain_bar);  // whatever was issued finishes reading shared memory before the block exits
+                (void)bar_wait_bounded(drain_bar, 0, dead + 1, kDrainPolls);
             }
         }
     } else {
         // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread; the two warps
-        // that share a lane quarter take half of the columns each ----
-        const bool ok = bar_wait_bounded(accum_bar, 0, dead);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            const int quarter = warp & 3;
-            const int row = m0 + quarter * 32 + lane;
-            __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(p.c) + static_cast<long long>(z) * p.c_z_stride +
-                                  static_cast<long long>(row) * p.c_row_stride + n0;
-            const int c_begin = (warp - 2) < 4 ? 0 : kBN / 64, c_end = c_begin + kBN / 64;
-#pragma unroll 1
-            for (int c = c_begin; c < c_end; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(c * 32), r);
+        // that share a lane quarter take half of the tile's columns each, 32 at a time ----
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        constexpr int kChunks = kBN / 64;  // per warp
+        uint32_t t = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++t) {
+            const uint32_t b = t & 1u;
+            ok = bar_wait_bounded(acc_full0 + b * 8, (t >> 1) & 1u, dead);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const TileCoord tc = tile_coord(tile, p);
+            const int row = tc.m0 + quarter * 32 + lane;
+            const int ncol0 = tc.n0 + half * (kBN / 2);
+            __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(p.c) + static_cast<long long>(tc.z) * p.c_z_stride +
+                                  static_cast<long long>(row) * p.c_row_stride + ncol0;
+            const uint32_t tsrc = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + b * kBN + static_cast<uint32_t>(half * (kBN / 2));
+            uint32_t r[2][32];
+            tmem_ld32(tsrc, r[0]);
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c) {
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (c + 1 < kChunks) {
+                    tmem_ld32(tsrc + static_cast<uint32_t>((c + 1) * 32), r[(c + 1) & 1]);
+                } else {
+                    // this warp's part of the accumulator is in registers: hand the buffer back to the tensor cores
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) bar_arrive(acc_empty0 + b * 8);
+                }
                 if (row < p.M) {
                     // 32 consecutive columns of this thread's row: round in pairs, store 16 bytes (8 columns) at a time
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        float x0 = __uint_as_float(r[i]), x1 = __uint_as_float(r[i + 1]);
-                        if (p.gelu) {
-                            x0 = 0.5f * x0 * (1.0f + erff(x0 * 0.70710678118654752440f));
-                            x1 = 0.5f * x1 * (1.0f + erff(x1 * 0.70710678118654752440f));
+                        float x0 = __uint_as_float(r[c & 1][i]), x1 = __uint_as_float(r[c & 1][i + 1]);
+                        if (GELU) {
+                            x0 = gelu_erf(x0);
+                            x1 = gelu_erf(x1);
                         }
-                        const __nv_bfloat162 b = __floats2bfloat162_rn(x0, x1);
-                        packed[i / 2] = *reinterpret_cast<const uint32_t *>(&b);
+                        const __nv_bfloat162 v = __floats2bfloat162_rn(x0, x1);
+                        packed[i / 2] = *reinterpret_cast<const uint32_t *>(&v);
                     }
-                    const int col0 = n0 + c * 32;
+                    const int col0 = ncol0 + c * 32;
                     if (col0 + 32 <= p.N) {
 #pragma unroll
                         for (int v = 0; v < 4; ++v)
@@ -227,15 +319,15 @@ __global__ void __launch_bounds__(kGemmThreads, 2) mole_gemm_tn_kernel(const __g
                     }
                 }
             }
-        } else if (lane == 0 && !*dead && p.status) {
-            atomicOr(p.status, MOLE_STATUS_TIMEOUT);
         }
+        if (!ok && lane == 0 && !*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
+        if (!ok && lane == 0) *dead = 1;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kBN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -281,13 +373,13 @@ static EncodeTiledFn encode_tiled()
 
 // K-major bf16 operand [z][rows][k]: rows row_stride elements apart, z slices z_stride elements apart
 static int make_operand_map(CUtensorMap *map, const void *base, long long k, long long rows, long long zs, long long row_stride,
-                            long long z_stride)
+                            long long z_stride, int box_rows)
 {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return MOLE_ERR_CUDA;
     const cuuint64_t dims[3] = {static_cast<cuuint64_t>(k), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(zs)};
     const cuuint64_t strides[2] = {static_cast<cuuint64_t>(row_stride) * 2, static_cast<cuuint64_t>(z_stride) * 2};
-    const cuuint32_t box[3] = {kBK, kBM, 1};
+    const cuuint32_t box[3] = {kBK, static_cast<cuuint32_t>(box_rows), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -301,11 +393,15 @@ static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stri
                        uint32_t *status, cudaStream_t st)
 {
     CUtensorMap map_a, map_b;
-    int rc = make_operand_map(&map_a, a, K, M, Z, a_row_stride, a_z_stride);
+    int rc = make_operand_map(&map_a, a, K, M, Z, a_row_stride, a_z_stride, kBM);
     if (rc != MOLE_OK) return rc;
-    rc = make_operand_map(&map_b, b, K, N, Z, b_row_stride, b_z_stride);
+    rc = make_operand_map(&map_b, b, K, N, Z, b_row_stride, b_z_stride, kBN);
     if (rc != MOLE_OK) return rc;
-    rc = ensure_smem_opt_in(reinterpret_cast<const void *>(mole_gemm_tn_kernel), static_cast<int>(kGemmSmem));
+    const void *fn = gelu ? reinterpret_cast<const void *>(mole_gemm_tn_kernel<1>) : reinterpret_cast<const void *>(mole_gemm_tn_kernel<0>);
+    rc = ensure_smem_opt_in(fn, static_cast<int>(kGemmSmem));
+    if (rc != MOLE_OK) return rc;
+    int sms = 0;
+    rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
     GemmParams p;
     p.c = c;
@@ -314,10 +410,17 @@ static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stri
     p.M = M;
     p.N = N;
     p.K = K;
-    p.gelu = gelu;
+    p.m_tiles = (M + kBM - 1) / kBM;
+    p.n_tiles = (N + kBN - 1) / kBN;
+    const long long total = static_cast<long long>(p.m_tiles) * p.n_tiles * Z;
+    if (total > 0x7fffffffLL) return MOLE_ERR_TOO_LARGE;
+    p.total_tiles = static_cast<int>(total);
     p.status = status;
-    dim3 grid(static_cast<unsigned>((M + kBM - 1) / kBM), static_cast<unsigned>((N + kBN - 1) / kBN), static_cast<unsigned>(Z));
-    mole_gemm_tn_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
+    const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);  // persistent: one block per SM
+    if (gelu)
+        mole_gemm_tn_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
+    else
+        mole_gemm_tn_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
     MOLE_CUDA_TRY(cudaGetLastError());
     return MOLE_OK;
 }

@@ -73,6 +73,7 @@ int launch_step(const StepLaunch &a);
 
 // kernels that need more than 48 KB of dynamic shared memory opt in once per device
 int ensure_smem_opt_in(const void *fn, int smem);
+int sm_count(int *out, int *dev_out = nullptr);  // SM count of the current device, asked once per device
 // poll limit of the bounded device-side waits (the default unless a debugging variable shortens it)
 uint32_t current_wait_polls();
 

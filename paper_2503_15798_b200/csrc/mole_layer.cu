@@ -293,17 +293,23 @@ static Variant pick_norm_kernel(int dtype, int n_fast, int lanes)
     if (lanes == 2) { MOLE_PICK_N_F32(2, 0, 1) }
     MOLE_PICK_N_F32(1, 0, 1)
 }
-// ... and, for the single-layer launches of the paper's three layer widths, with the sizes compiled in
+// ... and, for the paper's three layer widths, with the sizes compiled in (single layers and fused steps)
 static Variant pick_norm_shape_kernel(const StepPlan &plan, int dtype, int d, bool direct)
 {
     if (dtype != MOLE_DTYPE_BF16) return kNoVariant;
-    if (plan.n_fast == 16 && plan.lanes == 1 && plan.d_split == 1 && !plan.wr_in_ring) {
-        if (d == 768 && plan.consumers == 96) return direct ? MOLE_VB(16, 1, 2, 1, 1, 1) : MOLE_VB(16, 1, 2, 1, 0, 1);
-        if (d == 1024 && plan.consumers == 128) return direct ? MOLE_VB(16, 1, 2, 2, 1, 1) : MOLE_VB(16, 1, 2, 2, 0, 1);
+    if (plan.n_fast == 16 && plan.lanes == 1 && plan.d_split == 1) {
+        if (!plan.wr_in_ring) {
+            if (d == 768 && plan.consumers == 96) return direct ? MOLE_VB(16, 1, 2, 1, 1, 1) : MOLE_VB(16, 1, 2, 1, 0, 1);
+            if (d == 1024 && plan.consumers == 128) return direct ? MOLE_VB(16, 1, 2, 2, 1, 1) : MOLE_VB(16, 1, 2, 2, 0, 1);
+        } else {
+            if (d == 768 && plan.consumers == 96) return MOLE_VB(16, 1, 1, 1, 0, 1);
+            if (d == 1024 && plan.consumers == 128) return MOLE_VB(16, 1, 1, 2, 0, 1);
+        }
     }
-    if (plan.n_fast == 32 && plan.lanes == 2 && plan.d_split == 4 && d == 2048 && plan.dc == 512 && plan.consumers == 128 &&
-        plan.rows_by_expert)
-        return MOLE_VB(32, 2, 3, 3, 0, 1);
+    if (plan.n_fast == 32 && plan.lanes == 2 && d == 2048 && plan.consumers == 128 && plan.rows_by_expert) {
+        if (plan.d_split == 4 && plan.dc == 512) return MOLE_VB(32, 2, 3, 3, 0, 1);
+        if (plan.d_split == 2 && plan.dc == 1024) return MOLE_VB(32, 2, 3, 4, 0, 1);
+    }
     return kNoVariant;
 }
 
@@ -442,7 +448,7 @@ int ensure_smem_opt_in(const void *fn, int smem)
 }
 
 // SM count of the current device, asked once per device.
-static int sm_count(int *out, int *dev_out = nullptr)
+int sm_count(int *out, int *dev_out)
 {
     static std::atomic<int> cache[64];
     int dev = 0;
@@ -546,7 +552,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     const bool direct = M >= 128 && M <= 4LL * sms;  // see pick_kernel
     Variant v = kNoVariant;
     if (norm) {
-        if (L == 1) v = pick_norm_shape_kernel(plan, dtype, d, direct);
+        v = pick_norm_shape_kernel(plan, dtype, d, direct && L == 1);
         if (!v.fn) {
             rc = plan_step(M, L, N, d, dtype, d_split, &plan, true, sms, true);  // the general kernels cut the rows by columns
             if (rc != MOLE_OK) return rc;

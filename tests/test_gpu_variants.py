@@ -35,7 +35,6 @@ CASES = {
     "step<bf16,16,1,2,1,0,1>": [(700, 16, 768, 1, True, AUTO)],
     "step<bf16,16,1,2,2,1,1>": [(256, 16, 1024, 1, True, AUTO)],
     "step<bf16,16,1,2,2,0,1>": [(2500, 16, 1024, 1, True, AUTO)],
-    "step<bf16,32,2,3,3,0,1>": [(256, 32, 2048, 1, True, AUTO)],
     # fused steps: the decode arithmetic with a ring (default) ...
     "fstep<16,1,0>": [(256, 16, 768, 3, False, DEC), (64, 16, 768, 12, False, DEC), (256, 16, 1024, 3, False, DEC),
                       (8, 16, 1024, 8, False, DEC), (1, 16, 768, 12, False, DEC), (700, 16, 768, 2, False, DEC)],
@@ -50,11 +49,15 @@ CASES = {
     # ... and the ring kernel's own fused form (on request; the offload step's groups)
     "step<bf16,16,1,1,1,0,0>": [(256, 16, 768, 3, False, AUTO), (64, 16, 768, 12, False, AUTO)],
     "step<bf16,16,1,1,2,0,0>": [(256, 16, 1024, 3, False, AUTO), (64, 16, 1024, 4, False, AUTO), (8, 16, 1024, 8, False, AUTO)],
-    "step<bf16,16,1,0,0,0,1>": [(256, 16, 768, 3, True, AUTO), (64, 16, 1024, 2, True, AUTO)],
+    "step<bf16,16,1,1,1,0,1>": [(256, 16, 768, 3, True, AUTO), (8, 16, 768, 12, True, AUTO)],
+    "step<bf16,16,1,1,2,0,1>": [(256, 16, 1024, 3, True, AUTO), (64, 16, 1024, 2, True, AUTO)],
+    "step<bf16,16,1,0,0,0,1>": [(256, 16, 1536, 3, True, AUTO), (64, 16, 1536, 2, True, AUTO)],
     "step<bf16,32,2,3,3,0,0>": [(256, 32, 2048, 1, False, AUTO), (256, 32, 2048, 3, False, AUTO)],
     "step<bf16,32,2,3,4,0,0>": [(64, 32, 2048, 1, False, AUTO), (64, 32, 2048, 3, False, AUTO), (148, 32, 2048, 2, False, AUTO)],
-    "step<bf16,32,1,0,0,0,1>": [(16, 32, 2048, 1, True, AUTO), (16, 32, 2048, 2, True, AUTO)],
-    "step<bf16,32,2,0,0,0,1>": [(256, 32, 2048, 2, True, AUTO)],
+    "step<bf16,32,2,3,3,0,1>": [(256, 32, 2048, 1, True, AUTO), (256, 32, 2048, 2, True, AUTO)],
+    "step<bf16,32,2,3,4,0,1>": [(16, 32, 2048, 1, True, AUTO), (64, 32, 2048, 2, True, AUTO)],
+    "step<bf16,32,1,0,0,0,1>": [(16, 32, 1024, 2, True, AUTO)],
+    "step<bf16,32,2,0,0,0,1>": [(256, 32, 4096, 2, True, AUTO)],
 }
 FLAT = [(name,) + c for name, cs in CASES.items() for c in cs]
 
