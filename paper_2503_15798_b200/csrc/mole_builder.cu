@@ -36,14 +36,13 @@ constexpr int kEpiWarps = 8;
 constexpr int kGemmThreads = (2 + kEpiWarps) * 32;     // producer warp, MMA warp, eight epilogue warps
 constexpr int kRasterRows = 8;                         // tile rows walked together
 constexpr int kGemmBarriers = 2 * kGemmStages + 2 * kAccBuffers + 1;
-constexpr uint32_t kGemmSmem = kGemmStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kStoreBytes = 32 * 128;                  // an epilogue warp's staging tile: 32 rows x 64 bf16, 128-byte swizzle
+constexpr uint32_t kGemmSmem = kGemmStages * kStageBytes + kEpiWarps * kStoreBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+static_assert(kGemmSmem <= 232448, "one block's shared memory");
 constexpr uint32_t kGemmWaitPolls = 1u << 22;
-static_assert(kTmemCols == 512 && kGemmBarriers * 8 <= 128, "tensor-memory columns are a power of two; barriers fit their block");
+static_assert(kTmemCols == 512 && kGemmBarriers * 8 <= 128 && kEpiWarps % 4 == 0 && kBN % (8 * kEpiWarps) == 0, "tensor-memory columns are a power of two; barriers fit their block");
 
 struct GemmParams {
-    void *c;                // bf16 output
-    long long c_row_stride; // elements between rows of C
-    long long c_z_stride;   // elements between the z slices of C
     int M, N, K;            // per z slice
     int m_tiles, n_tiles;   // per z slice
     int total_tiles;        // over all z slices
@@ -57,6 +56,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(smem_dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
                  : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t smem_src, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_src)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -128,21 +138,44 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr));
 }
 
-// GELU(x) = x Phi(x) with Phi through erfc(|x| / sqrt 2) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-x^2 / 2),
-// t = 1 / (1 + p |x| / sqrt 2) (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7 on erf): within 3.5e-7 of the exact
-// GELU everywhere, a fraction of the bf16 rounding that follows, at about half the instructions of erff().
-__device__ __forceinline__ float gelu_erf(float x)
+// GELU(x) = x Phi(x) = max(x, 0) - |x| erfc(|x| / sqrt 2) / 2, with
+// erfc(u) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-u^2), t = 1 / (1 + p u)
+// (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7): within 4e-7 of the exact GELU everywhere, a fraction of the
+// bf16 rounding that follows.  Two elements at a time on the packed fp32 pipe; about a third of the
+// instructions of erff().
+__device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float rcp_approx(float v)
 {
-    const float au = fabsf(x) * 0.70710678118654752440f;
-    const float t = __fdividef(1.0f, fmaf(0.3275911f, au, 1.0f));
-    float poly = fmaf(1.061405429f, t, -1.453152027f);
-    poly = fmaf(poly, t, 1.421413741f);
-    poly = fmaf(poly, t, -0.284496736f);
-    poly = fmaf(poly, t, 0.254829592f);
-    float e;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"((x * x) * -0.72134752044448170368f));  // exp(-x^2 / 2)
-    const float erfc_au = poly * t * e;
-    return fmaxf(x, 0.0f) - fabsf(0.5f * x * erfc_au);  // x >= 0: x - x erfc / 2;  x < 0: x erfc / 2
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float ex2_approx(float v)
+{
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float2 gelu_erf2(float2 x)
+{
+    constexpr float kP = 0.3275911f * 0.70710678118654752440f;  // p / sqrt 2
+    float2 t;
+    t.x = rcp_approx(fmaf(fabsf(x.x), kP, 1.0f));
+    t.y = rcp_approx(fmaf(fabsf(x.y), kP, 1.0f));
+    float2 poly = __ffma2_rn(splat(0.5f * 1.061405429f), t, splat(0.5f * -1.453152027f));  // a_i / 2
+    poly = __ffma2_rn(poly, t, splat(0.5f * 1.421413741f));
+    poly = __ffma2_rn(poly, t, splat(0.5f * -0.284496736f));
+    poly = __ffma2_rn(poly, t, splat(0.5f * 0.254829592f));
+    poly = __fmul2_rn(poly, t);
+    const float2 arg = __fmul2_rn(__fmul2_rn(x, splat(-0.72134752044448170368f)), x);  // -x^2 / 2 in powers of two
+    float2 e;
+    e.x = ex2_approx(arg.x);
+    e.y = ex2_approx(arg.y);
+    const float2 h = __fmul2_rn(poly, e);  // erfc(|x| / sqrt 2) / 2
+    float2 g;
+    g.x = fmaf(-fabsf(x.x), h.x, fmaxf(x.x, 0.0f));
+    g.y = fmaf(-fabsf(x.y), h.y, fmaxf(x.y, 0.0f));
+    return g;
 }
 
 struct TileCoord {
@@ -166,12 +199,14 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, const GemmParams &p)
 
 template <int GELU>
 __global__ void __launch_bounds__(kGemmThreads, 1) mole_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                                    const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+                                                                    const __grid_constant__ CUtensorMap map_b,
+                                                                    const __grid_constant__ CUtensorMap map_c, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
-    unsigned char *ctl = smem_raw + (tiles - raw) + kGemmStages * kStageBytes;
+    const uint32_t staging = tiles + kGemmStages * kStageBytes;
+    unsigned char *ctl = smem_raw + (tiles - raw) + kGemmStages * kStageBytes + kEpiWarps * kStoreBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(ctl);  // full[stages], empty[stages], acc_full[2], acc_empty[2], drain
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(ctl + 128);
     volatile int *dead = reinterpret_cast<volatile int *>(tmem_slot + 1);
@@ -261,11 +296,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mole_gemm_tn_kernel(const __g
             }
         }
     } else {
-        // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread; the two warps
-        // that share a lane quarter take half of the tile's columns each, 32 at a time ----
+        // ---- epilogue: warp w reads tensor-memory lanes 32 (w % 4) .., one output row per thread; the warps
+        // that share a lane quarter take an equal part of the tile's columns each, 32 at a time.  The rounded
+        // values go through a staging tile in shared memory (32 rows x 64 columns, 128-byte swizzle: the eight
+        // lanes of a store phase hit eight different 16-byte columns) and leave with one bulk tensor store per
+        // 64 columns: whole 128-byte lines, clipped to the matrix by the copy engine ----
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;
-        constexpr int kChunks = kBN / 64;  // per warp
+        const int part = (warp - 2) >> 2;
+        constexpr int kColsPerWarp = kBN / (kEpiWarps / 4);
+        constexpr int kChunks = kColsPerWarp / 32;
+        static_assert(kChunks % 2 == 0, "a staging tile is two chunks wide");
+        const uint32_t stage_row = staging + static_cast<uint32_t>((warp - 2) * kStoreBytes + lane * 128);
         uint32_t t = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++t) {
@@ -274,11 +315,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mole_gemm_tn_kernel(const __g
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const TileCoord tc = tile_coord(tile, p);
-            const int row = tc.m0 + quarter * 32 + lane;
-            const int ncol0 = tc.n0 + half * (kBN / 2);
-            __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(p.c) + static_cast<long long>(tc.z) * p.c_z_stride +
-                                  static_cast<long long>(row) * p.c_row_stride + ncol0;
-            const uint32_t tsrc = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + b * kBN + static_cast<uint32_t>(half * (kBN / 2));
+            const int row0 = tc.m0 + quarter * 32;
+            const int ncol0 = tc.n0 + part * kColsPerWarp;
+            const uint32_t tsrc = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + b * kBN + static_cast<uint32_t>(part * kColsPerWarp);
             uint32_t r[2][32];
             tmem_ld32(tsrc, r[0]);
 #pragma unroll
@@ -292,34 +331,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mole_gemm_tn_kernel(const __g
                     __syncwarp();
                     if (lane == 0) bar_arrive(acc_empty0 + b * 8);
                 }
-                if (row < p.M) {
-                    // 32 consecutive columns of this thread's row: round in pairs, store 16 bytes (8 columns) at a time
-                    uint32_t packed[16];
+                uint32_t packed[16];  // 32 consecutive columns of this thread's row, rounded in pairs
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float x0 = __uint_as_float(r[c & 1][i]), x1 = __uint_as_float(r[c & 1][i + 1]);
-                        if (GELU) {
-                            x0 = gelu_erf(x0);
-                            x1 = gelu_erf(x1);
-                        }
-                        const __nv_bfloat162 v = __floats2bfloat162_rn(x0, x1);
-                        packed[i / 2] = *reinterpret_cast<const uint32_t *>(&v);
-                    }
-                    const int col0 = ncol0 + c * 32;
-                    if (col0 + 32 <= p.N) {
+                for (int i = 0; i < 32; i += 2) {
+                    float2 x = make_float2(__uint_as_float(r[c & 1][i]), __uint_as_float(r[c & 1][i + 1]));
+                    if (GELU) x = gelu_erf2(x);
+                    const __nv_bfloat162 v = __floats2bfloat162_rn(x.x, x.y);
+                    packed[i / 2] = *reinterpret_cast<const uint32_t *>(&v);
+                }
+                if ((c & 1) == 0) {  // the staging tile is free once the previous store has read it
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+                }
 #pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            *reinterpret_cast<uint4 *>(crow + c * 32 + v * 8) =
-                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < p.N)
-                                crow[c * 32 + i] = __ushort_as_bfloat16(static_cast<unsigned short>((i & 1) ? (packed[i / 2] >> 16) : (packed[i / 2] & 0xffffu)));
-                    }
+                for (int v = 0; v < 4; ++v)
+                    st_shared_v4(stage_row + static_cast<uint32_t>((((c & 1) * 4 + v) ^ (lane & 7)) * 16), packed[4 * v], packed[4 * v + 1],
+                                 packed[4 * v + 2], packed[4 * v + 3]);
+                if (c & 1) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    const int col0 = ncol0 + (c >> 1) * 64;
+                    if (lane == 0 && row0 < p.M && col0 < p.N) tma_store_3d(&map_c, stage_row, col0, row0, tc.z);
                 }
             }
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // this warp's stores have left shared memory and landed
         if (!ok && lane == 0 && !*dead && p.status) atomicOr(p.status, MOLE_STATUS_TIMEOUT);
         if (!ok && lane == 0) *dead = 1;
     }
@@ -371,9 +407,10 @@ static EncodeTiledFn encode_tiled()
     return fn;
 }
 
-// K-major bf16 operand [z][rows][k]: rows row_stride elements apart, z slices z_stride elements apart
-static int make_operand_map(CUtensorMap *map, const void *base, long long k, long long rows, long long zs, long long row_stride,
-                            long long z_stride, int box_rows)
+// bf16 matrix [z][rows][k], k contiguous: rows row_stride elements apart, z slices z_stride elements apart; tiles of
+// box_rows x 64 elements in the 128-byte swizzle (operands and the output alike)
+static int make_matrix_map(CUtensorMap *map, const void *base, long long k, long long rows, long long zs, long long row_stride,
+                           long long z_stride, int box_rows)
 {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return MOLE_ERR_CUDA;
@@ -392,10 +429,12 @@ static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stri
                        long long b_z_stride, void *c, long long c_row_stride, long long c_z_stride, int M, int N, int K, int Z, int gelu,
                        uint32_t *status, cudaStream_t st)
 {
-    CUtensorMap map_a, map_b;
-    int rc = make_operand_map(&map_a, a, K, M, Z, a_row_stride, a_z_stride, kBM);
+    CUtensorMap map_a, map_b, map_c;
+    int rc = make_matrix_map(&map_a, a, K, M, Z, a_row_stride, a_z_stride, kBM);
     if (rc != MOLE_OK) return rc;
-    rc = make_operand_map(&map_b, b, K, N, Z, b_row_stride, b_z_stride, kBN);
+    rc = make_matrix_map(&map_b, b, K, N, Z, b_row_stride, b_z_stride, kBN);
+    if (rc != MOLE_OK) return rc;
+    rc = make_matrix_map(&map_c, c, N, M, Z, c_row_stride, c_z_stride, 32);
     if (rc != MOLE_OK) return rc;
     const void *fn = gelu ? reinterpret_cast<const void *>(mole_gemm_tn_kernel<1>) : reinterpret_cast<const void *>(mole_gemm_tn_kernel<0>);
     rc = ensure_smem_opt_in(fn, static_cast<int>(kGemmSmem));
@@ -404,9 +443,6 @@ static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stri
     rc = sm_count(&sms);
     if (rc != MOLE_OK) return rc;
     GemmParams p;
-    p.c = c;
-    p.c_row_stride = c_row_stride;
-    p.c_z_stride = c_z_stride;
     p.M = M;
     p.N = N;
     p.K = K;
@@ -418,9 +454,9 @@ static int launch_gemm(const void *a, long long a_row_stride, long long a_z_stri
     p.status = status;
     const unsigned grid = static_cast<unsigned>(total < sms ? total : sms);  // persistent: one block per SM
     if (gelu)
-        mole_gemm_tn_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
+        mole_gemm_tn_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, map_c, p);
     else
-        mole_gemm_tn_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p);
+        mole_gemm_tn_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, map_c, p);
     MOLE_CUDA_TRY(cudaGetLastError());
     return MOLE_OK;
 }
