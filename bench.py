@@ -107,6 +107,7 @@ def timed_launch_shapes():
                 add(f"{name} batch {M} chained{tag}", M, sh, 1, norm)
                 if M <= 4096:
                     add(f"{name} batch {M} fused{tag}", M, sh, sh.L, norm)
+            add(f"{name} batch {M} chained, ring kernel", M, sh, 1, kernel=1)
             for L in (1, sh.L):
                 if (L == 1 or M <= 4096) and decode_family_covers(M, sh, L):
                     add(f"{name} batch {M} {'chained' if L == 1 else 'fused'}, one block per token", M, sh, L, kernel=2)
@@ -468,6 +469,8 @@ def config_rows(torch, mole, inputs, sh, L, luts, wrs, batches, steps, warmup, p
         modes = [("chained", mole.STEP_CHAINED, mole.KERNEL_AUTO, None)]
         if decode_family_covers(m, sh, 1):
             modes.append(("chained_one_block_per_token", mole.STEP_CHAINED, mole.KERNEL_DECODE, None))
+        if not mole.variant(m, sh.N, sh.d)[0].startswith("step"):  # the library's own choice is not the ring kernel: time that too
+            modes.append(("chained_ring", mole.STEP_CHAINED, mole.KERNEL_RING, None))
         if m <= 4096:
             modes.append(("fused", mole.STEP_FUSED, mole.KERNEL_AUTO, None))
             if decode_family_covers(m, sh, L):
@@ -570,9 +573,11 @@ def builder_row(torch, mole, inputs, dev, vocab=0):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     mole.build_lut(E, W1, W2, out=lut, status=status)  # allocates its scratch buffer through torch; synchronises
     times = []
-    for _ in range(3):
-        torch.cuda.synchronize()
-        times.append(event_ms(torch, lambda: mole.build_lut(E, W1, W2, out=lut, status=status)))
+    clocks = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))), period_s=0.002)
+    with clocks:
+        for _ in range(20):  # each build timed by itself (a burst, like the GEMM rate it is compared with)
+            torch.cuda.synchronize()
+            times.append(event_ms(torch, lambda: mole.build_lut(E, W1, W2, out=lut, status=status)))
     assert int(status.item()) == 0
     ms = statistics.median(times)
     flops = 2 * 2.0 * sh.V * sh.d * D * sh.N
@@ -581,7 +586,8 @@ def builder_row(torch, mole, inputs, dev, vocab=0):
     return {"V": sh.V, "d": sh.d, "D": D, "N": sh.N, "ms_per_layer": ms, "flops_per_layer": flops, "TFLOPps": tf,
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
                          "kernel": "mole_gemm_tn_kernel", "peak_source": src},
-            "table_rows_per_s": sh.V / (ms * 1e-3)}
+            "table_rows_per_s": sh.V / (ms * 1e-3), "ms_min": min(times), "ms_max": max(times), "builds_timed": len(times),
+            "clocks": clocks.summary()}
 
 
 def run_mole(args):
@@ -997,10 +1003,10 @@ def run_builder(args):
     torch.cuda.set_device(0)
     row = builder_row(torch, mole, inputs, torch.device("cuda", 0), args.vocab)
     line = {"metric": "MoLE table builder (Eq. 6-7) TFLOP/s, one 160M-shaped layer", "value": row["TFLOPps"], "unit": "TFLOP/s",
-            "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": row["ms_per_layer"], "higher_is_better": True, "scaling": "weak",
+            "n_gpus": 1, "steps": row["builds_timed"], "warmup": 1, "ms_per_step": row["ms_per_layer"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"re-parameterisation of one layer: V={row['V']}, d={row['d']}, D={row['D']}, N={row['N']}"},
-            "gpu_launches": 6, "roofline": row["roofline"], "builder": row}
+            "gpu_launches": 2 * row["builds_timed"], "roofline": row["roofline"], "clocks": row["clocks"], "builder": row}
     print(json.dumps(line), flush=True)
 
 

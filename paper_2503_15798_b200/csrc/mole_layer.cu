@@ -7,6 +7,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include "mole_cdecode.cuh"
 #include "mole_decode.cuh"
 #include "mole_fstep.cuh"
 #include "mole_kernel.cuh"
@@ -336,6 +337,27 @@ static DecodeVariant pick_decode(int N, bool norm)
     }
 }
 
+// The one-token-per-cluster kernel (mole_cdecode.cuh): bf16, d = 2048 (four blocks of 512 columns), N of 16 or 32,
+// a single layer with the plain router, the launch's own chunking.
+constexpr int kClusterBlocks = 4;
+static bool cdecode_shape_ok(int dtype, int N, int d, bool norm)
+{
+    return dtype == MOLE_DTYPE_BF16 && !norm && (N == 16 || N == 32) && d == kClusterBlocks * kClusterSlice;
+}
+// Measured on B200 (1B-shaped layers, chained steps): the cluster kernel is ahead of the ring kernel while all of a
+// launch's blocks (four per SM) are resident at once with room left for the next layer's blocks to prefetch under
+// them -- up to 128 tokens on 148 SMs -- and behind it from there on (a second wave of blocks cannot prefetch).
+static bool cdecode_preferred(long long M, int N, int sms)
+{
+    return N == 32 && M * kClusterBlocks * 8 <= 4LL * sms * 7;
+}
+static DecodeVariant pick_cdecode(int N)
+{
+    if (N == 32) return DecodeVariant{mole_cdecode_kernel<32, kClusterBlocks>, "cdecode<32,4>"};
+    if (N == 16) return DecodeVariant{mole_cdecode_kernel<16, kClusterBlocks>, "cdecode<16,4>"};
+    return DecodeVariant{nullptr, "none"};
+}
+
 // The fused step with the decode arithmetic (mole_fstep.cuh): bf16, N of 4, 8, 16 or 32, d a multiple of
 // 128 with d / 4 <= 512 compute threads, router matrix in 1, 2 or 4 column chunks of at most 32 KB, rows in
 // chunks of whole experts of at most 32 KB.
@@ -506,11 +528,13 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     c->decode = c->fstep = false;
     FStepPlan fplan;
     const bool fstep_ok = L > 1 && d_split == 0 && plan_fstep(M, L, N, d, dtype, norm, sms, &fplan);
-    if (kernel == MOLE_KERNEL_DECODE && !(decode_ok || fstep_ok)) return MOLE_ERR_UNSUPPORTED_SHAPE;
-    // MOLE_KERNEL_AUTO takes the ring kernel for plain tables: measured on B200, neither the one-block-per-token
-    // kernel (chained steps) nor the fused step built on it beats it -- a decode batch is bound by the latency of one
-    // token's dependent instruction stream, which the two families execute at about the same length.  They run on
-    // request (MOLE_KERNEL_DECODE), and their structure carries the quantised tables.
+    const bool cdecode_ok = L == 1 && d_split == 0 && cdecode_shape_ok(dtype, N, d, norm);
+    if (kernel == MOLE_KERNEL_DECODE && !(decode_ok || fstep_ok || cdecode_ok)) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    // MOLE_KERNEL_AUTO takes the ring kernel for plain tables, except for the widest layers at up to 128 tokens (the
+    // cluster kernel, see cdecode_preferred): measured on B200, neither the one-block-per-token kernel (chained steps)
+    // nor the fused step built on it beats it -- a decode batch is bound by the latency of one token's dependent
+    // instruction stream, which the two families execute at about the same length.  They run on request
+    // (MOLE_KERNEL_DECODE), and their structure carries the quantised tables.
     if (fstep_ok && kernel == MOLE_KERNEL_DECODE) {
         const FStepVariant v = pick_fstep(N, fplan.db, norm);
         if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
@@ -533,6 +557,20 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
         if (env.blocks_per_sm >= 1 && env.blocks_per_sm < per_sm) per_sm = env.blocks_per_sm;
         c->grid = static_cast<long long>(per_sm) * sms;
         if (c->grid > M) c->grid = M;
+        return MOLE_OK;
+    }
+    if (cdecode_ok && (kernel == MOLE_KERNEL_DECODE || (kernel == MOLE_KERNEL_AUTO && cdecode_preferred(M, N, sms)))) {
+        const DecodeVariant v = pick_cdecode(N);
+        if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
+        c->decode = true;
+        c->plan = plan;
+        c->step_fn = nullptr;
+        c->decode_fn = v.fn;
+        c->name = v.name;
+        c->threads = kClusterThreads;
+        c->smem = static_cast<int>(cdecode_smem_bytes(N));
+        c->grid = M * kClusterBlocks;  // one cluster per token
+        if (prepare) return ensure_smem_opt_in(reinterpret_cast<const void *>(v.fn), c->smem);
         return MOLE_OK;
     }
     if (decode_ok && kernel == MOLE_KERNEL_DECODE) {
@@ -824,7 +862,16 @@ int mole_decode_step_args(const mole_step_args *a)
     if (a->norm_weight_base &&
         (!aligned16(a->norm_weight_base) || (a->norm_layer_stride_bytes & 15) || !(a->norm_eps >= 0.f) || a->norm_eps > 3.0e38f))
         return MOLE_ERR_INVALID_ARG;
-    if (mode == MOLE_STEP_AUTO) mode = (quant || (L > 1 && M > kFusedMaxTokens)) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
+    if (mode == MOLE_STEP_AUTO) {
+        mode = (quant || (L > 1 && M > kFusedMaxTokens)) ? MOLE_STEP_CHAINED : MOLE_STEP_FUSED;
+        // the widest layers at up to 16 tokens: L chained launches of the cluster kernel are ahead of the fused launch
+        // (measured: 2.7 - 3.3 us against 3.5 - 3.65 us per layer); they need the caller's second buffer
+        int sms = kNumSMs;
+        if (mode == MOLE_STEP_FUSED && L > 1 && M <= 16 && a->d_split == 0 && a->kernel == MOLE_KERNEL_AUTO && debug_env(nullptr).kernel <= 0 &&
+            cdecode_shape_ok(a->dtype, a->N, a->d, a->norm_weight_base != nullptr) && sm_count(&sms) == MOLE_OK &&
+            cdecode_preferred(M, a->N, sms) && a->tmp && aligned16(a->tmp) && a->out != a->hidden_in && a->tmp != a->hidden_in && a->tmp != a->out)
+            mode = MOLE_STEP_CHAINED;
+    }
     if (quant) {
         // quantised tables run layer by layer (one block per token de-quantising inside the weighted sum)
         if (mode == MOLE_STEP_FUSED && L > 1) return MOLE_ERR_UNSUPPORTED_SHAPE;

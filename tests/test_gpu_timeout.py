@@ -25,6 +25,7 @@ def _padded_out(M, d):
     (mole.KERNEL_RING, 5, 16, 768),
     (mole.KERNEL_DECODE, 4, 4, 128),   # one block per token: the wait for the router matrix runs out
     (mole.KERNEL_DECODE, 7, 16, 768),
+    (mole.KERNEL_DECODE, 6, 32, 2048),  # one token per cluster: the waits for the router slice and for the peers' partial logits run out
 ])
 def test_a_wait_that_runs_out_reports_timeout_and_the_stream_stays_usable(kernel, M, N, d):
     hidden, ids, lut, wr = rand_case(M, N, d, 40, seed=M + d)
@@ -32,7 +33,7 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_stream_stays_usable(kernel
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     buf, out = _padded_out(M, d)
     name = mole.variant(M, N, d, kernel=kernel)[0]
-    assert name.startswith("decode" if kernel == mole.KERNEL_DECODE else "step")
+    assert name.startswith(("decode", "cdecode") if kernel == mole.KERNEL_DECODE else "step")
     with mole.debug_env(MOLE_DEBUG_WAIT_LIMIT=-1):
         mole.layer_forward(hidden, ids, lut, wr, out, status=status, kernel=kernel)
         torch.cuda.synchronize()  # the launch returns
