@@ -7,8 +7,8 @@
 // grid dependency is waited for, as in mole_decode.cuh), that slice of the hidden state, and the matching
 // 512 x N slice of the router matrix (one bulk copy into its own shared memory).  Each block reduces its
 // slice to N partial logits, PUSHES them into the shared memory of every block of the cluster
-// (st.shared::cluster, then one remote mbarrier arrive per destination with release at cluster scope), waits
-// -- bounded -- until the partials of all CS blocks have arrived, and from there on is the decode kernel again: every warp
+// (st.async: the value and its count at the destination's mbarrier travel together), waits -- bounded -- until
+// the CS x N values addressed to it have landed, and from there on is the decode kernel again: every warp
 // forms the softmax numerators itself and accumulates its rows.  Against a split of the layer over
 // independent blocks, where every block computes all logits by itself, the router matrix crosses from L2
 // into the SMs once per token instead of once per block (a quarter of the bytes at CS = 4, and a quarter of
@@ -17,7 +17,7 @@
 // Nobody reads another block's shared memory, so a block may exit as soon as it has received its partials:
 // by then every push addressed to it has landed and its own pushes are on their way to blocks that are
 // still waiting for them.  The hardware cluster barrier is used once, at the top (arrive) and just before the
-// pushes (wait): a push must not reach a block that has not initialised its barrier yet.  Every thread of
+// first push (wait): a push must not reach a block that has not initialised its barrier yet.  Every thread of
 // every block reaches both unconditionally.
 #pragma once
 
@@ -30,10 +30,11 @@ constexpr int kClusterThreads = kClusterSlice / 4;
 constexpr int kClusterWarps = kClusterThreads / 32;
 constexpr int kClusterMaxBlocks = 8;
 
-// shared memory: the router slice [512][N], per-warp partial logits, the partials of the cluster's blocks, two barriers
+// shared memory: the router slice [512][N], per-warp partial logits, the partials of the cluster's blocks, the
+// per-warp sums of squares, two barriers
 __host__ __device__ inline uint32_t cdecode_smem_bytes(int N)
 {
-    return up128(static_cast<uint32_t>(kClusterSlice) * N * 2) + kClusterWarps * 32 * 4 + kClusterMaxBlocks * 32 * 4 + 32;
+    return up128(static_cast<uint32_t>(kClusterSlice) * N * 2) + kClusterWarps * 32 * 4 + kClusterMaxBlocks * 32 * 4 + kClusterWarps * 4 + 32;
 }
 
 #ifdef __CUDACC__
@@ -53,13 +54,17 @@ __device__ __forceinline__ uint32_t cluster_map(uint32_t local, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void cluster_store_f32(uint32_t remote_addr, float v)
+// one value into another block's shared memory; its four bytes are counted in at that block's barrier when they land
+__device__ __forceinline__ void cluster_push_f32(uint32_t remote_addr, float v, uint32_t remote_bar)
 {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote_addr), "f"(v) : "memory");
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(remote_addr), "f"(v), "r"(remote_bar)
+                 : "memory");
 }
-__device__ __forceinline__ void cluster_arrive_remote(uint32_t remote_bar)
+__device__ __forceinline__ uint4 ldcg_v4(const void *p)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity)
 {
@@ -74,9 +79,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t pa
     return ok != 0;
 }
 
-// N: experts (16 or 32).  CS: blocks per cluster = d / 512.  Launch: grid = tokens x CS blocks of 128 threads,
-// dynamic shared memory cdecode_smem_bytes(N).
-template <int N, int CS>
+// N: experts (16 or 32).  CS: blocks per cluster = d / 512.  NORM: the router reads RMSNorm(hidden) rounded to bf16
+// (App. A.2 listing); every block then reads the whole hidden row for the mean of squares.
+// Launch: grid = tokens x CS blocks of 128 threads, dynamic shared memory cdecode_smem_bytes(N).
+template <int N, int CS, int NORM>
 __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mole_cdecode_kernel(const DecodeParams p)
 {
     using E = Elem<__nv_bfloat16>;
@@ -86,7 +92,7 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
     constexpr int R = N / 2;        // sweep vectors per thread: (512 * N / 8) / 128
     constexpr int T = kClusterThreads;
     static_assert(N == 16 || N == 32, "experts per lane of the exchange");
-    static_assert(CS >= 2 && CS <= kClusterMaxBlocks, "portable cluster sizes");
+    static_assert(CS >= 2 && CS <= kClusterMaxBlocks && CS % 2 == 0, "portable cluster sizes; a hidden row is CS / 2 passes of 16 bytes per thread");
     extern __shared__ __align__(128) unsigned char smem[];
 
     pdl_launch_dependents();
@@ -98,14 +104,16 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
     constexpr uint32_t wr_bytes = static_cast<uint32_t>(kClusterSlice) * N * 2;
     float *partial = reinterpret_cast<float *>(smem + up128(wr_bytes));  // [warps][N]
     float *xch = partial + kClusterWarps * 32;                           // [CS][N]: block c's partial logits
-    uint64_t *bar = reinterpret_cast<uint64_t *>(xch + kClusterMaxBlocks * 32);
+    float *scratch = xch + kClusterMaxBlocks * 32;                       // [warps]
+    uint64_t *bar = reinterpret_cast<uint64_t *>(scratch + kClusterWarps);
     uint64_t *xbar = bar + 1;
 
     // ---- requests that do not depend on the previous kernel ----
     if (tid == 0) {
         mbar_init(bar, 1);
-        mbar_init(xbar, CS);  // one arrival per block of the cluster, after its N values
+        mbar_init(xbar, 1);
         mbar_init_fence();
+        mbar_expect_tx(xbar, CS * N * 4);  // armed for the partial logits of all CS blocks (this block's own included)
         mbar_expect_tx(bar, wr_bytes);
         bulk_g2s(smem, static_cast<const unsigned char *>(p.w_router) + static_cast<size_t>(q) * wr_bytes, wr_bytes, bar);
     }
@@ -121,6 +129,14 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
 #pragma unroll
         for (int j = 0; j < N; ++j) rv[j] = ldg_stream_v2(row + static_cast<size_t>(j) * d * 2);
     }
+    float nw[NORM ? R : 1];
+    if constexpr (NORM) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int col = static_cast<int>(q) * kClusterSlice + (tid + r * T) / QL;
+            nw[r] = bf16_bits_to_float(__ldg(static_cast<const unsigned short *>(p.norm_weight) + col));
+        }
+    }
     __syncthreads();  // the barriers are initialised before anybody in this block polls them
 
     // ---- the previous kernel's output: this block's slice of the token's hidden state (and residual) ----
@@ -133,6 +149,32 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
         hs[r] = ldcg_u16(hrow + 2 * col);
     }
     uint2 res = ldcg_v2((p.residual ? static_cast<const unsigned char *>(p.residual) + static_cast<size_t>(t) * d * 2 : hrow) + own);
+
+    if constexpr (NORM) {
+        // y = (x / sqrt(mean(x^2) + eps)) * w in fp32, rounded once to bf16: what the router reads.  The mean runs over
+        // all d columns: every block reads the whole hidden row (4 KB from L2, 32 bytes per thread) and forms the
+        // sum of squares itself, in the same order in every block -- cheaper than a second exchange.
+        float ss = 0.f;
+#pragma unroll
+        for (int v = 0; v < CS / 2; ++v) {
+            const uint4 hv = ldcg_v4(hrow + (static_cast<size_t>(v) * T + tid) * 16);
+            const uint32_t w4[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = bf16_bits_to_float(w4[i] & 0xffffu), hi = __uint_as_float(w4[i] & 0xffff0000u);
+                ss = fmaf(hi, hi, fmaf(lo, lo, ss));
+            }
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) scratch[warp] = ss;
+        __syncthreads();
+        float total = 0.f;
+#pragma unroll
+        for (int w = 0; w < kClusterWarps; ++w) total += scratch[w];
+        const float rinv = 1.0f / sqrtf(total / static_cast<float>(d) + p.norm_eps);
+#pragma unroll
+        for (int r = 0; r < R; ++r) hs[r] = float_to_bf16_bits((bf16_bits_to_float(hs[r]) * rinv) * nw[r]);
+    }
 
     // ---- router slice in shared memory? (bounded; after a failure the block goes on with whatever is there) ----
     {
@@ -172,17 +214,13 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
 
     // ---- exchange: warp 0 sums the warps' partials (lane j <-> expert j) and pushes the sum to every block ----
     cluster_wait();  // every block of the cluster has initialised its barriers (since long)
-    if (warp == 0) {
-        if (lane < N) {
-            float z = 0.f;
+    if (warp == 0 && lane < N) {
+        float z = 0.f;
 #pragma unroll
-            for (int w = 0; w < kClusterWarps; ++w) z += partial[w * N + lane];
-            const uint32_t slot = smem_u32(xch + q * N + lane);
+        for (int w = 0; w < kClusterWarps; ++w) z += partial[w * N + lane];
+        const uint32_t slot = smem_u32(xch + q * N + lane), xb = smem_u32(xbar);
 #pragma unroll
-            for (int c = 0; c < CS; ++c) cluster_store_f32(cluster_map(slot, c), z);
-        }
-        __syncwarp();  // the lanes' stores are ordered before lane c's arrival with release at cluster scope
-        if (lane < CS) cluster_arrive_remote(cluster_map(smem_u32(xbar), lane));
+        for (int c = 0; c < CS; ++c) cluster_push_f32(cluster_map(slot, c), z, cluster_map(xb, c));
     }
     {
         bool ok = false;

@@ -338,11 +338,11 @@ static DecodeVariant pick_decode(int N, bool norm)
 }
 
 // The one-token-per-cluster kernel (mole_cdecode.cuh): bf16, d = 2048 (four blocks of 512 columns), N of 16 or 32,
-// a single layer with the plain router, the launch's own chunking.
+// a single layer, the launch's own chunking.
 constexpr int kClusterBlocks = 4;
-static bool cdecode_shape_ok(int dtype, int N, int d, bool norm)
+static bool cdecode_shape_ok(int dtype, int N, int d)
 {
-    return dtype == MOLE_DTYPE_BF16 && !norm && (N == 16 || N == 32) && d == kClusterBlocks * kClusterSlice;
+    return dtype == MOLE_DTYPE_BF16 && (N == 16 || N == 32) && d == kClusterBlocks * kClusterSlice;
 }
 // Measured on B200 (1B-shaped layers, chained steps): the cluster kernel is ahead of the ring kernel while all of a
 // launch's blocks (four per SM) are resident at once with room left for the next layer's blocks to prefetch under
@@ -351,10 +351,14 @@ static bool cdecode_preferred(long long M, int N, int sms)
 {
     return N == 32 && M * kClusterBlocks * 8 <= 4LL * sms * 7;
 }
-static DecodeVariant pick_cdecode(int N)
+static DecodeVariant pick_cdecode(int N, bool norm)
 {
-    if (N == 32) return DecodeVariant{mole_cdecode_kernel<32, kClusterBlocks>, "cdecode<32,4>"};
-    if (N == 16) return DecodeVariant{mole_cdecode_kernel<16, kClusterBlocks>, "cdecode<16,4>"};
+    if (N == 32)
+        return norm ? DecodeVariant{mole_cdecode_kernel<32, kClusterBlocks, 1>, "cdecode<32,4,1>"}
+                    : DecodeVariant{mole_cdecode_kernel<32, kClusterBlocks, 0>, "cdecode<32,4,0>"};
+    if (N == 16)
+        return norm ? DecodeVariant{mole_cdecode_kernel<16, kClusterBlocks, 1>, "cdecode<16,4,1>"}
+                    : DecodeVariant{mole_cdecode_kernel<16, kClusterBlocks, 0>, "cdecode<16,4,0>"};
     return DecodeVariant{nullptr, "none"};
 }
 
@@ -528,7 +532,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
     c->decode = c->fstep = false;
     FStepPlan fplan;
     const bool fstep_ok = L > 1 && d_split == 0 && plan_fstep(M, L, N, d, dtype, norm, sms, &fplan);
-    const bool cdecode_ok = L == 1 && d_split == 0 && cdecode_shape_ok(dtype, N, d, norm);
+    const bool cdecode_ok = L == 1 && d_split == 0 && cdecode_shape_ok(dtype, N, d);
     if (kernel == MOLE_KERNEL_DECODE && !(decode_ok || fstep_ok || cdecode_ok)) return MOLE_ERR_UNSUPPORTED_SHAPE;
     // MOLE_KERNEL_AUTO takes the ring kernel for plain tables, except for the widest layers at up to 128 tokens (the
     // cluster kernel, see cdecode_preferred): measured on B200, neither the one-block-per-token kernel (chained steps)
@@ -560,7 +564,7 @@ static int choose_launch(long long M, int L, int N, int d, int dtype, int d_spli
         return MOLE_OK;
     }
     if (cdecode_ok && (kernel == MOLE_KERNEL_DECODE || (kernel == MOLE_KERNEL_AUTO && cdecode_preferred(M, N, sms)))) {
-        const DecodeVariant v = pick_cdecode(N);
+        const DecodeVariant v = pick_cdecode(N, norm);
         if (!v.fn) return MOLE_ERR_UNSUPPORTED_SHAPE;
         c->decode = true;
         c->plan = plan;
@@ -868,7 +872,7 @@ int mole_decode_step_args(const mole_step_args *a)
         // (measured: 2.7 - 3.3 us against 3.5 - 3.65 us per layer); they need the caller's second buffer
         int sms = kNumSMs;
         if (mode == MOLE_STEP_FUSED && L > 1 && M <= 16 && a->d_split == 0 && a->kernel == MOLE_KERNEL_AUTO && debug_env(nullptr).kernel <= 0 &&
-            cdecode_shape_ok(a->dtype, a->N, a->d, a->norm_weight_base != nullptr) && sm_count(&sms) == MOLE_OK &&
+            cdecode_shape_ok(a->dtype, a->N, a->d) && sm_count(&sms) == MOLE_OK &&
             cdecode_preferred(M, a->N, sms) && a->tmp && aligned16(a->tmp) && a->out != a->hidden_in && a->tmp != a->hidden_in && a->tmp != a->out)
             mode = MOLE_STEP_CHAINED;
     }

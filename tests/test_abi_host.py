@@ -51,9 +51,10 @@ def test_variant_names_and_kernel_choice(lib):
     assert V(256, 16, 768, norm=True, kernel=D)[0] == "decode<16,1>" and V(64, 32, 1024, kernel=D)[0] == "decode<32,0>"
     assert V(256, 16, 768, L=12, kernel=D)[0] == "fstep<16,1,0>" and V(64, 32, 2048, L=16, kernel=D)[0] == "fstep<32,2,0>"
     # the widest layers: one token per cluster of four blocks, the library's own choice up to 128 tokens
-    assert V(256, 32, 2048, kernel=D)[:2] == ("cdecode<32,4>", 128) == V(128, 32, 2048)[:2] and V(16, 16, 2048, kernel=D)[0] == "cdecode<16,4>"
+    assert V(256, 32, 2048, kernel=D)[:2] == ("cdecode<32,4,0>", 128) == V(128, 32, 2048)[:2] and V(16, 16, 2048, kernel=D)[0] == "cdecode<16,4,0>"
     assert V(136, 32, 2048)[0].startswith("step<") and V(16, 16, 2048)[0].startswith("step<") and V(16, 32, 2048, kernel=R)[0].startswith("step<")
-    for args, kw in (((256, 32, 4096), {}), ((64, 32, 2048), {"norm": True}), ((64, 5, 768), {}), ((64, 16, 768), {"d_split": 2}), ((64, 4, 64, binding.DTYPE_F32), {})):
+    assert V(64, 32, 2048, norm=True)[0] == "cdecode<32,4,1>"
+    for args, kw in (((256, 32, 4096), {}), ((64, 5, 768), {}), ((64, 16, 768), {"d_split": 2}), ((64, 4, 64, binding.DTYPE_F32), {})):
         with pytest.raises(binding.MoleError) as e:  # shapes the family does not cover
             V(*args, kernel=D, **kw)
         assert e.value.code == binding.ERR_UNSUPPORTED_SHAPE

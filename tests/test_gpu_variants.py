@@ -28,9 +28,11 @@ CASES = {
     "decode<4,0>": [(19, 4, 128, 1, False, DEC)],
     "decode<4,1>": [(19, 4, 2048, 1, True, DEC)],
     # one token per cluster of four blocks (d = 2048)
-    "cdecode<32,4>": [(256, 32, 2048, 1, False, DEC), (16, 32, 2048, 1, False, DEC), (1, 32, 2048, 1, False, DEC),
-                      (333, 32, 2048, 1, False, DEC)],
-    "cdecode<16,4>": [(40, 16, 2048, 1, False, DEC)],
+    "cdecode<32,4,0>": [(256, 32, 2048, 1, False, DEC), (16, 32, 2048, 1, False, DEC), (1, 32, 2048, 1, False, DEC),
+                        (333, 32, 2048, 1, False, DEC)],
+    "cdecode<32,4,1>": [(256, 32, 2048, 1, True, DEC), (16, 32, 2048, 1, True, AUTO), (1, 32, 2048, 1, True, DEC)],
+    "cdecode<16,4,0>": [(40, 16, 2048, 1, False, DEC)],
+    "cdecode<16,4,1>": [(40, 16, 2048, 1, True, DEC)],
     "step<bf16,16,1,2,1,1,0>": [(256, 16, 768, 1, False, AUTO)],
     "step<bf16,16,1,2,1,0,0>": [(64, 16, 768, 1, False, AUTO), (3000, 16, 768, 1, False, AUTO)],
     "step<bf16,16,1,2,2,1,0>": [(256, 16, 1024, 1, False, AUTO)],
@@ -59,7 +61,7 @@ CASES = {
     "step<bf16,32,2,3,3,0,0>": [(256, 32, 2048, 1, False, AUTO), (256, 32, 2048, 3, False, AUTO)],
     "step<bf16,32,2,3,4,0,0>": [(64, 32, 2048, 1, False, RING), (140, 32, 2048, 1, False, AUTO), (64, 32, 2048, 3, False, AUTO), (148, 32, 2048, 2, False, AUTO)],
     "step<bf16,32,2,3,3,0,1>": [(256, 32, 2048, 1, True, AUTO), (256, 32, 2048, 2, True, AUTO)],
-    "step<bf16,32,2,3,4,0,1>": [(16, 32, 2048, 1, True, AUTO), (64, 32, 2048, 2, True, AUTO)],
+    "step<bf16,32,2,3,4,0,1>": [(16, 32, 2048, 1, True, RING), (64, 32, 2048, 2, True, AUTO)],
     "step<bf16,32,1,0,0,0,1>": [(16, 32, 1024, 2, True, AUTO)],
     "step<bf16,32,2,0,0,0,1>": [(256, 32, 4096, 2, True, AUTO)],
 }
@@ -158,23 +160,26 @@ def test_variant_against_the_oracle(name, M, N, d, L, norm, kernel):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("M,N", [(64, 32), (5, 16)])
-def test_cluster_kernel_chained_step(M, N):
+@pytest.mark.parametrize("M,N,norm", [(64, 32, False), (5, 16, False), (9, 32, True)])
+def test_cluster_kernel_chained_step(M, N, norm):
     """L chained launches of the one-token-per-cluster kernel (programmatic dependent launch between them)
     against the oracle's chain."""
     d, L, V = 2048, 3, 61
-    assert mole.variant(M, N, d, kernel=DECODE)[0] == f"cdecode<{N},4>"
+    assert mole.variant(M, N, d, kernel=DECODE, norm=norm)[0] == f"cdecode<{N},4,{int(norm)}>"
     g = torch.Generator().manual_seed(11 * M + N)
     luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16)
     wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16)
     hidden = (1.5 * torch.empty(M, d).normal_(0, 1, generator=g)).to(torch.bfloat16)
     ids = torch.randint(0, V, (M,), generator=g, dtype=torch.int32)
-    ref, _, _ = _oracle_chain(hidden, ids, luts, wrs, None, 0.0)
+    gammas = (1.0 + 0.2 * torch.empty(L, d).normal_(0, 1, generator=g)).to(torch.bfloat16) if norm else None
+    ref, _, _ = _oracle_chain(hidden, ids, luts, wrs, gammas, 1e-5)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     hd = hidden.to(DEV)
     out = mole.decode_step_args(hd, ids.to(DEV), luts.to(DEV), wrs.to(DEV), torch.empty_like(hd), torch.empty_like(hd),
-                                status=status, mode=mole.STEP_CHAINED, kernel=DECODE)
+                                status=status, mode=mole.STEP_CHAINED, kernel=DECODE, norm_weights=gammas.to(DEV) if norm else None,
+                                norm_eps=1e-5)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     err = np.abs(as_f64(out) - ref)
-    assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))).all(), float(err.max())
+    slack = L * 1e-3 * float(luts.abs().max()) * N if norm else 0.0  # a rounding tie in a normalised element moves a gate
+    assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref)) + slack).all(), float(err.max())
