@@ -81,11 +81,14 @@ extern "C" {
                                   written by that previous kernel. */
 
 /* which kernel family runs a single-layer launch (mole_args.kernel, mole_step_args.kernel) */
-#define MOLE_KERNEL_AUTO 0   /* the library's choice */
+#define MOLE_KERNEL_AUTO 0   /* the library's choice: the ring kernel, except d = 2048 with N = 32 at up to 128 tokens (on \
+                                148 SMs), where the one-token-per-cluster kernel of MOLE_KERNEL_DECODE runs */
 #define MOLE_KERNEL_RING 1   /* persistent blocks, rows and router chunks streamed through a shared-memory ring: any shape */
 #define MOLE_KERNEL_DECODE 2 /* one block per token (single layer: rows held in registers; fused step: rows through a ring, \
                                 router matrix through registers): bf16, N of 4, 8, 16 or 32, d a multiple of 128 up to   \
-                                2048 (single layer with N = 32: up to 1024), d_split 0 */
+                                2048 (single layer with N = 32: up to 1024), d_split 0.  A single layer with d = 2048 and \
+                                N of 16 or 32 runs one token per thread-block cluster of four blocks (512 columns each,    \
+                                partial router logits exchanged through distributed shared memory) */
 
 /* storage of a table (mole_args.lut_format): plain elements of `dtype`, or the quantised records of Sec. 4.5 / Table 8 */
 #define MOLE_LUT_PLAIN 0
@@ -93,7 +96,8 @@ extern "C" {
 #define MOLE_LUT_NF3 2 /* 3-bit NormalFloat codes, one float16 absmax scale per block (paper: block 128 -> 19.5 % of FP16) */
 
 /* mole_decode_step_ex mode: how the L layers of a step are launched */
-#define MOLE_STEP_AUTO 0    /* fused unless the batch is large (then chained) */
+#define MOLE_STEP_AUTO 0    /* fused unless the batch is large (then chained); also chained at up to 16 tokens where \
+                               MOLE_KERNEL_AUTO runs the cluster kernel and a tmp buffer was given */
 #define MOLE_STEP_FUSED 1   /* ONE launch: every block walks its tokens through all L layers */
 #define MOLE_STEP_CHAINED 2 /* L launches chained with programmatic dependent launch */
 
