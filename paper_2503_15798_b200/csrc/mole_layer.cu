@@ -179,6 +179,17 @@ int plan_step(long long M, int L, int N, int d, int dtype, int d_split, StepPlan
     const long long blocks = M < cap ? (M > 0 ? M : 1) : cap;
     const long long chunks = ((M + blocks - 1) / blocks) * per_tok * K;
     if (stages > chunks) stages = chunks < 2 ? 2 : static_cast<int>(chunks);
+    // A single layer with its router matrix resident and more tokens than two-slot blocks fit at once, but no more
+    // than one-slot blocks do: one token per block, all of them resident, instead of two tokens in a row per block
+    // (measured, 160M shape, 512 tokens: 4.66 -> 3.80 us per layer).
+    if (L == 1 && !in_ring && K == 1) {
+        auto fit = [&](int s) {
+            int n = kSmemPerSM / (static_cast<int>(total_smem(K, s)) + 1024);
+            const int by_threads = 2048 / (consumers + 32);
+            return n < by_threads ? n : by_threads;
+        };
+        if (M > static_cast<long long>(fit(2)) * sms && M <= static_cast<long long>(fit(1)) * sms) stages = 1;
+    }
     const int forced = env.stages;
     if (forced >= 2 && forced <= kMaxStages && total_smem(K, forced) <= static_cast<uint32_t>(kSmemPerBlockMax)) stages = forced;
     const int hring = (stages + per_tok * K - 1) / (per_tok * K) + 1;

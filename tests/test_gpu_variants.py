@@ -33,9 +33,9 @@ CASES = {
     "cdecode<32,4,1>": [(256, 32, 2048, 1, True, DEC), (16, 32, 2048, 1, True, AUTO), (1, 32, 2048, 1, True, DEC)],
     "cdecode<16,4,0>": [(40, 16, 2048, 1, False, DEC)],
     "cdecode<16,4,1>": [(40, 16, 2048, 1, True, DEC)],
-    "step<bf16,16,1,2,1,1,0>": [(256, 16, 768, 1, False, AUTO)],
+    "step<bf16,16,1,2,1,1,0>": [(256, 16, 768, 1, False, AUTO), (500, 16, 768, 1, False, AUTO)],  # the second: a one-slot ring
     "step<bf16,16,1,2,1,0,0>": [(64, 16, 768, 1, False, AUTO), (3000, 16, 768, 1, False, AUTO)],
-    "step<bf16,16,1,2,2,1,0>": [(256, 16, 1024, 1, False, AUTO)],
+    "step<bf16,16,1,2,2,1,0>": [(256, 16, 1024, 1, False, AUTO), (400, 16, 1024, 1, False, AUTO)],
     "step<bf16,16,1,2,2,0,0>": [(64, 16, 1024, 1, False, AUTO), (2500, 16, 1024, 1, False, AUTO)],
     "step<bf16,16,1,2,1,1,1>": [(256, 16, 768, 1, True, AUTO)],
     "step<bf16,16,1,2,1,0,1>": [(700, 16, 768, 1, True, AUTO)],
