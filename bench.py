@@ -749,8 +749,8 @@ def run_mole(args):
         mole.decode_step_host(h_host, ids_host[k % N_BATCHES], out_host, dev_bufs[0], dev_ids, dev_bufs[1],
                               dev_bufs[2], luts, wrs)
 
-    for k in range(3):  # uncaptured calls first (kernel attributes), then one CUDA graph per id batch:
-        e2e_call(k)     # two host->device copies, the step, one device->host copy
+    for k in range(3):  # uncaptured calls first (kernel attributes), then one CUDA graph per id batch
+        e2e_call(k)
     torch.cuda.synchronize()
     e2e_graphs = []
     for k in range(N_BATCHES):
@@ -768,9 +768,10 @@ def run_mole(args):
     line["e2e"] = {"value": whole_job_tokens_per_s(world, M, e2e_steps, ms_e2e), "unit": UNIT,
                    "h2d_bytes_per_step": M * sh.d * 2 + M * 4, "d2h_bytes_per_step": M * sh.d * 2,
                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps, "repeats": spread_e["repeats"],
-                   "how": "mole_decode_step_host captured into one CUDA graph per id batch: pinned host hidden+ids -> device, "
-                          "the step as mole_decode_step launches it by itself (one fused launch over all layers up to "
-                          "4096 tokens), result -> pinned host; one graph launch and one stream synchronisation per step"}
+                   "how": "mole_decode_step_host captured into one CUDA graph per id batch; the host buffers are pinned and "
+                          "mapped, so the step's one fused launch reads hidden + ids across the host link itself and stores "
+                          "the last layer's output into the host buffer (the same bytes as with staged copies, no copy "
+                          "operations around the kernel); one graph launch and one stream synchronisation per step"}
     e2e_out = out_host.clone()
     del e2e_graphs
 

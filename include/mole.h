@@ -241,9 +241,13 @@ MOLE_API int mole_decode_step_args(const mole_step_args *args);
 
 /*
  * mole_decode_step_host -- mole_decode_step for a caller whose activations live in HOST
- * memory: copies hidden_host and ids_host to the device buffers, runs the L layers, copies
- * the result to out_host, all on `stream` (asynchronous when the host buffers are pinned).
- *   hidden_host, out_host  host [M][d]      ids_host host int32 [M]
+ * memory, all on `stream`.  When the three host buffers are pinned and mapped (cudaHostAlloc,
+ * cudaHostRegister) and the step runs as one launch (L == 1 or up to 4096 tokens), the launch reads
+ * hidden_host and ids_host across the host link itself and stores the last layer's output into
+ * out_host: the device buffers are not touched.  Otherwise hidden_host and ids_host are copied to
+ * the device buffers, the L layers run there, and the result is copied to out_host (asynchronous
+ * when the host buffers are pinned).  The result is the same bits either way.
+ *   hidden_host, out_host  host [M][d] (distinct)      ids_host host int32 [M]
  *   dev_hidden, dev_out, dev_tmp device [M][d] scratch owned by the caller; dev_ids device int32 [M]
  * The result is in out_host once the stream has been synchronised.
  */

@@ -388,19 +388,28 @@ def test_decode_step_fused_in_place_and_bad_ids():
     assert torch.equal(h[7], hidden[7]) and torch.equal(h[31], hidden[31])  # no routed term in any layer
 
 
-def test_decode_step_host_round_trip():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_host_round_trip(pinned):
+    """Pinned, mapped host buffers: the launch reads and writes them itself and leaves the device buffers alone;
+    pageable ones: staged through the device buffers.  The same bits either way."""
     M, N, d, L, V = 64, 16, 768, 4, 300
     g = torch.Generator().manual_seed(5)
     luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16).to(DEV)
     wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
-    h_host = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).pin_memory()
-    ids_host = torch.from_numpy(inputs.zipf_ids(M, V, seed=6)).pin_memory()
-    out_host = torch.empty_like(h_host).pin_memory()
-    dev = [torch.empty(M, d, dtype=torch.bfloat16, device=DEV) for _ in range(3)]
-    dev_ids = torch.empty(M, dtype=torch.int32, device=DEV)
-    mole.decode_step_host(h_host, ids_host, out_host, dev[0], dev_ids, dev[1], dev[2], luts, wrs)
+    h_host = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16)
+    ids_host = torch.from_numpy(inputs.zipf_ids(M, V, seed=6))
+    out_host = torch.empty_like(h_host)
+    if pinned:
+        h_host, ids_host, out_host = h_host.pin_memory(), ids_host.pin_memory(), out_host.pin_memory()
+    dev = [torch.full((M, d), 777.0, dtype=torch.bfloat16, device=DEV) for _ in range(3)]
+    dev_ids = torch.full((M,), -5, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mole.decode_step_host(h_host, ids_host, out_host, dev[0], dev_ids, dev[1], dev[2], luts, wrs, status=status)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0
     want = torch.empty(M, d, dtype=torch.bfloat16, device=DEV)
     mole.decode_step(h_host.to(DEV), ids_host.to(DEV), luts, wrs, want, torch.empty_like(want))
     torch.cuda.synchronize()
     assert torch.equal(out_host, want.cpu())
+    untouched = bool((dev[0] == 777.0).all()) and bool((dev_ids == -5).all())
+    assert untouched == pinned

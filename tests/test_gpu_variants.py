@@ -183,3 +183,25 @@ def test_cluster_kernel_chained_step(M, N, norm):
     err = np.abs(as_f64(out) - ref)
     slack = L * 1e-3 * float(luts.abs().max()) * N if norm else 0.0  # a rounding tie in a normalised element moves a gate
     assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref)) + slack).all(), float(err.max())
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("with_tmp", [True, False])
+def test_step_auto_on_the_widest_layers_at_few_tokens(with_tmp):
+    """mole_decode_step's own choice (MOLE_STEP_AUTO) for d = 2048 at up to 16 tokens: chained launches of the
+    cluster kernel when the caller gave a second buffer, the fused ring launch when not; both against the oracle."""
+    M, N, d, L, V = 8, 32, 2048, 3, 41
+    g = torch.Generator().manual_seed(5)
+    luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16)
+    wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16)
+    hidden = (1.5 * torch.empty(M, d).normal_(0, 1, generator=g)).to(torch.bfloat16)
+    ids = torch.randint(0, V, (M,), generator=g, dtype=torch.int32)
+    ref, _, _ = _oracle_chain(hidden, ids, luts, wrs, None, 0.0)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    hd = hidden.to(DEV)
+    out = mole.decode_step_args(hd, ids.to(DEV), luts.to(DEV), wrs.to(DEV), torch.empty_like(hd),
+                                torch.empty_like(hd) if with_tmp else None, status=status, mode=mole.STEP_AUTO)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    err = np.abs(as_f64(out) - ref)
+    assert (err <= L * 2.0 ** -7 * np.maximum(1.0, np.abs(ref))).all(), float(err.max())
