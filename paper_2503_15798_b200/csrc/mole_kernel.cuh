@@ -497,6 +497,10 @@ __device__ __forceinline__ void rmsnorm_to_shared(uint32_t src, uint32_t dst, co
     using E = Elem<T>;
     constexpr int VEC = E::VEC;
     const int ngrp = d / VEC;
+    const uint4 *wg = static_cast<const uint4 *>(weight_g);
+    // this thread's first vector of the scale comes from L2: asked for before the sum of squares, not after it
+    uint4 w_first = make_uint4(0u, 0u, 0u, 0u);
+    if (tid < ngrp) w_first = __ldg(wg + tid);
     float ss = 0.f;
     for (int g = tid; g < ngrp; g += nc) {
         float x[VEC];
@@ -510,11 +514,10 @@ __device__ __forceinline__ void rmsnorm_to_shared(uint32_t src, uint32_t dst, co
     float total = 0.f;
     for (int w = 0; w < nwarps; ++w) total += scratch[w];  // the same order in every thread
     const float r = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
-    const uint4 *wg = static_cast<const uint4 *>(weight_g);
     for (int g = tid; g < ngrp; g += nc) {
         float x[VEC], w[VEC];
         E::unpack(lds128(src + 16u * g), x);
-        E::unpack(__ldg(wg + g), w);
+        E::unpack(g == tid ? w_first : __ldg(wg + g), w);
         uint32_t o[4];
         if constexpr (VEC == 8) {
 #pragma unroll
