@@ -517,11 +517,16 @@ def isolated_rows(torch, mole, inputs, sh, luts, wrs, batches, peak, dev):
         out = torch.empty_like(hid)
         reps = 100 if m <= 1024 else 20
         res = {}
-        for cold in (False, True):
-            def filler(r):
-                if cold:
-                    flush.fill_(r & 0xFF)
-                else:
+        for mode in ("steady", "cold", "prefetched"):
+            cold = mode != "steady"
+
+            def filler(r, mode=mode):
+                if mode == "steady":
+                    torch.cuda._sleep(20000)
+                    return
+                flush.fill_(r & 0xFF)
+                if mode == "prefetched":  # the step's rows asked for ahead of the layer, then other work (a spin) in between
+                    mole.prefetch_rows(bl[r % N_BATCHES_EXTRA], luts, layers=1)
                     torch.cuda._sleep(20000)
 
             def with_launches():
@@ -537,13 +542,15 @@ def isolated_rows(torch, mole, inputs, sh, luts, wrs, batches, peak, dev):
             torch.cuda.synchronize()
             t1 = min(event_ms(torch, with_launches) for _ in range(3))
             t0 = min(event_ms(torch, without) for _ in range(3))
-            res["cold" if cold else "steady"] = max(t1 - t0, 0.0) * 1e3 / reps
+            res[mode] = max(t1 - t0, 0.0) * 1e3 / reps
         nbytes = sh.layer_bytes(m)
         rows.append({"batch": m, "isolated_steady_us": res["steady"], "isolated_cold_us": res["cold"],
+                     "isolated_cold_prefetched_us": res["prefetched"],
                      "isolated_cold_GBps": nbytes / max(res["cold"], 1e-3) / 1e3,
                      "isolated_cold_frac_of_peak": nbytes / max(res["cold"], 1e-3) / 1e3 / peak,
-                     "how": f"{reps} launches, each after an L2 flush (cold) or a spin (steady), inside one event pair, "
-                            "minus the region without the launches"})
+                     "how": f"{reps} launches, each after an L2 flush (cold), a spin (steady), or an L2 flush followed by "
+                            "mole_prefetch_rows for the launch's ids and a spin (prefetched), inside one event pair, minus the "
+                            "same region without the launches"})
     del flush
     return rows
 

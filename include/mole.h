@@ -257,6 +257,19 @@ MOLE_API int mole_decode_step_host(const void *hidden_host, const int32_t *ids_h
                           int64_t wr_layer_stride_bytes, uint32_t *status, int L, int B, int T, int N, int d,
                           int V, int dtype, void *stream);
 
+/*
+ * mole_prefetch_rows -- ask L2 for the table rows a step will gather, ahead of the layers that gather
+ * them.  The rows of every layer depend only on the input ids (Sec. 3.3: the experts' inputs are
+ * embedding tokens), so a caller whose model runs other work between the lookup layers can issue this
+ * at the start of a step, or a few layers ahead: one L2 prefetch per (token, layer) row of N*d elements,
+ * for `layers` consecutive tables from lut_base on (layer l at + l*lut_layer_stride_bytes).  A hint
+ * only: nothing is written, no result changes, ids outside [0, V) are skipped.  What stays in L2 until
+ * the layer runs is the hardware's business; keep layers * M * row bytes well under the L2 size.
+ *   ids device int32 [M] (int64 with MOLE_FLAG_IDS_INT64); lut_base device, 16-byte aligned.
+ */
+MOLE_API int mole_prefetch_rows(const void *ids, int M, const void *lut_base, int64_t lut_layer_stride_bytes, int layers,
+                                int N, int d, int V, int dtype, uint32_t flags, void *stream);
+
 /* ---------------------------------------------------------------------------------------
  * Quantised tables (Sec. 4.5, Table 8): post-training quantisation of a 16-bit table to the NF4 / NF3
  * NormalFloat types of the QLoRA paper, block-wise absmax scaling.  Per block: scale = max |x| (stored as

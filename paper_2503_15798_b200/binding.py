@@ -33,6 +33,7 @@ EXPORTS = (
     "mole_status_string", "mole_last_cuda_error", "mole_version", "mole_plan", "mole_variant", "mole_reload_debug_env",
     "mole_build_lut", "mole_build_lut_scratch_bytes", "mole_table_file_write", "mole_table_file_info", "mole_table_file_read", "mole_table_file_read_rows",
     "mole_decode_step_args", "mole_offload_create_ex", "mole_offload_set_hot_rows", "mole_offload_hot_hits", "mole_nf_codebook", "mole_quant_record_bytes", "mole_quantize_lut",
+    "mole_prefetch_rows",
 )
 
 
@@ -133,6 +134,7 @@ def lib() -> ctypes.CDLL:
         L.mole_nf_codebook.argtypes = [c_int, POINTER(ctypes.c_float)]
         L.mole_quant_record_bytes.argtypes = [c_int, c_int, c_int, c_int, POINTER(c_int64)]
         L.mole_quantize_lut.argtypes = [vp, vp, c_int64, c_int, c_int, c_int, c_int, vp]
+        L.mole_prefetch_rows.argtypes = [vp, c_int, vp, c_int64, c_int, c_int, c_int, c_int, c_int, ctypes.c_uint32, vp]
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is not c_char_p:
@@ -349,6 +351,17 @@ def decode_step_host(hidden_host, ids_host, out_host, dev_hidden, dev_ids, dev_o
                                        w_routers.stride(0) * w_routers.element_size(), _ptr(status), L, M, 1, N, d,
                                        V, tag, _stream(stream)), "mole_decode_step_host")
     return out_host
+
+
+def prefetch_rows(ids, luts, layers: int = 0, first_layer: int = 0, stream=None):
+    """mole_prefetch_rows: an L2 prefetch of the rows of `ids` in `layers` tables of luts [L][V][N][d] from
+    first_layer on (all of them by default).  A hint; no result changes."""
+    L, V, N, d = luts.shape
+    n = layers if layers > 0 else L - first_layer
+    flags = FLAG_IDS_INT64 if ids.dtype == torch.int64 else 0
+    _check(lib().mole_prefetch_rows(_ptr(ids), ids.numel(), ctypes.c_void_p(luts.data_ptr() + first_layer * luts.stride(0) * luts.element_size()),
+                                    luts.stride(0) * luts.element_size(), n, N, d, V, _dtype_tag(luts), flags, _stream(stream)),
+           "mole_prefetch_rows")
 
 
 def dedup_ids(ids, V: int, scratch, uniq, slot, count, status=None, stream=None):

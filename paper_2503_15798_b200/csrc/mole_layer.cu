@@ -771,6 +771,23 @@ int launch_step(const StepLaunch &a)
     return MOLE_OK;
 }
 
+// One thread per (token, layer): an L2 prefetch of the token's N rows of that layer's table, in pieces of at most
+// 32 KB.  A hint: nothing is written, nothing waits for it.
+constexpr uint32_t kPrefetchPiece = 32 * 1024;
+__global__ void mole_prefetch_rows_kernel(const void *ids, long long M, const unsigned char *lut_base, long long lut_stride,
+                                          long long row_bytes, long long rows, int ids64)
+{
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= M) return;
+    const long long id = ids64 ? static_cast<const long long *>(ids)[t] : static_cast<long long>(static_cast<const int *>(ids)[t]);
+    if (id < 0 || id >= rows) return;
+    const unsigned char *row = lut_base + static_cast<size_t>(blockIdx.y) * lut_stride + static_cast<size_t>(id) * row_bytes;
+    for (long long off = 0; off < row_bytes; off += kPrefetchPiece) {
+        const long long left = row_bytes - off;
+        bulk_prefetch_l2(row + off, static_cast<uint32_t>(left < kPrefetchPiece ? left : kPrefetchPiece));
+    }
+}
+
 static int check_common(const void *hidden, const void *ids, const void *lut, const void *w_router, const void *out,
                         const void *residual, int B, int T, int N, int d, int V, int dtype)
 {
@@ -1069,6 +1086,26 @@ static int sms_or_nominal()
         sms = kNumSMs;
     }
     return sms;
+}
+
+int mole_prefetch_rows(const void *ids, int M, const void *lut_base, int64_t lut_layer_stride_bytes, int layers, int N, int d, int V,
+                       int dtype, uint32_t flags, void *stream)
+{
+    if (dtype != MOLE_DTYPE_BF16 && dtype != MOLE_DTYPE_F32) return MOLE_ERR_INVALID_ARG;
+    if (flags & ~MOLE_FLAG_IDS_INT64) return MOLE_ERR_INVALID_ARG;
+    if (M < 0 || layers < 0) return MOLE_ERR_INVALID_ARG;
+    const int vec = 16 / elem_bytes(dtype);
+    if (N < 1 || N > kMaxN || V < 1 || d < vec || d % vec != 0) return MOLE_ERR_UNSUPPORTED_SHAPE;
+    if (M == 0 || layers == 0) return MOLE_OK;
+    if (layers > 65535) return MOLE_ERR_TOO_LARGE;
+    if (!ids || !lut_base || !aligned16(lut_base) || (lut_layer_stride_bytes & 15)) return MOLE_ERR_INVALID_ARG;
+    const long long row_bytes = static_cast<long long>(N) * d * elem_bytes(dtype);
+    const int threads = 128;
+    dim3 grid(static_cast<unsigned>((M + threads - 1) / threads), static_cast<unsigned>(layers));
+    mole_prefetch_rows_kernel<<<grid, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        ids, M, static_cast<const unsigned char *>(lut_base), lut_layer_stride_bytes, row_bytes, V, (flags & MOLE_FLAG_IDS_INT64) ? 1 : 0);
+    MOLE_CUDA_TRY(cudaGetLastError());
+    return MOLE_OK;
 }
 
 int mole_plan(int M, int L, int N, int d, int dtype, int d_split, int *out_d_split, int *out_threads, int *out_smem_bytes,

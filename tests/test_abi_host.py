@@ -193,6 +193,13 @@ def test_decode_step_and_offload_argument_checks(lib):
     assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG
     sa.norm_eps, sa.flags = 1e-5, 1  # only MOLE_FLAG_CHAIN is a flag of a step
     assert lib.mole_decode_step_args(ctypes.byref(sa)) == binding.ERR_INVALID_ARG
+    pf = lib.mole_prefetch_rows  # the L2 hint validates like the layer it serves
+    assert pf(good, 4, good, 16, 2, 16, 768, 100, 0, 4, None) == binding.ERR_INVALID_ARG        # unknown flag
+    assert pf(good, 4, good + 8, 16, 2, 16, 768, 100, 0, 0, None) == binding.ERR_INVALID_ARG    # table not 16-byte aligned
+    assert pf(good, 4, good, 24, 2, 16, 768, 100, 0, 0, None) == binding.ERR_INVALID_ARG        # layer stride not a multiple of 16
+    assert pf(good, 4, good, 16, 2, 16, 772, 100, 0, 0, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert pf(good, 4, good, 16, 70000, 16, 768, 100, 0, 0, None) == binding.ERR_TOO_LARGE
+    assert pf(None, 0, None, 0, 2, 16, 768, 100, 0, 0, None) == binding.OK                      # nothing to do
     dd = lib.mole_dedup_ids
     assert dd(good, -1, 10, good, good, good, good, None, None) == binding.ERR_INVALID_ARG
     assert dd(good, (1 << 20) + 1, 10, good, good, good, good, None, None) == binding.ERR_TOO_LARGE

@@ -413,3 +413,26 @@ def test_decode_step_host_round_trip(pinned):
     assert torch.equal(out_host, want.cpu())
     untouched = bool((dev[0] == 777.0).all()) and bool((dev_ids == -5).all())
     assert untouched == pinned
+
+
+@pytest.mark.parametrize("wide", [False, True])
+def test_prefetch_rows_is_a_hint(wide):
+    """mole_prefetch_rows before a step: the same bits as without it; ids outside the table are skipped (the
+    layer reports them as before); int64 ids."""
+    M, N, d, L, V = (40, 32, 2048, 2, 50) if wide else (70, 16, 768, 3, 300)
+    g = torch.Generator().manual_seed(9)
+    luts = torch.empty(L, V, N, d).normal_(0, 0.05, generator=g).to(torch.bfloat16).to(DEV)
+    wrs = torch.empty(L, d, N).normal_(0, 0.02, generator=g).to(torch.bfloat16).to(DEV)
+    hidden = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16).to(DEV)
+    ids = torch.randint(0, V, (M,), generator=g, dtype=torch.int32)
+    ids[3], ids[M - 1] = -1, V + 5
+    ids = ids.to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    want = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == mole.STATUS_BAD_ID
+    mole.prefetch_rows(ids, luts)
+    mole.prefetch_rows(ids.to(torch.int64), luts, layers=1, first_layer=L - 1)
+    got = mole.decode_step(hidden, ids, luts, wrs, torch.empty_like(hidden), torch.empty_like(hidden), status=status)
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
