@@ -441,7 +441,8 @@ MOLE_API int mole_offload_buffers(mole_offload_ctx *ctx, int buf, const int32_t 
 
 /* ---------------------------------------------------------------------------------------
  * Re-parameterisation (Sec. 3.3, Eq. 6-7): build a layer's table from its routed experts,
- *     LUT[i][j][:] = FFN_j(x_i),   FFN_j(x) = W2_j . gelu(W1_j . x)   (two matrices, no bias, exact erf GELU),
+ *     LUT[i][j][:] = FFN_j(x_i),   FFN_j(x) = W2_j . gelu(W1_j . x)   (two matrices, no bias, the erf GELU
+ *     x Phi(x), evaluated to within 4e-7 of its exact value before the rounding to bf16),
  *     x_i = Embedding(i), or RMSNorm(Embedding(i)) * norm_weight when norm_weight is given (the
  *     expert_layernorm of the training listing in App. A.1, folded into the table),
  * as one forward pass over the whole embedding matrix: two bf16 tensor-core GEMMs with fp32 accumulation;
