@@ -87,3 +87,33 @@ def test_builder_argument_checks():
     with pytest.raises(mole.MoleError) as e:  # d not a multiple of 8
         mole.build_lut(E[:, :60].contiguous().to(DEV), W1[:, :, :60].contiguous().to(DEV), W2[:, :60].contiguous().to(DEV))
     assert e.value.code in (mole.ERR_INVALID_ARG, mole.ERR_UNSUPPORTED_SHAPE)
+
+
+@pytest.mark.parametrize("V,N,d,D,norm", [(4096, 8, 256, 1024, False), (3000, 4, 768, 3072, True)])
+def test_many_tiles_per_block_sampled_rows(V, N, d, D, norm):
+    """Shapes with several hundred output tiles per GEMM, so that every persistent block walks many tiles (both
+    accumulators in tensor memory and the operand ring reused again and again, ragged last tile rows): sampled
+    ids' rows of the table against the oracle's builder run on those embedding rows alone."""
+    E, W1, W2 = _weights(V, N, d, D, seed=V + D)
+    gamma = None
+    if norm:
+        gamma = (1.0 + 0.2 * torch.empty(d).normal_(0, 1, generator=torch.Generator().manual_seed(2))).to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    lut = mole.build_lut(E.to(DEV), W1.to(DEV), W2.to(DEV), None if gamma is None else gamma.to(DEV), 1e-5, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rng = np.random.default_rng(V)
+    sample = np.unique(np.concatenate([rng.integers(0, V, 48), [0, 127, 128, V - 129, V - 1]]))
+    E64 = as_f64(E[sample])
+    if norm:
+        normed = np.stack([oracle.rmsnorm(E64[i], as_f64(gamma), 1e-5) for i in range(len(sample))])
+        E64 = as_f64(torch.from_numpy(normed).to(torch.bfloat16))
+    ref = oracle.build_lut(E64, as_f64(W1), as_f64(W2))
+    got = as_f64(lut[torch.from_numpy(sample).to(DEV)])
+    err = np.abs(got - ref)
+    bound = _bound(E64, W1, W2, ref)
+    if norm:
+        bound = bound + 2.0 ** -7 * np.abs(ref) + 2.0 ** -6
+    assert (err <= bound).all(), float((err / bound).max())
+    # every row was written: no tile skipped (rows of a zero-filled output would be exactly zero)
+    assert bool((lut.abs().amax(dim=(1, 2)) > 0).all())
