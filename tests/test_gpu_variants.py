@@ -37,7 +37,7 @@ CASES = {
     "step<bf16,16,1,2,1,0,0>": [(64, 16, 768, 1, False, AUTO), (3000, 16, 768, 1, False, AUTO)],
     "step<bf16,16,1,2,2,1,0>": [(256, 16, 1024, 1, False, AUTO), (400, 16, 1024, 1, False, AUTO)],
     "step<bf16,16,1,2,2,0,0>": [(64, 16, 1024, 1, False, AUTO), (2500, 16, 1024, 1, False, AUTO)],
-    "step<bf16,16,1,2,1,1,1>": [(256, 16, 768, 1, True, AUTO)],
+    "step<bf16,16,1,2,1,1,1>": [(256, 16, 768, 1, True, AUTO), (400, 16, 768, 1, True, AUTO)],  # the second: a one-slot ring
     "step<bf16,16,1,2,1,0,1>": [(700, 16, 768, 1, True, AUTO)],
     "step<bf16,16,1,2,2,1,1>": [(256, 16, 1024, 1, True, AUTO)],
     "step<bf16,16,1,2,2,0,1>": [(2500, 16, 1024, 1, True, AUTO)],
