@@ -219,6 +219,20 @@ struct Elem<__nv_bfloat16> {
         f[6] = __uint_as_float(v.w << 16);
         f[7] = __uint_as_float(v.w & 0xffff0000u);
     }
+    // acc[0..7] += g * (the 8 values of v): the weighted sum's inner step.  Two values per instruction on the
+    // packed fp32 pipe (fma.rn.f32x2: two independent IEEE fmas, the same bits as eight fmaf).
+    static __device__ __forceinline__ void fma_row(float (&acc)[8], const uint4 &v, float g)
+    {
+        const float2 g2 = make_float2(g, g);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 r = __ffma2_rn(g2, make_float2(__uint_as_float(w[k] << 16), __uint_as_float(w[k] & 0xffff0000u)),
+                                        make_float2(acc[2 * k], acc[2 * k + 1]));
+            acc[2 * k] = r.x;
+            acc[2 * k + 1] = r.y;
+        }
+    }
     // element i of an array in shared memory (32-bit shared address)
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds16(base + 2 * i) << 16); }
     // the same element as a raw 16-bit operand of the mixed-precision fma below
@@ -249,6 +263,13 @@ struct Elem<float> {
         f[1] = __uint_as_float(v.y);
         f[2] = __uint_as_float(v.z);
         f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ void fma_row(float (&acc)[4], const uint4 &v, float g)
+    {
+        acc[0] = fmaf(g, __uint_as_float(v.x), acc[0]);
+        acc[1] = fmaf(g, __uint_as_float(v.y), acc[1]);
+        acc[2] = fmaf(g, __uint_as_float(v.z), acc[2]);
+        acc[3] = fmaf(g, __uint_as_float(v.w), acc[3]);
     }
     static __device__ __forceinline__ float lds_scalar(uint32_t base, int i) { return __uint_as_float(lds32(base + 4 * i)); }
     typedef float H;

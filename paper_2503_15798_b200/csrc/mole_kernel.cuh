@@ -298,11 +298,8 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
                 float es[4] = {0.f, 0.f, 0.f, 0.f};  // their sum, four short chains instead of one long one
 #pragma unroll
                 for (int r = 0; r < UNR; ++r) {
-                    float vf[VEC];
-                    E::unpack(rv[r], vf);
                     es[r & 3] += gv[r];
-#pragma unroll
-                    for (int i = 0; i < VEC; ++i) acc[i] = fmaf(gv[r], vf[i], acc[i]);
+                    E::fma_row(acc, rv[r], gv[r]);
                 }
                 esum += (es[0] + es[1]) + (es[2] + es[3]);
             }
@@ -310,11 +307,8 @@ __device__ __forceinline__ void combine_item(uint32_t rows, uint32_t haddr, uint
             for (; j0 < je; ++j0) {  // tail
                 const uint4 rv = lds128(rows + 16u * (j0 * ngrp + gg));
                 const float g = __uint_as_float(lds32(gates + 4u * j0));
-                float vf[VEC];
-                E::unpack(rv, vf);
                 esum += g;
-#pragma unroll
-                for (int i = 0; i < VEC; ++i) acc[i] = fmaf(g, vf[i], acc[i]);
+                E::fma_row(acc, rv, g);
             }
         }
         int base = 0;
@@ -428,12 +422,7 @@ struct RowSums {
 #pragma unroll
             for (int i = 0; i < GPL; ++i)
 #pragma unroll
-                for (int r = 0; r < UNR; ++r) {
-                    float vf[VEC];
-                    E::unpack(rv[i][r], vf);
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) acc[i][e] = fmaf(gv[r], vf[e], acc[i][e]);
-                }
+                for (int r = 0; r < UNR; ++r) E::fma_row(acc[i], rv[i][r], gv[r]);
         }
 #pragma unroll 1
         for (; j0 < ne; ++j0) {  // tail (and every chunk of fewer than UNR experts)
@@ -444,10 +433,7 @@ struct RowSums {
                 const int grp = tid + i * nc;
                 const int gg = grp < ngrp ? grp : ngrp - 1;
                 const uint4 rv = lds128(rows + 16u * (j0 * ngrp + gg));
-                float vf[VEC];
-                E::unpack(rv, vf);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) acc[i][e] = fmaf(g, vf[e], acc[i][e]);
+                E::fma_row(acc[i], rv, g);
             }
         }
     }
