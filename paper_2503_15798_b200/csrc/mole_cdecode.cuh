@@ -247,10 +247,13 @@ __global__ void __cluster_dims__(CS, 1, 1) __launch_bounds__(kClusterThreads) mo
     for (int j = 0; j < N; ++j) {
         const float g = __shfl_sync(0xffffffffu, e, j);
         es[j & 3] += g;
-        a0 = fmaf(g, bf16_bits_to_float(rv[j].x & 0xffffu), a0);
-        a1 = fmaf(g, __uint_as_float(rv[j].x & 0xffff0000u), a1);
-        a2 = fmaf(g, bf16_bits_to_float(rv[j].y & 0xffffu), a2);
-        a3 = fmaf(g, __uint_as_float(rv[j].y & 0xffff0000u), a3);
+        // two values per fma on the packed fp32 pipe (two independent IEEE fmas: the bits of four fmaf)
+        const float2 g2 = make_float2(g, g);
+        const float2 lo = __ffma2_rn(g2, make_float2(bf16_bits_to_float(rv[j].x & 0xffffu), __uint_as_float(rv[j].x & 0xffff0000u)),
+                                     make_float2(a0, a1));
+        const float2 hi = __ffma2_rn(g2, make_float2(bf16_bits_to_float(rv[j].y & 0xffffu), __uint_as_float(rv[j].y & 0xffff0000u)),
+                                     make_float2(a2, a3));
+        a0 = lo.x, a1 = lo.y, a2 = hi.x, a3 = hi.y;
     }
     const float esum = (es[0] + es[1]) + (es[2] + es[3]);
     const float inv = __frcp_rn(esum);
