@@ -105,3 +105,32 @@ def test_unit_weight_and_unit_rms_rows_match_the_plain_router():
     torch.cuda.synchronize()
     assert np.abs(as_f64(gates_n) - as_f64(gates_p)).max() <= 1e-6
     assert np.abs(as_f64(out_n) - as_f64(out_p)).max() <= 2.0 ** -7
+
+
+@pytest.mark.parametrize("norm", [False, True])
+def test_cluster_kernel_with_a_separate_residual(norm):
+    """d = 2048: the one-token-per-cluster kernel with a residual that is not the hidden state (the App. A.2 layer
+    adds the shared expert's output to it), with and without the RMSNorm in front of the router, gates included."""
+    M, N, d, V = 19, 32, 2048, 45
+    hidden, ids, lut, wr = rand_case(M, N, d, V, seed=77)
+    g = torch.Generator().manual_seed(3)
+    residual = torch.empty(M, d).normal_(0, 1, generator=g).to(torch.bfloat16)
+    assert mole.variant(M, N, d, norm=norm)[0] == f"cdecode<32,4,{int(norm)}>"
+    if norm:
+        gamma = (1.0 + 0.2 * torch.empty(d).normal_(0, 1, generator=g)).to(torch.bfloat16)
+        ref, gref, normed = oracle_norm_layer(hidden, ids, lut, wr, gamma, 1e-5, residual=residual)
+        out, gates, status = run(hidden, ids, lut, wr, gamma, 1e-5, residual=residual)
+        assert status == 0
+        check_gates_normed_router(gates, gref, normed, wr)
+        check_out_after_flips(out, ref, gates, gref, lut)
+    else:
+        ref, gref, bad = oracle.layer_lookup(bits(hidden), ids.cpu().numpy(), bits(lut), bits(wr), residual=bits(residual))
+        gates = torch.zeros(M, N, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        out = mole.layer_forward(hidden.to(DEV), ids.to(DEV), lut.to(DEV), wr.to(DEV), gates_out=gates, status=status,
+                                 residual=residual.to(DEV))
+        torch.cuda.synchronize()
+        assert bad == 0 and int(status.item()) == 0
+        assert np.abs(as_f64(gates) - gref).max() <= 1e-5
+        err = np.abs(as_f64(out) - ref)
+        assert (err <= 2.0 ** -8 * np.abs(ref) + 2e-5).all(), float(err.max())
