@@ -66,12 +66,12 @@ FUSED_TRAFFIC = {
 }
 
 
-def offload_groups(L: int, M: int, row_bytes: int) -> int:
+def offload_groups(L: int, M: int, row_bytes: int, hot: bool = False) -> int:
     """Groups of layers mole_offload_decode_step forms on a context of OFFLOAD_CONTEXT_TOKENS tokens (one
     fetch launch and one fused layer launch per group): as many layers as the staging area holds, but at
-    least three groups unless the whole step's rows are at most 1 MB."""
+    least three groups unless the whole step's rows are at most 256 KB (1 MB with a hot-row cache)."""
     g = min(L, max(1, OFFLOAD_CONTEXT_TOKENS // M))
-    if M * row_bytes * L > (1 << 20):
+    if M * row_bytes * L > ((1 << 20) if hot else (1 << 18)):
         g = min(g, (L + 2) // 3)
     return -(-L // g)
 
@@ -115,10 +115,11 @@ def timed_launch_shapes():
                 add(f"{name} batch {M} chained, {tag} table", M, sh, 1, fmt=fmt, block=QUANT_BLOCKS[name][tag])
     sh = inputs.SHAPES["410m"]
     for M in OFFLOAD_BATCHES:
-        groups = offload_groups(sh.L, M, sh.row_bytes)
-        per = -(-sh.L // groups)
-        for L in {per, sh.L - per * (groups - 1)}:
-            add(f"410m offload batch {M}, group of {L} layers", M, sh, L, kernel=1)
+        for hot in (False, True):
+            groups = offload_groups(sh.L, M, sh.row_bytes, hot)
+            per = -(-sh.L // groups)
+            for L in {per, sh.L - per * (groups - 1)}:
+                add(f"410m offload batch {M}, group of {L} layers", M, sh, L, kernel=1)
         for fmt, tag in ((1, "nf4"), (2, "nf3")):
             add(f"410m offload batch {M}, {tag} records", M, sh, 1, fmt=fmt, block=QUANT_BLOCKS["410m"][tag])
     return shapes
