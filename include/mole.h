@@ -414,7 +414,7 @@ MOLE_API int mole_layer_forward_offload(mole_offload_ctx *ctx, int buf, const vo
  * stream (the paper issues the row transfer first so that it overlaps the rest of the layer, App. A.2
  * listing).  A staging area holds max_tokens rows, so with B*T tokens one fetch launch brings the rows
  * of up to max_tokens / (B*T) consecutive layers (at least one; at least three groups per step once the
- * step's rows exceed 1 MB, so that fetches overlap layers), and one fused launch then runs those layers:
+ * step's rows exceed 256 KB (1 MB with a hot-row cache), so that fetches overlap layers), and one fused launch then runs those layers:
  * a context created for the largest batch serves small batches with few, large fetches and few launches.
  * Needs a context with n_buffers >= 2.
  *   hidden_in device [M][d], read only;  out device [M][d] final result;  tmp device [M][d]
